@@ -1,0 +1,101 @@
+"""ctypes front-end of the fp64 recurrence oracle (``qdelta_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY (see the package docstring).  Every array is converted
+to contiguous float64 before the call; layouts are token-major:
+q,k [B,T,H,dk]; v,o,dO [B,T,H,dv]; beta,alpha,lam [B,T,H]; states [B,H,dk,dv].
+"""
+import ctypes
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(_build.build())
+        dp = ctypes.POINTER(ctypes.c_double)
+        lib.qd_oracle_fwd.restype = ctypes.c_int
+        lib.qd_oracle_fwd.argtypes = [ctypes.c_int] * 5 + [dp] * 9
+        lib.qd_oracle_bwd.restype = ctypes.c_int
+        lib.qd_oracle_bwd.argtypes = [ctypes.c_int] * 6 + [dp] * 16
+        lib.qd_oracle_max_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _c(a, shape=None):
+    if a is None:
+        return None
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    if shape is not None:
+        assert a.shape == tuple(shape), (a.shape, shape)
+    return a
+
+
+def _p(a):
+    if a is None:
+        return ctypes.POINTER(ctypes.c_double)()
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def max_threads() -> int:
+    return int(_load().qd_oracle_max_threads())
+
+
+def forward(q, k, v, beta, alpha=None, lam=None, h0=None):
+    """Token-by-token Q-Delta recurrence (Section 3.3.1).  Returns (o, hT)."""
+    lib = _load()
+    q = _c(q)
+    B, T, H, dk = q.shape
+    dv = np.shape(v)[-1]
+    k = _c(k, (B, T, H, dk)); v = _c(v, (B, T, H, dv))
+    beta = _c(beta, (B, T, H)); alpha = _c(alpha, (B, T, H)); lam = _c(lam, (B, T, H))
+    h0 = _c(h0, (B, H, dk, dv))
+    o = np.empty((B, T, H, dv), np.float64)
+    hT = np.empty((B, H, dk, dv), np.float64)
+    rc = lib.qd_oracle_fwd(B, T, H, dk, dv, _p(q), _p(k), _p(v), _p(beta), _p(alpha),
+                           _p(lam), _p(h0), _p(o), _p(hT))
+    if rc != 0:
+        raise RuntimeError("qd_oracle_fwd failed: %d" % rc)
+    return o, hT
+
+
+def backward(q, k, v, beta, alpha, lam, h0, dO, dhT=None, ckpt=64):
+    """Reverse pass of the recurrence for L = <o,dO> + <hT,dhT>.
+
+    Returns dict(dq, dk, dv, dbeta, dalpha, dlam, dh0); dalpha is the derivative
+    with respect to alpha itself.  alpha=None means alpha==1, lam=None means 0
+    (their gradients are still returned)."""
+    lib = _load()
+    q = _c(q)
+    B, T, H, dk = q.shape
+    dv = np.shape(v)[-1]
+    k = _c(k, (B, T, H, dk)); v = _c(v, (B, T, H, dv))
+    beta = _c(beta, (B, T, H)); alpha = _c(alpha, (B, T, H)); lam = _c(lam, (B, T, H))
+    h0 = _c(h0, (B, H, dk, dv)); dO = _c(dO, (B, T, H, dv)); dhT = _c(dhT, (B, H, dk, dv))
+    out = dict(dq=np.empty((B, T, H, dk)), dk=np.empty((B, T, H, dk)),
+               dv=np.empty((B, T, H, dv)), dbeta=np.empty((B, T, H)),
+               dalpha=np.empty((B, T, H)), dlam=np.empty((B, T, H)),
+               dh0=np.empty((B, H, dk, dv)))
+    rc = lib.qd_oracle_bwd(B, T, H, dk, dv, int(ckpt), _p(q), _p(k), _p(v), _p(beta),
+                           _p(alpha), _p(lam), _p(h0), _p(dO), _p(dhT),
+                           _p(out["dq"]), _p(out["dk"]), _p(out["dv"]), _p(out["dbeta"]),
+                           _p(out["dalpha"]), _p(out["dlam"]), _p(out["dh0"]))
+    if rc != 0:
+        raise RuntimeError("qd_oracle_bwd failed: %d" % rc)
+    return out
+
+
+def decode(state, q, k, v, beta, alpha=None, lam=None):
+    """`steps` single-token updates of [Bn,H,dk,dv] states.
+
+    q,k [steps,Bn,H,dk], v [steps,Bn,H,dv], coefficients [steps,Bn,H].
+    Returns (o [steps,Bn,H,dv], final state).  It is the forward recurrence
+    with time as the leading axis."""
+    tr = lambda a: None if a is None else np.moveaxis(np.asarray(a, np.float64), 0, 1)
+    o, hT = forward(tr(q), tr(k), tr(v), tr(beta), tr(alpha), tr(lam), state)
+    return np.moveaxis(o, 1, 0), hT
