@@ -1,0 +1,138 @@
+/*
+ * qdelta.h -- C ABI of the B200 (sm_100a) Q-Delta library.
+ *
+ * Q-Delta (arXiv 2606.08804) evolves a d_k x d_v associative state per (batch, head):
+ *
+ *     x_t = k_t + lambda_t q_t                                   (Section 3.3.2, definition of x_t)
+ *     S_t = alpha_t S_{t-1} (I - beta_t x_t k_t^T) + beta_t v_t k_t^T      (Section 3.3.1, final rule)
+ *     o_t = S_t q_t
+ *
+ * This library keeps the state transposed, h_t = S_t^T in R^{d_k x d_v}, row-major, fp32:
+ *
+ *     h_t = alpha_t h_{t-1} + k_t (beta_t (v_t - alpha_t h_{t-1}^T x_t))^T ,   o_t = h_t^T q_t .
+ *
+ * Conventions that hold for every entry point
+ *   - All tensor pointers are DEVICE pointers, dense and contiguous, token-major:
+ *       q, k            [B, T, H, dk]          v, o, dO          [B, T, H, dv]
+ *       beta, alpha, lambda (and their gradients) [B, T, H]
+ *       states h0, hT, dhT, dh0                 [B, H, dk, dv]  fp32 always
+ *     q,k,v,o,dO,dq,dk,dv,beta,alpha,lambda are stored in `dtype` (fp32 or bf16);
+ *     dbeta,dalpha,dlambda and every state are fp32.
+ *   - The caller owns every buffer, including the workspace whose size it queries.  The library
+ *     never allocates, frees or synchronises; all work is enqueued on `stream`.
+ *   - Inputs are read-only.  Outputs are fully overwritten.  Pointers must be 16-byte aligned.
+ *   - Coefficient domains: beta, lambda in [0,1], alpha in (0,1] (Section 3.3.1); not checked on device.
+ *   - Return value: QD_OK, or an error code reported synchronously; on error nothing was enqueued.
+ *     Conditions found on the device (a bounded wait that ran out) are written to the first
+ *     32-bit word of the workspace and can be read with qdelta_workspace_status after the
+ *     caller has synchronised the stream.
+ *   - Supported shapes: chunk = 64, T a multiple of chunk, dk and dv in {64, 128}.
+ */
+#ifndef QDELTA_H_
+#define QDELTA_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    QD_OK = 0,
+    QD_ERR_INVALID_ARG = 1,   /* null required pointer, non-positive size, T % chunk != 0, misaligned pointer */
+    QD_ERR_UNSUPPORTED = 2,   /* (dk, dv, chunk, dtype) outside the supported set */
+    QD_ERR_WORKSPACE = 3,     /* workspace null or smaller than qdelta_chunk_workspace_bytes */
+    QD_ERR_CUDA = 4,          /* a CUDA runtime call (launch, attribute) failed */
+    QD_ERR_TIMEOUT = 5        /* device side: a bounded wait expired (see qdelta_workspace_status) */
+} qd_status;
+
+typedef enum { QD_F32 = 0, QD_BF16 = 1 } qd_dtype;
+
+/* flags of qdelta_chunk_fwd / qdelta_chunk_bwd */
+enum {
+    QD_FWD_SAVE_FOR_BWD = 1,  /* fwd: also keep the per-chunk states etc. in a backward-sized workspace */
+    QD_BWD_REUSE_FWD = 2      /* bwd: the workspace still holds what a QD_FWD_SAVE_FOR_BWD forward of the
+                                 SAME inputs left there; skip the recomputation */
+};
+
+typedef struct {
+    int B, T, H;      /* batch, tokens per sequence, heads */
+    int dk, dv;       /* key/query and value head dimensions */
+    int chunk;        /* chunk length C of the chunkwise form; 64 */
+    int dtype;        /* qd_dtype of q,k,v,beta,alpha,lambda,o,dO,dq,dk,dv */
+} qd_shape;
+
+typedef struct CUstream_st *qd_stream;   /* a cudaStream_t */
+
+/* Bytes of device workspace the chunkwise calls need for this shape (0 on invalid shape).
+ * for_backward != 0: the size qdelta_chunk_bwd (and a QD_FWD_SAVE_FOR_BWD forward) needs. */
+size_t qdelta_chunk_workspace_bytes(const qd_shape *shape, int for_backward);
+
+/*
+ * Chunkwise-parallel forward (Section 3.3.2: chunk expansion, extended WY representation,
+ * UT transform, chunk-level state update and output).  The result equals the token-by-token
+ * recurrence of Section 3.3.1 up to rounding:
+ *     o   [B,T,H,dv]   o_t = h_t^T q_t           (read-out from the post-update state)
+ *     hT  [B,H,dk,dv]  final state, fp32         (NULL: not returned)
+ * alpha NULL means alpha == 1 (no forgetting); lambda NULL means lambda == 0 (the gated delta rule);
+ * h0 NULL means a zero initial state.
+ */
+int qdelta_chunk_fwd(const qd_shape *shape,
+                     const void *q, const void *k, const void *v,
+                     const void *beta, const void *alpha, const void *lambda,
+                     const float *h0, void *o, float *hT,
+                     void *workspace, size_t workspace_bytes, unsigned flags, qd_stream stream);
+
+/*
+ * Backward of qdelta_chunk_fwd for the scalar  L = sum_t <o_t, dO_t> + <h_T, dhT>_F.
+ * The paper prints no backward pass; this is the exact gradient of the chunk equations of
+ * Section 3.3.2 (equivalently of the recurrence of Section 3.3.1).
+ *     dq, dk [B,T,H,dk], dv [B,T,H,dv] in `dtype`;  dbeta, dalpha, dlambda [B,T,H] fp32;
+ *     dh0 [B,H,dk,dv] fp32 (NULL: skipped).  dalpha is the derivative with respect to alpha itself.
+ * dhT NULL means zero.  alpha / lambda / h0 NULL as in the forward (dalpha / dlambda are still
+ * written when their pointers are non-NULL; they may be NULL only if the input was NULL).
+ */
+int qdelta_chunk_bwd(const qd_shape *shape,
+                     const void *q, const void *k, const void *v,
+                     const void *beta, const void *alpha, const void *lambda,
+                     const float *h0, const void *dO, const float *dhT,
+                     void *dq, void *dk, void *dv,
+                     float *dbeta, float *dalpha, float *dlambda, float *dh0,
+                     void *workspace, size_t workspace_bytes, unsigned flags, qd_stream stream);
+
+/*
+ * One token of the recurrence of Section 3.3.1 for B*H independent states, in place:
+ *     state [B,H,dk,dv] fp32  h <- alpha h + k (beta (v - alpha h^T (k + lambda q)))^T
+ *     o     [B,H,dv]          o = h_new^T q
+ * q,k [B,H,dk], v [B,H,dv], beta/alpha/lambda [B,H] in `dtype` (alpha, lambda may be NULL).
+ * `state` is the only in/out buffer.  Needs no workspace.
+ */
+int qdelta_recurrent_step(int B, int H, int dk, int dv, int dtype,
+                          const void *q, const void *k, const void *v,
+                          const void *beta, const void *alpha, const void *lambda,
+                          float *state, void *o, qd_stream stream);
+
+/* Copies the device status word of `workspace` to *status_out (a qd_status) with a blocking
+ * 4-byte device-to-host copy on `stream`.  Returns QD_OK or QD_ERR_CUDA / QD_ERR_INVALID_ARG. */
+int qdelta_workspace_status(const void *workspace, int *status_out, qd_stream stream);
+
+/*
+ * Per-kernel timing aid for benchmarks (the paper has no counterpart).  While enabled, every kernel
+ * the entry points enqueue is bracketed by two CUDA events recorded on the caller's stream;
+ * qdelta_profile_read waits for the recorded events, adds their elapsed times to per-stage totals and
+ * returns the total milliseconds and number of launches of `stage` (reset != 0 clears that total).
+ * Stages are numbered 0 .. qdelta_profile_stage_count()-1; qdelta_profile_stage_name names them.
+ * Events are created on first use and reused.  Not thread-safe; off by default.
+ */
+int qdelta_profile_enable(int on);
+int qdelta_profile_stage_count(void);
+const char *qdelta_profile_stage_name(int stage);
+int qdelta_profile_read(int stage, double *total_ms, long long *launches, int reset);
+
+/* Human-readable name of a qd_status. */
+const char *qdelta_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QDELTA_H_ */

@@ -1,0 +1,107 @@
+// Single-token recurrent step (Section 3.3.1, final update rule and read-out), in place:
+//   x = k + lambda q ;  p = alpha h^T x ;  delta = beta (v - p) ;  h <- alpha h + k delta^T ;
+//   o = h_new^T q = alpha h^T q + (k.q) delta .
+// The step is bound by HBM traffic: the fp32 state is read once and written once.  A CTA owns
+// DVS columns of one state (columns evolve independently); every thread keeps its part of the
+// slice in registers between the read and the write, all loads are issued before the first use.
+#include "internal.h"
+
+namespace qd {
+namespace {
+
+template <typename IO, int DK, int DVS, int NT>
+__global__ void __launch_bounds__(NT) k_decode(int dv, const IO* __restrict__ q, const IO* __restrict__ k,
+                                               const IO* __restrict__ v, const IO* __restrict__ beta,
+                                               const IO* __restrict__ alpha, const IO* __restrict__ lam,
+                                               float* __restrict__ state, IO* __restrict__ o) {
+    constexpr int C4 = DVS / 4;          // threads across one row of the slice
+    constexpr int RP = NT / C4;          // rows per pass
+    constexpr int NP = DK / RP;          // passes (float4 registers per thread)
+    static_assert(NT % C4 == 0 && DK % RP == 0, "bad decode tiling");
+    __shared__ float sx[DK], sq[DK], sk[DK];
+    __shared__ float redx[RP][DVS], redq[RP][DVS];
+    __shared__ float sdelta[DVS];
+    __shared__ float skq[NT / 32];
+    const int nsl = dv / DVS, bh = blockIdx.x / nsl, j0 = (blockIdx.x % nsl) * DVS, tid = threadIdx.x;
+    const int c4 = tid % C4, rg = tid / C4;
+
+    // issue all state loads first
+    float4* base = reinterpret_cast<float4*>(state + (size_t)bh * DK * dv + j0) + c4;
+    const int rstride = dv / 4;
+    float4 h[NP];
+#pragma unroll
+    for (int pz = 0; pz < NP; ++pz) h[pz] = __ldcs(base + (size_t)(pz * RP + rg) * rstride);
+
+    const float be = ld(beta, bh);
+    const float al = alpha ? ld(alpha, bh) : 1.f;
+    const float la = lam ? ld(lam, bh) : 0.f;
+    float kq = 0.f;
+    for (int i = tid; i < DK; i += NT) {
+        const float qi = ld(q, (size_t)bh * DK + i), ki = ld(k, (size_t)bh * DK + i);
+        sq[i] = qi; sk[i] = ki; sx[i] = fmaf(la, qi, ki);
+        kq = fmaf(ki, qi, kq);
+    }
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) kq += __shfl_xor_sync(0xffffffffu, kq, s);
+    if ((tid & 31) == 0) skq[tid >> 5] = kq;
+    __syncthreads();
+
+    float4 ax = make_float4(0.f, 0.f, 0.f, 0.f), aq = ax;
+#pragma unroll
+    for (int pz = 0; pz < NP; ++pz) {
+        const float xi = sx[pz * RP + rg], qi = sq[pz * RP + rg];
+        ax.x = fmaf(h[pz].x, xi, ax.x); ax.y = fmaf(h[pz].y, xi, ax.y);
+        ax.z = fmaf(h[pz].z, xi, ax.z); ax.w = fmaf(h[pz].w, xi, ax.w);
+        aq.x = fmaf(h[pz].x, qi, aq.x); aq.y = fmaf(h[pz].y, qi, aq.y);
+        aq.z = fmaf(h[pz].z, qi, aq.z); aq.w = fmaf(h[pz].w, qi, aq.w);
+    }
+    *reinterpret_cast<float4*>(&redx[rg][c4 * 4]) = ax;
+    *reinterpret_cast<float4*>(&redq[rg][c4 * 4]) = aq;
+    __syncthreads();
+    if (tid < DVS) {
+        float rx = 0.f, rq = 0.f, kqt = 0.f;
+#pragma unroll
+        for (int r = 0; r < RP; ++r) { rx += redx[r][tid]; rq += redq[r][tid]; }
+#pragma unroll
+        for (int w = 0; w < NT / 32; ++w) kqt += skq[w];
+        const float dl = be * (ld(v, (size_t)bh * dv + j0 + tid) - al * rx);
+        sdelta[tid] = dl;
+        st(o, (size_t)bh * dv + j0 + tid, fmaf(al, rq, kqt * dl));
+    }
+    __syncthreads();
+    const float4 dl = *reinterpret_cast<const float4*>(&sdelta[c4 * 4]);
+#pragma unroll
+    for (int pz = 0; pz < NP; ++pz) {
+        const float ki = sk[pz * RP + rg];
+        float4 r;
+        r.x = fmaf(al, h[pz].x, ki * dl.x); r.y = fmaf(al, h[pz].y, ki * dl.y);
+        r.z = fmaf(al, h[pz].z, ki * dl.z); r.w = fmaf(al, h[pz].w, ki * dl.w);
+        __stcs(base + (size_t)(pz * RP + rg) * rstride, r);
+    }
+}
+
+template <typename IO, int DK>
+cudaError_t launch(int BH, int dv, const void* q, const void* k, const void* v, const void* beta,
+                   const void* alpha, const void* lam, float* state, void* o, cudaStream_t stream) {
+    constexpr int DVS = 64, NT = 128;
+    dim3 grid((unsigned)(dv / DVS) * (unsigned)BH);
+    k_decode<IO, DK, DVS, NT><<<grid, NT, 0, stream>>>(dv, (const IO*)q, (const IO*)k, (const IO*)v,
+                                                       (const IO*)beta, (const IO*)alpha, (const IO*)lam,
+                                                       state, (IO*)o);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
+                        const void* beta, const void* alpha, const void* lam, float* state, void* o,
+                        cudaStream_t stream) {
+    if (dtype == QD_BF16) {
+        if (dk == 128) return launch<__nv_bfloat16, 128>(BH, dv, q, k, v, beta, alpha, lam, state, o, stream);
+        return launch<__nv_bfloat16, 64>(BH, dv, q, k, v, beta, alpha, lam, state, o, stream);
+    }
+    if (dk == 128) return launch<float, 128>(BH, dv, q, k, v, beta, alpha, lam, state, o, stream);
+    return launch<float, 64>(BH, dv, q, k, v, beta, alpha, lam, state, o, stream);
+}
+
+}  // namespace qd

@@ -1,0 +1,78 @@
+// Internal declarations shared by the translation units of libqdelta.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/qdelta.h"
+
+namespace qd {
+
+constexpr int kChunk = 64;        // chunk length C of the chunkwise form
+constexpr int kSliceSimt = 32;    // d_v columns one CTA of the SIMT state chains owns
+
+// Byte offsets of the sections of the caller-provided workspace.  Every section starts on a
+// 256-byte boundary.  "io" sections are stored in the call's dtype.
+struct WsLayout {
+    size_t status;   // u32 status word (+ padding)
+    size_t g;        // fp32 [BH*T]        in-chunk cumulative log-decay g_r = sum_{i<=r} log alpha_i
+    size_t P;        // io   [BH*T*C]      Gamma o (Q K^T), causal incl. diagonal, row = token
+    size_t W;        // io   [BH*T*dk]     W<- = T diag(gamma) X
+    size_t U;        // io   [BH*T*dv]     U~  = T V
+    size_t fwd_end;
+    // backward only
+    size_t hs;       // fp32 [BH*N*dk*dv]  state at the entry of every chunk
+    size_t D;        // io   [BH*T*dv]     Delta = U~ - W<- h   (row r = delta_r of the recurrence)
+    size_t dhs;      // fp32 [BH*N*dk*dv]  gradient w.r.t. the state at the EXIT of every chunk
+    size_t dD;       // io   [BH*T*dv]     gradient w.r.t. Delta
+    size_t kdhd;     // fp32 [S][BH*T]     per d_v-slice partial of <(K-> dh)_r, Delta_r>
+    size_t dhh;      // fp32 [S][BH*N]     per d_v-slice partial of <dh, h>_F
+    size_t scratch;  // fp32 per-CTA scratch of the SIMT chunk backward
+    size_t bwd_end;
+    int nslices;
+    int bwd_ctas;
+};
+
+WsLayout ws_layout(const qd_shape& s);
+
+struct ChunkArgs {
+    qd_shape s;
+    const void *q, *k, *v, *beta, *alpha, *lam;
+    const float* h0;
+    void* o;
+    float* hT;
+    // backward
+    const void* dO;
+    const float* dhT;
+    void *dq, *dk, *dv;
+    float *dbeta, *dalpha, *dlam, *dh0;
+    char* ws;
+    WsLayout L;
+    bool save;       // forward: keep hs and D
+    cudaStream_t stream;
+};
+
+// SIMT fp32-arithmetic path (any supported dtype for storage)
+cudaError_t simt_prep(const ChunkArgs& a);        // g, P, W<-, U~
+cudaError_t simt_chain_fwd(const ChunkArgs& a);   // Delta, O, state chain (+ hs, D when a.save)
+cudaError_t simt_chain_bwd(const ChunkArgs& a);   // dDelta, dhs, dh0, scalar partials
+cudaError_t simt_chunk_bwd(const ChunkArgs& a);   // dq, dk, dv, dbeta, dalpha, dlambda
+
+cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
+                        const void* beta, const void* alpha, const void* lam, float* state, void* o,
+                        cudaStream_t stream);
+
+// ---- storage-dtype helpers -------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ float ld(const T* p, size_t i);
+template <> __device__ __forceinline__ float ld<float>(const float* p, size_t i) { return p[i]; }
+template <> __device__ __forceinline__ float ld<__nv_bfloat16>(const __nv_bfloat16* p, size_t i) {
+    return __bfloat162float(p[i]);
+}
+template <typename T> __device__ __forceinline__ void st(T* p, size_t i, float x);
+template <> __device__ __forceinline__ void st<float>(float* p, size_t i, float x) { p[i] = x; }
+template <> __device__ __forceinline__ void st<__nv_bfloat16>(__nv_bfloat16* p, size_t i, float x) {
+    p[i] = __float2bfloat16_rn(x);
+}
+
+}  // namespace qd

@@ -1,0 +1,156 @@
+"""GPU-vs-oracle parity of the chunkwise forward and backward (through the C ABI)."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2606_08804_b200 import inputs as gen
+import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def _fwd_check(cfg, d=None, pairs=None, check_status=True):
+    from paper_2606_08804_b200 import binding as qd
+    d = gen.make_chunk_inputs(cfg) if d is None else d
+    t = gu.dev_inputs(d, cfg.dtype)
+    o, hT, ws = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], chunk=cfg.chunk)
+    torch.cuda.synchronize()
+    if check_status:
+        assert qd.workspace_status(ws) == 0
+    if pairs is None:
+        ro, rh = gu.oracle_fwd(d)
+        eo, eh = gu.rel_err(o, ro), gu.rel_err(hT, rh)
+    else:
+        ro, rh = gu.oracle_fwd(gu.pick_sequences(d, pairs))
+        eo, eh = gu.rel_err(gu.pick_result(o, pairs), ro), gu.rel_err(gu.pick_result(hT, pairs, True), rh)
+    tol = gu.TOL[cfg.dtype]
+    assert eo <= tol and eh <= tol, (cfg.name, cfg.regime, eo, eh)
+    return eo, eh
+
+
+def _bwd_check(cfg, d=None, pairs=None, reuse=False):
+    from paper_2606_08804_b200 import binding as qd
+    d = gen.make_chunk_inputs(cfg) if d is None else d
+    t = gu.dev_inputs(d, cfg.dtype)
+    ws = None
+    if reuse:
+        o, hT, ws = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"],
+                                 chunk=cfg.chunk, save_for_bwd=True)
+    g = qd.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], t["dO"], t["dhT"],
+                     chunk=cfg.chunk, workspace=ws, reuse_fwd=reuse)
+    torch.cuda.synchronize()
+    sub = d if pairs is None else gu.pick_sequences(d, pairs)
+    ref = gu.oracle_bwd(sub)
+    tol = gu.TOL[cfg.dtype]
+    errs = {}
+    for n in ("dq", "dk", "dv", "dbeta", "dalpha", "dlam", "dh0"):
+        if g.get(n) is None:
+            continue
+        got = g[n] if pairs is None else gu.pick_result(g[n], pairs, n == "dh0")
+        errs[n] = gu.rel_err(got, ref[n])
+    assert all(e <= tol for e in errs.values()), (cfg.name, cfg.regime, errs)
+    return errs
+
+
+def test_cfg0_tiny_fp32_forward():
+    _fwd_check(gen.CONFIGS["cfg0"])
+
+
+@pytest.mark.parametrize("regime", gen.REGIMES)
+def test_small_fp32_forward_backward_regimes(regime):
+    cfg = replace(gen.CONFIGS["cfg0"], B=2, H=2, T=192, h0=True, backward=True, regime=regime, seed=3)
+    _fwd_check(cfg)
+    _bwd_check(cfg)
+
+
+@pytest.mark.parametrize("regime", gen.REGIMES)
+def test_small_bf16_forward_backward_regimes(regime):
+    cfg = replace(gen.CONFIGS["cfg2"], B=2, H=3, T=320, regime=regime, seed=5)
+    _fwd_check(cfg)
+    _bwd_check(cfg)
+    _bwd_check(cfg, reuse=True)
+
+
+def test_mixed_head_dims_fp32():
+    cfg = replace(gen.CONFIGS["cfg0"], B=1, H=2, T=128, dk=128, dv=64, h0=True, backward=True, seed=7)
+    _fwd_check(cfg)
+    _bwd_check(cfg)
+    cfg = replace(cfg, dk=64, dv=128)
+    _fwd_check(cfg)
+    _bwd_check(cfg)
+
+
+def test_single_chunk_and_optional_inputs():
+    from paper_2606_08804_b200 import binding as qd
+    cfg = replace(gen.CONFIGS["cfg2"], B=1, H=2, T=64, seed=9)
+    d = gen.make_chunk_inputs(cfg)
+    _fwd_check(cfg, d)
+    _bwd_check(cfg, d)
+    # alpha = lambda = h0 = dhT = NULL
+    d2 = dict(d, alpha=None, lam=None, h0=None, dhT=None)
+    t = gu.dev_inputs(d2, cfg.dtype)
+    o, hT, _ = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"])
+    ro, rh = gu.oracle_fwd(d2)
+    assert gu.rel_err(o, ro) <= 2e-2 and gu.rel_err(hT, rh) <= 2e-2
+    g = qd.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], None, None, None, t["dO"], None)
+    ref = gu.oracle_bwd(d2)
+    for n in ("dq", "dk", "dv", "dbeta", "dh0"):
+        assert gu.rel_err(g[n], ref[n]) <= 2e-2, n
+    assert g["dalpha"] is None and g["dlam"] is None
+
+
+def test_segment_invariance_on_gpu():
+    from paper_2606_08804_b200 import binding as qd
+    cfg = replace(gen.CONFIGS["cfg1"], B=1, H=2, T=256, regime="alpha_slow", seed=11)
+    d = gen.make_chunk_inputs(cfg)
+    t = gu.dev_inputs(d, cfg.dtype)
+    o, hT, _ = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"])
+    c = lambda x, s: x[:, s].contiguous()
+    a, b = slice(0, 128), slice(128, 256)
+    o1, h1, _ = qd.chunk_fwd(c(t["q"], a), c(t["k"], a), c(t["v"], a), c(t["beta"], a), c(t["alpha"], a),
+                             c(t["lam"], a), t["h0"])
+    o2, h2, _ = qd.chunk_fwd(c(t["q"], b), c(t["k"], b), c(t["v"], b), c(t["beta"], b), c(t["alpha"], b),
+                             c(t["lam"], b), h1)
+    torch.cuda.synchronize()
+    assert torch.equal(torch.cat([o1, o2], dim=1), o)
+    assert torch.equal(h2, hT)
+
+
+def test_deterministic_bitwise():
+    from paper_2606_08804_b200 import binding as qd
+    cfg = replace(gen.CONFIGS["cfg2"], B=2, H=2, T=256, seed=13)
+    t = gu.dev_inputs(gen.make_chunk_inputs(cfg), cfg.dtype)
+    runs = []
+    for _ in range(2):
+        o, hT, _ = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"])
+        g = qd.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], t["dO"], t["dhT"])
+        torch.cuda.synchronize()
+        runs.append([o, hT] + [g[n] for n in sorted(g)])
+    for x, y in zip(*runs):
+        assert torch.equal(x, y)
+
+
+def _sample_pairs(cfg, n, seed=0):
+    r = np.random.default_rng(seed)
+    idx = r.choice(cfg.B * cfg.H, size=min(n, cfg.B * cfg.H), replace=False)
+    return [(int(i) // cfg.H, int(i) % cfg.H) for i in idx]
+
+
+def test_cfg1_cfg2_full_size():
+    # config 1 (forward) and config 2 (forward + backward) share inputs; every sequence is run on the
+    # GPU in the benchmarked launch configuration, the oracle checks a sample of whole sequences
+    cfg = gen.CONFIGS["cfg2"]
+    d = gen.make_chunk_inputs(cfg)
+    pairs = _sample_pairs(cfg, 16)
+    _fwd_check(cfg, d, pairs)
+    _bwd_check(cfg, d, pairs, reuse=True)
+
+
+def test_cfg3_long_context_full_size():
+    cfg = gen.CONFIGS["cfg3"]
+    d = gen.make_chunk_inputs(cfg)
+    pairs = _sample_pairs(cfg, 4)
+    _fwd_check(cfg, d, pairs)
+    _bwd_check(cfg, d, pairs, reuse=True)

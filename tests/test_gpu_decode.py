@@ -1,0 +1,103 @@
+"""GPU-vs-oracle parity of the recurrent decode step (through the C ABI)."""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import recurrence as orc
+from paper_2606_08804_b200 import inputs as gen
+import gpu_util as gu
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(cfg, steps, check_at, sample=None, null_coeffs=False):
+    from paper_2606_08804_b200 import binding as qd
+    t = gu.TDT[cfg.dtype]
+    s0 = gen.make_decode_state(cfg)
+    state = gu.to_dev(s0, torch.float32)
+    Bn, H = cfg.B, cfg.H
+    if sample is None:
+        sel_b, sel_h = np.meshgrid(np.arange(Bn), np.arange(H), indexing="ij")
+        sel_b, sel_h = sel_b.ravel(), sel_h.ravel()
+    else:
+        r = np.random.default_rng(1)
+        idx = r.choice(Bn * H, size=sample, replace=False)
+        sel_b, sel_h = idx // H, idx % H
+    ref_state = s0[sel_b, sel_h][:, None].astype(np.float64)           # [n,1,dk,dv]
+    done = 0
+    block = 50
+    while done < steps:
+        n = min(block, steps - done)
+        tok = gen.make_decode_tokens(cfg, done, n)
+        if null_coeffs:
+            tok["alpha"] = None; tok["lam"] = None
+        dev = {k_: gu.to_dev(a, t) for k_, a in tok.items()}
+        outs = []
+        for i in range(n):
+            o = qd.recurrent_step(dev["q"][i], dev["k"][i], dev["v"][i], dev["beta"][i],
+                                  None if null_coeffs else dev["alpha"][i],
+                                  None if null_coeffs else dev["lam"][i], state)
+            outs.append(o)
+        torch.cuda.synchronize()
+        sub = {k_: (None if a is None else a[:, sel_b, sel_h][:, :, None]) for k_, a in tok.items()}
+        ro, ref_state = orc.decode(ref_state, sub["q"], sub["k"], sub["v"], sub["beta"], sub["alpha"], sub["lam"])
+        for i in range(n):
+            step = done + i + 1
+            if step in check_at:
+                got = outs[i][sel_b, sel_h][:, None]
+                e = gu.rel_err(got, ro[i])
+                assert e <= gu.TOL[cfg.dtype], ("o", step, e)
+                if i == n - 1:
+                    es = gu.rel_err(state[sel_b, sel_h][:, None], ref_state)
+                    assert es <= gu.TOL[cfg.dtype], ("state", step, es)
+        done += n
+    es = gu.rel_err(state[sel_b, sel_h][:, None], ref_state)
+    assert es <= gu.TOL[cfg.dtype], ("final state", es)
+
+
+def test_decode_small_bf16_all_states():
+    cfg = replace(gen.CONFIGS["cfg4"], B=3, H=5)
+    _run(cfg, 60, set(range(1, 61)))
+
+
+@pytest.mark.parametrize("dk,dv", [(64, 64), (128, 64), (64, 128)])
+def test_decode_fp32_shapes(dk, dv):
+    cfg = replace(gen.CONFIGS["cfg4"], B=2, H=3, dk=dk, dv=dv, dtype="f32")
+    _run(cfg, 20, set(range(1, 21)))
+
+
+def test_decode_null_coefficients():
+    cfg = replace(gen.CONFIGS["cfg4"], B=2, H=2)
+    _run(cfg, 10, set(range(1, 11)), null_coeffs=True)
+
+
+def test_decode_slow_decay_long():
+    cfg = replace(gen.CONFIGS["cfg4"], B=2, H=4, regime="trained_like")
+    _run(cfg, 300, {1, 10, 100, 300})
+
+
+def test_cfg4_full_size_1000_steps_sampled():
+    # the benchmarked launch shape (256 x 16 states of 128 x 128); the oracle follows 48 sampled states
+    cfg = gen.CONFIGS["cfg4"]
+    _run(cfg, 1000, {1, 10, 100, 1000}, sample=48)
+
+
+def test_decode_matches_chunk_forward_on_gpu():
+    from paper_2606_08804_b200 import binding as qd
+    cfg = replace(gen.CONFIGS["cfg1"], B=2, H=2, T=128, regime="alpha_slow", seed=21)
+    d = gen.make_chunk_inputs(cfg)
+    t = gu.dev_inputs(d, cfg.dtype)
+    o, hT, _ = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"])
+    state = t["h0"].clone()
+    outs = []
+    for s in range(cfg.T):
+        outs.append(qd.recurrent_step(t["q"][:, s].contiguous(), t["k"][:, s].contiguous(), t["v"][:, s].contiguous(),
+                                      t["beta"][:, s].contiguous(), t["alpha"][:, s].contiguous(),
+                                      t["lam"][:, s].contiguous(), state))
+    torch.cuda.synchronize()
+    o2 = torch.stack(outs, dim=1)
+    den = o.float().abs().max()
+    assert ((o2.float() - o.float()).abs().max() / den).item() <= 2e-2
+    assert ((state - hT).abs().max() / hT.abs().max()).item() <= 2e-2
