@@ -1,0 +1,351 @@
+#!/usr/bin/env python
+"""Benchmark of the Q-Delta hot path on B200.
+
+A step is one chunkwise forward (saving what the backward needs) plus one chunkwise backward over
+one batch of synthetic input of the headline configuration (bf16, B=8, H=16, T=2048,
+d_k=d_v=128, chunk 64); the decode step is timed separately on its own configuration and reported
+under "decode".  One process per GPU; with N > 1 every rank runs its own batch (weak scaling, no
+collective on the data path).  Prints ONE JSON line on rank 0.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+`--impl reference` times the fp64 CPU oracle (the only "reference implementation" this method has
+here) on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from dataclasses import replace
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "Q-Delta chunkwise fwd+bwd tokens/s (bf16, d=128) and % of roofline on 1 B200"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ---- algorithmic work per token-head (one head's share of one token), bf16 storage ---------------
+def path_bytes_per_token_head(dk, dv):
+    fwd = 2 * (2 * dk + dv) + 6 + 2 * dv                       # read q,k,v + 3 coefficients, write o
+    bwd = 2 * (2 * dk + 2 * dv) + 6 + 2 * (2 * dk + dv) + 12   # read q,k,v,dO + coeffs, write dq,dk,dv + 3 fp32
+    return fwd, bwd
+
+
+def path_flops_per_token_head(dk, dv, C):
+    s = 2.0 * C * C * dk / C          # one C x C x d product, per token
+    b = 2.0 * C * dk * dv / C         # one C x d x d product, per token
+    return 5 * s + 3 * b, 11 * s + 6 * b
+
+
+def stage_bytes_per_token_head(dk, dv, C):
+    """Compulsory HBM bytes of each kernel of the present decomposition, per token-head (bf16
+    intermediates, fp32 per-chunk states)."""
+    st = 4.0 * dk * dv / C            # one fp32 state per chunk, per token
+    return {
+        "prep": 2 * (2 * dk + dv) + 6 + 2 * (dk + dv) + 2 * C + 4,
+        "chain_fwd": 2 * (2 * dk + dv + dk) + 2 * C + 4 + 2 * dv + st + 2 * dv,
+        "chain_bwd": 2 * (2 * dk + dv) + 2 * dk + 2 * C + 2 * dv + 4 + st + 2 * dv + st,
+        "chunk_bwd": 2 * (2 * dk + 2 * dv) + 6 + 4 + 2 * C + 4 * dv + 2 * st + 2 * (2 * dk + dv) + 12,
+    }
+
+
+class ClockSampler(threading.Thread):
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.stop_flag = index, [], threading.Event()
+
+    def run(self):
+        while not self.stop_flag.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5).stdout
+                f = [x.strip() for x in out.strip().split(",")]
+                if len(f) >= 6:
+                    self.samples.append(f)
+            except Exception:
+                pass
+            self.stop_flag.wait(0.2)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        sm = sorted(float(s[0]) for s in self.samples)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(self.samples[0][1]), "reasons": reasons,
+                "samples": len(sm)}
+
+
+def oracle_sample(cfg, nseq, steps=1, warmup=0):
+    """Time the fp64 oracle (forward + reverse pass) on the first `nseq` sequences of cfg."""
+    from paper_2606_08804_b200 import inputs as gen
+    from oracle import recurrence as orc
+    sub = replace(cfg, B=1, H=nseq)
+    d = gen.make_chunk_inputs(sub)
+
+    def run():
+        orc.forward(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"])
+        orc.backward(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"], d["dO"], d["dhT"])
+    for _ in range(warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        run()
+    dt = (time.perf_counter() - t0) / steps
+    tokens = nseq * cfg.T / cfg.H            # a token carries all H heads
+    return tokens / dt, dt, orc.max_threads()
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = os.cpu_count() or 1
+    nseq = max(1, min(cfg.B * cfg.H, 4 * cores))
+    val, dt, thr = oracle_sample(cfg, nseq, steps=args.steps, warmup=min(args.warmup, 1))
+    sample = "first %d of %d (batch, head) sequences of %s, forward + reverse pass, fp64" % (nseq, cfg.B * cfg.H, cfg.name)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "sample": sample},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def workload_name(cfg):
+    return "%s: bf16 fwd+bwd B=%d H=%d T=%d dk=%d dv=%d chunk=%d" % (cfg.name, cfg.B, cfg.H, cfg.T, cfg.dk, cfg.dv, cfg.chunk)
+
+
+def run_ours(args, cfg):
+    import torch
+    from paper_2606_08804_b200 import binding as qd
+    from paper_2606_08804_b200 import inputs as gen
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    qd.load()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- inputs: pinned host copies and device copies ------------------------------------------
+    d = gen.make_chunk_inputs(cfg, seed=cfg.seed + rank)
+    bf, f32 = torch.bfloat16, torch.float32
+    host, dev = {}, {}
+    for n in ("q", "k", "v", "beta", "alpha", "lam", "dO"):
+        host[n] = torch.from_numpy(d[n]).to(bf).pin_memory()
+    for n in ("h0", "dhT"):
+        host[n] = torch.from_numpy(d[n]).pin_memory()
+    for n, t in host.items():
+        dev[n] = t.to("cuda", non_blocking=True)
+    del d
+    B, T, H, dk, dv = cfg.B, cfg.T, cfg.H, cfg.dk, cfg.dv
+    shape = qd.make_shape(dev["q"], dev["v"], cfg.chunk)
+    ws = qd.alloc_workspace(shape, True, "cuda")
+    o = torch.empty((B, T, H, dv), dtype=bf, device="cuda")
+    hT = torch.empty((B, H, dk, dv), dtype=f32, device="cuda")
+    grads = {}
+
+    def step():
+        qd.chunk_fwd(dev["q"], dev["k"], dev["v"], dev["beta"], dev["alpha"], dev["lam"], dev["h0"],
+                     chunk=cfg.chunk, save_for_bwd=True, workspace=ws, o=o, hT=hT)
+        qd.chunk_bwd(dev["q"], dev["k"], dev["v"], dev["beta"], dev["alpha"], dev["lam"], dev["h0"],
+                     dev["dO"], dev["dhT"], chunk=cfg.chunk, workspace=ws, reuse_fwd=True, out=grads)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    assert qd.workspace_status(ws) == 0, "device-side status word is set"
+
+    # ---- timed region: K steps, CUDA events on the launching stream, per-kernel events inside -----
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    qd.profile_read(reset=True)
+    qd.profile_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        step()
+    e1.record()
+    barrier()
+    qd.profile_enable(False)
+    ms = e0.elapsed_time(e1)
+    stages = qd.profile_read(reset=True)
+    sampler.stop_flag.set()
+    sampler.join()
+    if dist is not None:
+        tms = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+        ms = float(tms.item())
+    ms_step = ms / args.steps
+    tokens_step = B * T * world
+    value = tokens_step / (ms_step * 1e-3)
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region ------------
+    out_host = {"o": torch.empty_like(o, device="cpu").pin_memory(), "hT": torch.empty_like(hT, device="cpu").pin_memory()}
+    for n, t in grads.items():
+        out_host[n] = torch.empty_like(t, device="cpu").pin_memory()
+    h2d = sum(t.numel() * t.element_size() for t in host.values())
+    d2h = sum(t.numel() * t.element_size() for t in out_host.values())
+
+    def e2e_step():
+        for n, t in host.items():
+            dev[n].copy_(t, non_blocking=True)
+        step()
+        out_host["o"].copy_(o, non_blocking=True)
+        out_host["hT"].copy_(hT, non_blocking=True)
+        for n, t in grads.items():
+            out_host[n].copy_(t, non_blocking=True)
+
+    e2e_steps = max(1, min(args.steps, 10))
+    e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    ems = e0.elapsed_time(e1)
+    if dist is not None:
+        tms = torch.tensor([ems], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
+        ems = float(tms.item())
+    e2e_value = tokens_step / (ems / e2e_steps * 1e-3)
+
+    # ---- roofline of the dominant kernel and of the whole path -----------------------------------
+    pk, pk_kind = peaks()
+    th = B * T * H                                     # token-heads one launch processes
+    sb = stage_bytes_per_token_head(dk, dv, cfg.chunk)
+    chunk_stages = {n: v for n, v in stages.items() if n in sb and v[1] > 0}
+    dom = max(chunk_stages, key=lambda n: chunk_stages[n][0])
+    dom_ms = chunk_stages[dom][0] / chunk_stages[dom][1]
+    ach = sb[dom] * th / (dom_ms * 1e-3) / 1e9
+    roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / pk["hbm_gbs"], "traffic": None, "peak_kind": "of " + pk_kind,
+                "ms_per_launch": dom_ms, "algorithmic_bytes_per_launch": sb[dom] * th}
+    fb, bb = path_bytes_per_token_head(dk, dv)
+    ff, fbw = path_flops_per_token_head(dk, dv, cfg.chunk)
+    state_io = 4 * dk * dv * 4 * B * H
+    t_bytes = ((fb + bb) * th + state_io) / (pk["hbm_gbs"] * 1e9)
+    t_flops = (ff + fbw) * th / (pk["bf16_tflops"] * 1e12)
+    per_rank_ms = ms_step
+    path = {"bytes_per_step": (fb + bb) * th + state_io, "flops_per_step": (ff + fbw) * th,
+            "roofline_ms": max(t_bytes, t_flops) * 1e3, "frac": max(t_bytes, t_flops) * 1e3 / per_rank_ms,
+            "peak_kind": "of " + pk_kind,
+            "stage_ms_per_launch": {n: v[0] / v[1] for n, v in chunk_stages.items()}}
+    launches = int(sum(v[1] for v in stages.values()))
+
+    # ---- decode step (separate configuration), in place over a long run of steps ------------------
+    decode = bench_decode(args, qd, gen, torch, pk, pk_kind) if rank == 0 else None
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "l2": "inputs larger than L2 (no flush)",
+                       "tokens_per_step": tokens_step, "parallelism": "batch sharded over %d rank(s), no collective" % world},
+            "clocks": sampler.summary(),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": e2e_steps},
+            "gpu_launches": launches, "roofline": roofline, "roofline_path": path, "decode": decode}
+    if rank == 0:
+        if world == 1:
+            cores = os.cpu_count() or 1
+            nseq = max(1, min(B * H, 4 * cores))
+            v, dt, thr = oracle_sample(cfg, nseq)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": thr, "kind": "oracle",
+                                    "sample": "first %d of %d (batch, head) sequences, fwd + reverse pass, fp64, %.1f s"
+                                              % (nseq, B * H, dt)}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def bench_decode(args, qd, gen, torch, pk, pk_kind):
+    cfg = gen.CONFIGS["cfg4"]
+    bf = torch.bfloat16
+    state = torch.from_numpy(gen.make_decode_state(cfg)).cuda()
+    pool = 8
+    tok = gen.make_decode_tokens(cfg, 0, pool)
+    tok = {n: torch.from_numpy(a).to("cuda", bf) for n, a in tok.items()}
+    o = torch.empty((cfg.B, cfg.H, cfg.dv), dtype=bf, device="cuda")
+    nsteps = 200
+
+    def one(i):
+        j = i % pool
+        qd.recurrent_step(tok["q"][j], tok["k"][j], tok["v"][j], tok["beta"][j], tok["alpha"][j], tok["lam"][j],
+                          state, o)
+    for i in range(10):
+        one(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(nsteps):
+        one(i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / nsteps
+    nstates = cfg.B * cfg.H
+    bytes_step = nstates * (2 * cfg.dk * cfg.dv * 4 + 2 * (2 * cfg.dk + cfg.dv) + 6 + 2 * cfg.dv)
+    gbs = bytes_step / (ms * 1e-3) / 1e9
+    return {"workload": "cfg4: batch=%d H=%d dk=%d dv=%d fp32 state in place, bf16 tokens" % (cfg.B, cfg.H, cfg.dk, cfg.dv),
+            "steps": nsteps, "us_per_step": ms * 1e3, "tokens_per_s": cfg.B / (ms * 1e-3),
+            "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                         "frac": gbs / pk["hbm_gbs"], "peak_kind": "of " + pk_kind,
+                         "algorithmic_bytes_per_launch": bytes_step, "state_larger_than_l2": True}}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    from paper_2606_08804_b200 import inputs as gen
+    cfg = gen.CONFIGS["cfg2"]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

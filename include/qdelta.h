@@ -20,7 +20,9 @@
  *     dbeta,dalpha,dlambda and every state are fp32.
  *   - The caller owns every buffer, including the workspace whose size it queries.  The library
  *     never allocates, frees or synchronises; all work is enqueued on `stream`.
- *   - Inputs are read-only.  Outputs are fully overwritten.  Pointers must be 16-byte aligned.
+ *   - Inputs are read-only.  Outputs are fully overwritten.  q,k,v,o,dO,dq,dk,dv, the
+ *     states and the workspace must be 16-byte aligned; coefficient tensors (and the decode step's o)
+ *     need only the alignment of their element type.
  *   - Coefficient domains: beta, lambda in [0,1], alpha in (0,1] (Section 3.3.1); not checked on device.
  *   - Return value: QD_OK, or an error code reported synchronously; on error nothing was enqueued.
  *     Conditions found on the device (a bounded wait that ran out) are written to the first

@@ -101,9 +101,12 @@ int qdelta_chunk_fwd(const qd_shape* shape, const void* q, const void* k, const 
     int rc = check_shape(shape);
     if (rc != QD_OK) return rc;
     if (!q || !k || !v || !beta || !o) return QD_ERR_INVALID_ARG;
-    const void* ptrs[] = {q, k, v, beta, alpha, lambda, h0, o, hT, workspace};
+    const void* ptrs[] = {q, k, v, h0, o, hT, workspace};
     for (const void* p : ptrs)
         if (p && misaligned(p)) return QD_ERR_INVALID_ARG;
+    const void* coef[] = {beta, alpha, lambda};
+    for (const void* p : coef)
+        if (p && ((uintptr_t)p & (shape->dtype == QD_BF16 ? 1 : 3))) return QD_ERR_INVALID_ARG;
     if (flags & ~(unsigned)QD_FWD_SAVE_FOR_BWD) return QD_ERR_INVALID_ARG;
     ChunkArgs a{};
     a.s = *shape;
@@ -127,9 +130,15 @@ int qdelta_chunk_bwd(const qd_shape* shape, const void* q, const void* k, const 
     if (rc != QD_OK) return rc;
     if (!q || !k || !v || !beta || !dO || !dq || !dk || !dv || !dbeta) return QD_ERR_INVALID_ARG;
     if ((alpha && !dalpha) || (lambda && !dlambda)) return QD_ERR_INVALID_ARG;
-    const void* ptrs[] = {q, k, v, beta, alpha, lambda, h0, dO, dhT, dq, dk, dv, dbeta, dalpha, dlambda, dh0, workspace};
+    const void* ptrs[] = {q, k, v, h0, dO, dhT, dq, dk, dv, dh0, workspace};
     for (const void* p : ptrs)
         if (p && misaligned(p)) return QD_ERR_INVALID_ARG;
+    const void* coef[] = {beta, alpha, lambda};
+    for (const void* p : coef)
+        if (p && ((uintptr_t)p & (shape->dtype == QD_BF16 ? 1 : 3))) return QD_ERR_INVALID_ARG;
+    const void* gcoef[] = {dbeta, dalpha, dlambda};
+    for (const void* p : gcoef)
+        if (p && ((uintptr_t)p & 3)) return QD_ERR_INVALID_ARG;
     if (flags & ~(unsigned)QD_BWD_REUSE_FWD) return QD_ERR_INVALID_ARG;
     ChunkArgs a{};
     a.s = *shape;
@@ -163,9 +172,12 @@ int qdelta_recurrent_step(int B, int H, int dk, int dv, int dtype, const void* q
     if ((dk != 64 && dk != 128) || (dv != 64 && dv != 128)) return QD_ERR_UNSUPPORTED;
     if (!q || !k || !v || !beta || !state || !o) return QD_ERR_INVALID_ARG;
     if ((long long)B * H > 0x3fffffffLL) return QD_ERR_UNSUPPORTED;
-    const void* ptrs[] = {q, k, v, beta, alpha, lambda, state, o};
+    const void* ptrs[] = {q, k, v, state};
     for (const void* p : ptrs)
         if (p && misaligned(p)) return QD_ERR_INVALID_ARG;
+    const void* coef[] = {beta, alpha, lambda, o};
+    for (const void* p : coef)
+        if (p && ((uintptr_t)p & (dtype == QD_BF16 ? 1 : 3))) return QD_ERR_INVALID_ARG;
     if (timed(ST_DECODE, (cudaStream_t)stream, [&] {
             return decode_step(B * H, dk, dv, dtype, q, k, v, beta, alpha, lambda, state, o, (cudaStream_t)stream);
         }) != cudaSuccess)
