@@ -306,7 +306,7 @@ def bench_decode(args, qd, gen, torch, pk, pk_kind):
     tok = gen.make_decode_tokens(cfg, 0, pool)
     tok = {n: torch.from_numpy(a).to("cuda", bf) for n, a in tok.items()}
     o = torch.empty((cfg.B, cfg.H, cfg.dv), dtype=bf, device="cuda")
-    nsteps = 200
+    nsteps = args.decode_steps
 
     def one(i):
         j = i % pool
@@ -338,10 +338,18 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--only", default="all", choices=["all", "decode"],
+                    help="'decode': time only the decode step (small runs for profiler captures)")
+    ap.add_argument("--decode-steps", type=int, default=200)
     args = ap.parse_args()
     from paper_2606_08804_b200 import inputs as gen
     cfg = gen.CONFIGS["cfg2"]
-    if args.impl == "reference":
+    if args.only == "decode":
+        import torch
+        from paper_2606_08804_b200 import binding as qd
+        pk, pk_kind = peaks()
+        print(json.dumps({"decode": bench_decode(args, qd, gen, torch, pk, pk_kind)}))
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         run_ours(args, cfg)
