@@ -92,7 +92,12 @@ extern "C" {
 size_t qdelta_chunk_workspace_bytes(const qd_shape* shape, int for_backward) {
     if (check_shape(shape) != QD_OK) return 0;
     WsLayout L = ws_layout(*shape);
-    return for_backward ? L.bwd_end : L.fwd_end;
+    size_t n = for_backward ? L.bwd_end : L.fwd_end;
+    if (tc_supported(*shape)) {
+        TcLayout TL = tc_layout(*shape);
+        if (TL.fwd_end > n) n = TL.fwd_end;
+    }
+    return n;
 }
 
 int qdelta_chunk_fwd(const qd_shape* shape, const void* q, const void* k, const void* v, const void* beta,
@@ -117,6 +122,13 @@ int qdelta_chunk_fwd(const qd_shape* shape, const void* q, const void* k, const 
     a.ws = (char*)workspace;
     a.stream = (cudaStream_t)stream;
     if (cudaMemsetAsync(a.ws + a.L.status, 0, 256, a.stream) != cudaSuccess) return QD_ERR_CUDA;
+    if (!a.save && tc_supported(*shape)) {
+        a.TL = tc_layout(*shape);
+        if (workspace_bytes < a.TL.fwd_end) return QD_ERR_WORKSPACE;
+        if (timed(ST_PREP, a.stream, [&] { return tc_prep(a); }) != cudaSuccess) return QD_ERR_CUDA;
+        if (timed(ST_CHAIN_FWD, a.stream, [&] { return tc_chain_fwd(a); }) != cudaSuccess) return QD_ERR_CUDA;
+        return QD_OK;
+    }
     if (timed(ST_PREP, a.stream, [&] { return simt_prep(a); }) != cudaSuccess) return QD_ERR_CUDA;
     if (timed(ST_CHAIN_FWD, a.stream, [&] { return simt_chain_fwd(a); }) != cudaSuccess) return QD_ERR_CUDA;
     return QD_OK;

@@ -36,6 +36,19 @@ struct WsLayout {
 
 WsLayout ws_layout(const qd_shape& s);
 
+// Workspace of the tensor-core path (bf16, d_k = d_v = 128).  Sections start on 1024-byte boundaries.
+struct TcLayout {
+    size_t status;   // u32 status word
+    size_t g;        // fp32 [BH*T]
+    size_t Qg;       // bf16 [BH*T][dk]        diag(gamma) Q
+    size_t P;        // bf16 [BH*T][C]         Gamma o (Q K^T), causal incl. diagonal
+    size_t Wt;       // bf16 [BH*N][dk][C]     (T diag(gamma) X)^T per chunk
+    size_t Ut;       // bf16 [BH*N][dv][C]     (T V)^T per chunk
+    size_t fwd_end;
+};
+TcLayout tc_layout(const qd_shape& s);
+bool tc_supported(const qd_shape& s);
+
 struct ChunkArgs {
     qd_shape s;
     const void *q, *k, *v, *beta, *alpha, *lam;
@@ -49,6 +62,7 @@ struct ChunkArgs {
     float *dbeta, *dalpha, *dlam, *dh0;
     char* ws;
     WsLayout L;
+    TcLayout TL;
     bool save;       // forward: keep hs and D
     cudaStream_t stream;
 };
@@ -58,6 +72,10 @@ cudaError_t simt_prep(const ChunkArgs& a);        // g, P, W<-, U~
 cudaError_t simt_chain_fwd(const ChunkArgs& a);   // Delta, O, state chain (+ hs, D when a.save)
 cudaError_t simt_chain_bwd(const ChunkArgs& a);   // dDelta, dhs, dh0, scalar partials
 cudaError_t simt_chunk_bwd(const ChunkArgs& a);   // dq, dk, dv, dbeta, dalpha, dlambda
+
+// tcgen05 path
+cudaError_t tc_prep(const ChunkArgs& a);
+cudaError_t tc_chain_fwd(const ChunkArgs& a);
 
 cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
                         const void* beta, const void* alpha, const void* lam, float* state, void* o,

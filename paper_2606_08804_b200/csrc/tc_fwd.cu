@@ -1,0 +1,503 @@
+// Tensor-core (tcgen05 / TMEM / TMA) chunkwise forward for bf16, d_k = d_v = 128, chunk 64.
+//
+// Two kernels, following Section 3.3.2:
+//   k_tc_prep       one CTA per PAIR of chunks (128 tokens): g, X = K + diag(lambda) Q, the Gram
+//                   blocks X K^T and Q K^T, the UT-transform inverse, and the WY factors.  It leaves,
+//                   per chunk, in bf16:  Qg = diag(gamma) Q  [token][dk],
+//                   P = Gamma o (Q K^T) causal incl. diagonal [token][64],
+//                   Wt = (T diag(gamma) X)^T  [dk][64 tokens],   Ut = (T V)^T  [dv][64 tokens].
+//   k_tc_chain_fwd  one CTA per (batch, head): walks the chunks in order with the fp32 state in
+//                   registers (thread j owns row j of h^T, i.e. column j of h), everything
+//                   transposed so that d_v = 128 is the MMA M dimension:
+//                     Delta^T = Ut - h^T Wt            O^T = h^T Qg^T + Delta^T P^T
+//                     h^T <- gamma_C h^T + (Delta diag(gamma_C/gamma))^T K
+// All waits are bounded; on expiry the CTA records QD_ERR_TIMEOUT in the workspace status word,
+// releases its tensor memory and returns.
+#include "internal.h"
+#include "sm100.cuh"
+
+namespace qd {
+namespace {
+using namespace sm100;
+typedef __nv_bfloat16 bf16;
+
+constexpr int C = kChunk;      // 64
+constexpr int D = 128;         // d_k = d_v
+constexpr int LDA = C + 1;
+
+__device__ __forceinline__ void load8(const unsigned char* p, float* f) {
+    const uint4 u = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+    uint4 u;
+    u.x = pack_bf16(f[0], f[1]); u.y = pack_bf16(f[2], f[3]); u.z = pack_bf16(f[4], f[5]); u.w = pack_bf16(f[6], f[7]);
+    return u;
+}
+
+// =================================================================================================
+struct PrepParams {
+    int T, H, N;
+    const bf16 *beta, *alpha, *lam;
+    float* g;
+    bf16 *Qg, *P, *Wt, *Ut;
+    unsigned* status;
+};
+
+constexpr int kPrepSmem = 4 * 32768 + 2 * C * LDA * 4 + 1024;
+
+__global__ void __launch_bounds__(128) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
+                                                 const __grid_constant__ CUtensorMap mapK,
+                                                 const __grid_constant__ CUtensorMap mapV, PrepParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *sQ = smem, *sK = smem + 32768, *sV = smem + 65536, *sX = smem + 98304;
+    float* sA = reinterpret_cast<float*>(smem);                 // [2][64][65], aliases sQ/sK once the Grams are read
+    float* sM = reinterpret_cast<float*>(smem + 131072);        // [2][64][65]
+    unsigned char* sT = smem;                                   // [2] T_c, [2] T_c diag(gamma): 8 KB each, alias sA
+    __shared__ uint64_t bar_load, bar_mma;
+    __shared__ uint32_t tmem_slot;
+    __shared__ float sg[128], swsum[4];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int c = tid >> 6, r = tid & 63;
+    const int pairs = p.N / 2, bh = blockIdx.x / pairs, pr = blockIdx.x % pairs;
+    const int b = bh / p.H, hh = bh % p.H;
+    const size_t tok = (size_t)b * p.T + (size_t)pr * 128 + tid;      // row in the [B*T] view
+    const size_t wtok = (size_t)bh * p.T + (size_t)pr * 128 + tid;    // row in the [BH*T] view
+
+    if (tid == 0) {
+        mbar_init(&bar_load, 1);
+        mbar_init(&bar_mma, 1);
+        mbar_init_fence();
+    }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = tmem_slot;
+
+    if (tid == 0) {
+        mbar_expect_tx(&bar_load, 3 * 32768);
+        const int y = (int)((size_t)b * p.T + (size_t)pr * 128);
+        for (int blk = 0; blk < 2; ++blk) {
+            tma_load_2d(sQ + blk * 16384, &mapQ, hh * D + blk * 64, y, &bar_load);
+            tma_load_2d(sK + blk * 16384, &mapK, hh * D + blk * 64, y, &bar_load);
+            tma_load_2d(sV + blk * 16384, &mapV, hh * D + blk * 64, y, &bar_load);
+        }
+    }
+    // coefficients of my token; in-chunk cumulative log-decay by a two-warp scan
+    const size_t crow = tok * p.H + hh;
+    const float beta = __bfloat162float(p.beta[crow]);
+    const float lam = p.lam ? __bfloat162float(p.lam[crow]) : 0.f;
+    const float alpha = p.alpha ? __bfloat162float(p.alpha[crow]) : 1.f;
+    float g = logf(alpha);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float t = __shfl_up_sync(0xffffffffu, g, o);
+        if (lane >= o) g += t;
+    }
+    if (lane == 31) swsum[warp] = g;
+    __syncthreads();
+    if (warp & 1) g += swsum[warp - 1];
+    sg[tid] = g;
+    p.g[wtok] = g;
+    const float gam = expf(g);
+
+    bool fail = !mbar_wait(&bar_load, 0);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        // loads may still be in flight: give them one more bounded chance before leaving
+        mbar_wait(&bar_load, 0);
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tbase, 256);
+        return;
+    }
+    // X = K + lambda Q (row `tid`, in the K-major swizzled layout); Qg = gamma Q to the workspace
+    {
+        bf16* qg = p.Qg + wtok * D;
+#pragma unroll
+        for (int blk = 0; blk < 2; ++blk)
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+                const uint32_t off = blk * 16384 + sw128_chunk(tid, ch);
+                float qv[8], kv[8], xv[8], gv[8];
+                load8(sQ + off, qv);
+                load8(sK + off, kv);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { xv[e] = fmaf(lam, qv[e], kv[e]); gv[e] = gam * qv[e]; }
+                *reinterpret_cast<uint4*>(sX + off) = pack8(xv);
+                *reinterpret_cast<uint4*>(qg + blk * 64 + ch * 8) = pack8(gv);
+            }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+        tc_fence_after();
+        // G1 = X K^T -> columns [0,128);  G2 = Q K^T -> columns [128,256)
+        umma_product<false, false>(tbase, smem_u32(sX), 16384, smem_u32(sK), 16384, 128, 128, false);
+        umma_product<false, false>(tbase + 128, smem_u32(sQ), 16384, smem_u32(sK), 16384, 128, 128, false);
+        umma_commit(&bar_mma);
+    }
+    fail = !mbar_wait(&bar_mma, 0);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        if (warp == 0) tmem_dealloc(tbase, 256);
+        return;
+    }
+    tc_fence_after();
+    // A = strictLower(beta_r Gamma_ri (x_r . k_i)) -> shared fp32;  P = Gamma_ri (q_r . k_i), i <= r -> workspace
+    {
+        float* arow = sA + c * C * LDA + r * LDA;
+        bf16* prow = p.P + wtok * C;
+        const float* gc = sg + c * C;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            float v1[32], v2[32];
+            tmem_ld32(tmem_addr(tbase, warp * 32, c * C + half * 32), v1);
+            tmem_ld32(tmem_addr(tbase, warp * 32, 128 + c * C + half * 32), v2);
+            tmem_ld_wait();
+            float pv[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int col = half * 32 + i;
+                const float dec = (col <= r) ? expf(g - gc[col]) : 0.f;
+                arow[col] = (col < r) ? beta * dec * v1[i] : 0.f;
+                pv[i] = dec * v2[i];
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(prow + half * 32 + i * 8) = pack8(pv + i * 8);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    // M_c = (I + A_c)^-1: thread (c, j) solves column j by forward substitution
+    {
+        const float* A = sA + c * C * LDA;
+        float* M = sM + c * C * LDA;
+        const int j = r;
+        for (int rr = 0; rr < j; ++rr) M[rr * LDA + j] = 0.f;
+        M[j * LDA + j] = 1.f;
+        for (int rr = j + 1; rr < C; ++rr) {
+            float acc = 0.f;
+            for (int i = j; i < rr; ++i) acc = fmaf(A[rr * LDA + i], M[i * LDA + j], acc);
+            M[rr * LDA + j] = -acc;
+        }
+    }
+    __syncthreads();
+    // T_c = M_c diag(beta), T_c diag(gamma): thread (c, i) owns column i and writes line i (MN-major tile)
+    {
+        const float* M = sM + c * C * LDA;
+        unsigned char* t0 = sT + c * 8192;
+        unsigned char* t1 = sT + 16384 + c * 8192;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+            float a[8], bq[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float m = M[(ch * 8 + e) * LDA + r] * beta;
+                a[e] = m; bq[e] = m * gam;
+            }
+            *reinterpret_cast<uint4*>(t0 + sw128_chunk(r, ch)) = pack8(a);
+            *reinterpret_cast<uint4*>(t1 + sw128_chunk(r, ch)) = pack8(bq);
+        }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+        tc_fence_after();
+        for (int cc = 0; cc < 2; ++cc) {
+            // Ut_c = V_c^T T_c^T  -> columns [cc*64, +64);   Wt_c = X_c^T (T_c diag(gamma))^T -> 128 + ...
+            umma_product<true, true>(tbase + cc * C, smem_u32(sV) + cc * C * 128, 16384,
+                                     smem_u32(sT) + cc * 8192, 8192, C, C, false);
+            umma_product<true, true>(tbase + 128 + cc * C, smem_u32(sX) + cc * C * 128, 16384,
+                                     smem_u32(sT) + 16384 + cc * 8192, 8192, C, C, false);
+        }
+        umma_commit(&bar_mma);
+    }
+    fail = !mbar_wait(&bar_mma, 1);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        if (warp == 0) tmem_dealloc(tbase, 256);
+        return;
+    }
+    tc_fence_after();
+    // rows `tid` (a d_v resp. d_k index) of Ut and Wt, both chunks
+#pragma unroll
+    for (int which = 0; which < 2; ++which) {
+        bf16* dst = which ? p.Wt : p.Ut;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            float v[32];
+            tmem_ld32(tmem_addr(tbase, warp * 32, which * 128 + q4 * 32), v);
+            tmem_ld_wait();
+            const int cc = q4 >> 1;
+            bf16* row = dst + (((size_t)bh * p.N + 2 * pr + cc) * D + tid) * C + (q4 & 1) * 32;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(row + i * 8) = pack8(v + i * 8);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tbase, 256);
+}
+
+// =================================================================================================
+struct ChainParams {
+    int T, H, N;
+    const float* g;
+    const float* h0;
+    bf16* o;
+    float* hT;
+    unsigned* status;
+};
+
+constexpr int kStage = 73728;                           // Wt 16K | Ut 16K | Qg 16K | K 16K | P 8K
+constexpr int kChainSmem = 2 * kStage + 65536 + 1024;   // + hT operand 32K, Delta^T 16K, scaled Delta^T 16K
+
+__global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CUtensorMap mapWt,
+                                                      const __grid_constant__ CUtensorMap mapUt,
+                                                      const __grid_constant__ CUtensorMap mapQg,
+                                                      const __grid_constant__ CUtensorMap mapK,
+                                                      const __grid_constant__ CUtensorMap mapP, ChainParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char* sH = smem + 2 * kStage;          // h^T as A operand: K-major, 2 blocks of [128 lines][64]
+    unsigned char* sD = sH + 32768;                 // Delta^T: K-major [128 lines (dv)][64 tokens]
+    unsigned char* sDs = sD + 16384;                // Delta^T scaled by gamma_C/gamma_r per token
+    __shared__ uint64_t bar_load[2], bar_a, bar_b;
+    __shared__ uint32_t tmem_slot;
+    __shared__ float sg[2][C];
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int bh = blockIdx.x, b = bh / p.H, hh = bh % p.H;
+
+    if (tid == 0) {
+        mbar_init(&bar_load[0], 1); mbar_init(&bar_load[1], 1);
+        mbar_init(&bar_a, 1); mbar_init(&bar_b, 1);
+        mbar_init_fence();
+    }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = tmem_slot;
+    const uint32_t tD = tbase, tO = tbase + 64, tH = tbase + 128;
+
+    auto issue_load = [&](int n) {
+        unsigned char* st = smem + (n & 1) * kStage;
+        uint64_t* bar = &bar_load[n & 1];
+        mbar_expect_tx(bar, kStage);
+        const int yc = (int)(((size_t)bh * p.N + n) * D);
+        const int yt = (int)((size_t)bh * p.T + (size_t)n * C);
+        tma_load_2d(st, &mapWt, 0, yc, bar);
+        tma_load_2d(st + 16384, &mapUt, 0, yc, bar);
+        tma_load_2d(st + 32768, &mapQg, 0, yt, bar);
+        tma_load_2d(st + 32768 + 8192, &mapQg, 64, yt, bar);
+        const int yk = (int)((size_t)b * p.T + (size_t)n * C);
+        tma_load_2d(st + 49152, &mapK, hh * D, yk, bar);
+        tma_load_2d(st + 49152 + 8192, &mapK, hh * D + 64, yk, bar);
+        tma_load_2d(st + 65536, &mapP, 0, yt, bar);
+    };
+    if (tid == 0) { issue_load(0); if (p.N > 1) issue_load(1); }
+
+    // state: thread j holds row j of h^T (= column j of h), fp32
+    float h[D];
+    if (p.h0) {
+        const float* src = p.h0 + (size_t)bh * D * D + tid;
+#pragma unroll
+        for (int i = 0; i < D; ++i) h[i] = src[(size_t)i * D];
+    } else {
+#pragma unroll
+        for (int i = 0; i < D; ++i) h[i] = 0.f;
+    }
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk)
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch)
+            *reinterpret_cast<uint4*>(sH + blk * 16384 + sw128_chunk(tid, ch)) = pack8(h + blk * 64 + ch * 8);
+    if (tid < C) sg[0][tid] = p.g[(size_t)bh * p.T + tid];
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+
+    bool aborted = false;
+    int loads_waited = 0;
+    for (int n = 0; n < p.N; ++n) {
+        unsigned char* st = smem + (n & 1) * kStage;
+        const float* gc = sg[n & 1];
+        bool fail = !mbar_wait(&bar_load[n & 1], (n >> 1) & 1);
+        if (__syncthreads_or(fail)) { aborted = true; break; }
+        loads_waited = n + 1;
+        if (tid == 0) {
+            tc_fence_after();
+            // Delta-accumulator = h^T Wt (B: MN-major, lines = d_k);  O-accumulator = h^T Qg^T (B: K-major)
+            umma_product<false, true>(tD, smem_u32(sH), 16384, smem_u32(st), 8192, C, D, false);
+            umma_product<false, false>(tO, smem_u32(sH), 16384, smem_u32(st + 32768), 8192, C, D, false);
+            umma_commit(&bar_a);
+        }
+        fail = !mbar_wait(&bar_a, n & 1);
+        if (__syncthreads_or(fail)) { aborted = true; break; }
+        tc_fence_after();
+        // Delta^T = Ut - acc ; two bf16 copies (plain, and scaled by gamma_C/gamma_r) as A operands
+        {
+            const float gC = gc[C - 1];
+            const unsigned char* ut = st + 16384;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                float v[32];
+                tmem_ld32(tmem_addr(tD, warp * 32, half * 32), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    float u[8], d0[8], d1[8];
+                    const uint32_t off = sw128_chunk(tid, half * 4 + ch);
+                    load8(ut + off, u);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        d0[e] = u[e] - v[ch * 8 + e];
+                        d1[e] = d0[e] * expf(gC - gc[half * 32 + ch * 8 + e]);
+                    }
+                    *reinterpret_cast<uint4*>(sD + off) = pack8(d0);
+                    *reinterpret_cast<uint4*>(sDs + off) = pack8(d1);
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            // O += Delta^T P^T (B: K-major [r][s]);   H-accumulator = scaled Delta^T K (B: MN-major, lines = tokens)
+            umma_product<false, false>(tO, smem_u32(sD), 16384, smem_u32(st + 65536), 8192, C, C, true);
+            umma_product<false, true>(tH, smem_u32(sDs), 16384, smem_u32(st + 49152), 8192, D, C, false);
+            umma_commit(&bar_b);
+        }
+        fail = !mbar_wait(&bar_b, n & 1);
+        if (__syncthreads_or(fail)) { aborted = true; break; }
+        tc_fence_after();
+        // this stage's tiles are consumed: refill it with chunk n+2
+        if (tid == 0 && n + 2 < p.N) issue_load(n + 2);
+        // h^T <- gamma_C h^T + acc, refresh the bf16 operand copy
+        {
+            const float gamC = expf(gc[C - 1]);
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                float v[32];
+                tmem_ld32(tmem_addr(tH, warp * 32, q4 * 32), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) h[q4 * 32 + i] = fmaf(gamC, h[q4 * 32 + i], v[i]);
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch)
+                    *reinterpret_cast<uint4*>(sH + (q4 >> 1) * 16384 + sw128_chunk(tid, (q4 & 1) * 4 + ch)) =
+                        pack8(h + q4 * 32 + ch * 8);
+            }
+        }
+        // O^T row j -> o[b, t0 + r, hh, j]
+        {
+            bf16* orow = p.o + (((size_t)b * p.T + (size_t)n * C) * p.H + hh) * D + tid;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                float v[32];
+                tmem_ld32(tmem_addr(tO, warp * 32, half * 32), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) orow[(size_t)(half * 32 + i) * p.H * D] = __float2bfloat16_rn(v[i]);
+            }
+        }
+        if (tid < C && n + 1 < p.N) sg[(n + 1) & 1][tid] = p.g[(size_t)bh * p.T + (size_t)(n + 1) * C + tid];
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+    }
+    if (aborted) {
+        if (tid == 0) {
+            *p.status = QD_ERR_TIMEOUT;
+            // loads already issued for chunks loads_waited .. min(N, loads_waited + 2) - 1 may be in flight
+            for (int n = loads_waited; n < p.N && n < loads_waited + 2; ++n) mbar_wait(&bar_load[n & 1], (n >> 1) & 1);
+        }
+    } else if (p.hT) {
+        float* dst = p.hT + (size_t)bh * D * D + tid;
+#pragma unroll
+        for (int i = 0; i < D; ++i) dst[(size_t)i * D] = h[i];
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tbase, 256);
+}
+
+template <class K>
+cudaError_t set_smem(K kern, size_t bytes) {
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+}  // namespace
+
+bool tc_supported(const qd_shape& s) {
+    return s.dtype == QD_BF16 && s.dk == 128 && s.dv == 128 && s.chunk == kChunk && s.T % 128 == 0 &&
+           (long long)s.B * s.H * s.T * 128 < 0x7fffffffLL * 64;
+}
+
+TcLayout tc_layout(const qd_shape& s) {
+    TcLayout L{};
+    const size_t BH = (size_t)s.B * s.H, T = s.T;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = (off + bytes + 1023) & ~(size_t)1023; return o; };
+    L.status = take(256);
+    L.g = take(BH * T * 4);
+    L.Qg = take(BH * T * s.dk * 2);
+    L.P = take(BH * T * kChunk * 2);
+    L.Wt = take(BH * T * s.dk * 2);
+    L.Ut = take(BH * T * s.dv * 2);
+    L.fwd_end = off;
+    return L;
+}
+
+cudaError_t tc_prep(const ChunkArgs& a) {
+    const qd_shape& s = a.s;
+    CUtensorMap mQ, mK, mV;
+    const uint64_t rows = (uint64_t)s.B * s.T, cols = (uint64_t)s.H * D;
+    if (!make_tmap_bf16_2d(&mQ, a.q, cols, rows, cols * 2, 128) || !make_tmap_bf16_2d(&mK, a.k, cols, rows, cols * 2, 128) ||
+        !make_tmap_bf16_2d(&mV, a.v, cols, rows, cols * 2, 128))
+        return cudaErrorInvalidValue;
+    PrepParams p{};
+    p.T = s.T; p.H = s.H; p.N = s.T / kChunk;
+    p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
+    p.g = (float*)(a.ws + a.TL.g);
+    p.Qg = (bf16*)(a.ws + a.TL.Qg); p.P = (bf16*)(a.ws + a.TL.P);
+    p.Wt = (bf16*)(a.ws + a.TL.Wt); p.Ut = (bf16*)(a.ws + a.TL.Ut);
+    p.status = (unsigned*)(a.ws + a.TL.status);
+    cudaError_t e = set_smem(k_tc_prep, kPrepSmem);
+    if (e != cudaSuccess) return e;
+    const int grid = s.B * s.H * (p.N / 2);
+    k_tc_prep<<<grid, 128, kPrepSmem, a.stream>>>(mQ, mK, mV, p);
+    return cudaGetLastError();
+}
+
+cudaError_t tc_chain_fwd(const ChunkArgs& a) {
+    const qd_shape& s = a.s;
+    const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
+    CUtensorMap mWt, mUt, mQg, mK, mP;
+    if (!make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, BH * N * D, 128, 128) ||
+        !make_tmap_bf16_2d(&mUt, a.ws + a.TL.Ut, 64, BH * N * D, 128, 128) ||
+        !make_tmap_bf16_2d(&mQg, a.ws + a.TL.Qg, D, BH * s.T, D * 2, 64) ||
+        !make_tmap_bf16_2d(&mK, a.k, (uint64_t)s.H * D, (uint64_t)s.B * s.T, (uint64_t)s.H * D * 2, 64) ||
+        !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * s.T, 128, 64))
+        return cudaErrorInvalidValue;
+    ChainParams p{};
+    p.T = s.T; p.H = s.H; p.N = (int)N;
+    p.g = (const float*)(a.ws + a.TL.g);
+    p.h0 = a.h0; p.o = (bf16*)a.o; p.hT = a.hT;
+    p.status = (unsigned*)(a.ws + a.TL.status);
+    cudaError_t e = set_smem(k_tc_chain_fwd, kChainSmem);
+    if (e != cudaSuccess) return e;
+    k_tc_chain_fwd<<<(unsigned)BH, 128, kChainSmem, a.stream>>>(mWt, mUt, mQg, mK, mP, p);
+    return cudaGetLastError();
+}
+
+}  // namespace qd

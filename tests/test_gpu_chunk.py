@@ -154,3 +154,15 @@ def test_cfg3_long_context_full_size():
     pairs = _sample_pairs(cfg, 4)
     _fwd_check(cfg, d, pairs)
     _bwd_check(cfg, d, pairs, reuse=True)
+
+
+@pytest.mark.parametrize("regime", gen.REGIMES)
+def test_tensor_core_forward_regimes(regime):
+    # bf16, d = 128, T a multiple of 128: the tcgen05 kernels run the forward
+    cfg = replace(gen.CONFIGS["cfg1"], B=2, H=3, T=384, regime=regime, seed=17)
+    _fwd_check(cfg)
+
+
+def test_tensor_core_forward_single_pair_no_h0():
+    cfg = replace(gen.CONFIGS["cfg1"], B=1, H=1, T=128, h0=False, seed=19)
+    _fwd_check(cfg)
