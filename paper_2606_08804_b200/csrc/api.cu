@@ -95,7 +95,8 @@ size_t qdelta_chunk_workspace_bytes(const qd_shape* shape, int for_backward) {
     size_t n = for_backward ? L.bwd_end : L.fwd_end;
     if (tc_supported(*shape)) {
         TcLayout TL = tc_layout(*shape);
-        if (TL.fwd_end > n) n = TL.fwd_end;
+        const size_t m = for_backward ? TL.bwd_end : TL.fwd_end;
+        if (m > n) n = m;
     }
     return n;
 }
@@ -122,9 +123,9 @@ int qdelta_chunk_fwd(const qd_shape* shape, const void* q, const void* k, const 
     a.ws = (char*)workspace;
     a.stream = (cudaStream_t)stream;
     if (cudaMemsetAsync(a.ws + a.L.status, 0, 256, a.stream) != cudaSuccess) return QD_ERR_CUDA;
-    if (!a.save && tc_supported(*shape)) {
+    if (tc_supported(*shape)) {
         a.TL = tc_layout(*shape);
-        if (workspace_bytes < a.TL.fwd_end) return QD_ERR_WORKSPACE;
+        if (workspace_bytes < (a.save ? a.TL.bwd_end : a.TL.fwd_end)) return QD_ERR_WORKSPACE;
         if (timed(ST_PREP, a.stream, [&] { return tc_prep(a); }) != cudaSuccess) return QD_ERR_CUDA;
         if (timed(ST_CHAIN_FWD, a.stream, [&] { return tc_chain_fwd(a); }) != cudaSuccess) return QD_ERR_CUDA;
         return QD_OK;
@@ -162,6 +163,22 @@ int qdelta_chunk_bwd(const qd_shape* shape, const void* q, const void* k, const 
     a.dbeta = dbeta; a.dalpha = dalpha; a.dlam = dlambda; a.dh0 = dh0;
     a.ws = (char*)workspace;
     a.stream = (cudaStream_t)stream;
+    if (tc_supported(*shape)) {
+        a.TL = tc_layout(*shape);
+        if (workspace_bytes < a.TL.bwd_end) return QD_ERR_WORKSPACE;
+        if (!(flags & QD_BWD_REUSE_FWD)) {
+            // recompute what a saving forward leaves behind; its o goes to the dDelta section, which
+            // the reverse chain overwrites afterwards
+            if (cudaMemsetAsync(a.ws + a.TL.status, 0, 256, a.stream) != cudaSuccess) return QD_ERR_CUDA;
+            a.o = a.ws + a.TL.dDt;
+            a.hT = nullptr;
+            if (timed(ST_PREP, a.stream, [&] { return tc_prep(a); }) != cudaSuccess) return QD_ERR_CUDA;
+            if (timed(ST_CHAIN_FWD, a.stream, [&] { return tc_chain_fwd(a); }) != cudaSuccess) return QD_ERR_CUDA;
+        }
+        if (timed(ST_CHAIN_BWD, a.stream, [&] { return tc_chain_bwd(a); }) != cudaSuccess) return QD_ERR_CUDA;
+        if (timed(ST_CHUNK_BWD, a.stream, [&] { return tc_chunk_bwd(a); }) != cudaSuccess) return QD_ERR_CUDA;
+        return QD_OK;
+    }
     if (!(flags & QD_BWD_REUSE_FWD)) {
         // recompute the forward intermediates (outputs of the forward itself are not rewritten:
         // o goes to the dD section, which the reverse chain overwrites afterwards)

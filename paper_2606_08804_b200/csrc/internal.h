@@ -45,6 +45,13 @@ struct TcLayout {
     size_t Wt;       // bf16 [BH*N][dk][C]     (T diag(gamma) X)^T per chunk
     size_t Ut;       // bf16 [BH*N][dv][C]     (T V)^T per chunk
     size_t fwd_end;
+    // kept for / produced by the backward
+    size_t Mt;       // bf16 [BH*N][C][C]      ((I+A)^-1)^T per chunk: [column][row]
+    size_t hsT;      // bf16 [BH*N][dv][dk]    h^T at the entry of every chunk
+    size_t Dt;       // bf16 [BH*N][dv][C]     Delta^T per chunk
+    size_t dhsT;     // bf16 [BH*N][dv][dk]    (dL/dh)^T at the exit of every chunk
+    size_t dDt;      // bf16 [BH*N][dv][C]     (dL/dDelta)^T per chunk
+    size_t bwd_end;
 };
 TcLayout tc_layout(const qd_shape& s);
 bool tc_supported(const qd_shape& s);
@@ -76,6 +83,8 @@ cudaError_t simt_chunk_bwd(const ChunkArgs& a);   // dq, dk, dv, dbeta, dalpha, 
 // tcgen05 path
 cudaError_t tc_prep(const ChunkArgs& a);
 cudaError_t tc_chain_fwd(const ChunkArgs& a);
+cudaError_t tc_chain_bwd(const ChunkArgs& a);
+cudaError_t tc_chunk_bwd(const ChunkArgs& a);
 
 cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
                         const void* beta, const void* alpha, const void* lam, float* state, void* o,

@@ -1,0 +1,695 @@
+// Tensor-core (tcgen05 / TMEM / TMA) chunkwise backward for bf16, d_k = d_v = 128, chunk 64.
+//
+// The paper prints no backward pass; these kernels evaluate the exact gradient of the chunk
+// equations of Section 3.3.2 (see the forward kernels for the notation):
+//   k_tc_chain_bwd  one CTA per (batch, head), chunks in REVERSE order, dh^T (fp32) in registers:
+//                     dDelta^T = dO^T P + diag-scaled (dh^T K^T)          (scale gamma_C/gamma_s per token s)
+//                     dh^T <- gamma_C dh^T + dO^T Qg - dDelta^T W<-
+//                   leaves per chunk dDelta^T and the bf16 dh^T at the chunk's exit.
+//   k_tc_chunk_bwd  one CTA per chunk: every remaining product (dP, dT, dA = -M^T dM M^T, dX, ...),
+//                   d_k/d_v-shaped results transposed (d index on the 128 TMEM lanes), 64 x 64-shaped
+//                   ones in natural orientation on lanes 0..63; row dot-products that run across lanes
+//                   use a warp-shuffle column reduction.
+// All waits are bounded (see tc_fwd.cu).
+#include "internal.h"
+#include "sm100.cuh"
+
+namespace qd {
+namespace {
+using namespace sm100;
+typedef __nv_bfloat16 bf16;
+
+constexpr int C = kChunk;      // 64
+constexpr int D = 128;         // d_k = d_v
+
+__device__ __forceinline__ void load8(const unsigned char* p, float* f) {
+    const uint4 u = *reinterpret_cast<const uint4*>(p);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { const float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+}
+__device__ __forceinline__ uint4 pack8(const float* f) {
+    uint4 u;
+    u.x = pack_bf16(f[0], f[1]); u.y = pack_bf16(f[2], f[3]); u.z = pack_bf16(f[4], f[5]); u.w = pack_bf16(f[6], f[7]);
+    return u;
+}
+// 64 TMEM columns of this thread's lane
+__device__ __forceinline__ void ld64(uint32_t taddr, float* v) {
+    tmem_ld32(taddr, v);
+    tmem_ld32(taddr + 32, v + 32);
+    tmem_ld_wait();
+}
+
+// Column sums across the 32 lanes of a warp: every lane passes 64 values; on return v[0], v[1] hold
+// the warp-wide sums of columns col, col+1 with col = col_of_lane(lane).
+template <int N>
+__device__ __forceinline__ void fold(float* v, int lane, int off) {
+    const bool up = (lane & off) != 0;
+#pragma unroll
+    for (int k = 0; k < N / 2; ++k) {
+        const float keep = up ? v[N / 2 + k] : v[k];
+        const float send = up ? v[k] : v[N / 2 + k];
+        v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+    }
+}
+__device__ __forceinline__ void col_reduce64(float* v, int lane) {
+    fold<64>(v, lane, 16); fold<32>(v, lane, 8); fold<16>(v, lane, 4); fold<8>(v, lane, 2); fold<4>(v, lane, 1);
+}
+__device__ __forceinline__ int col_of_lane(int lane) {
+    return ((lane & 16) ? 32 : 0) + ((lane & 8) ? 16 : 0) + ((lane & 4) ? 8 : 0) + ((lane & 2) ? 4 : 0) + ((lane & 1) ? 2 : 0);
+}
+
+// =================================================================================================
+struct ChainBwdParams {
+    int T, H, N;
+    const float* g;
+    const float* dhT;
+    float* dh0;
+    bf16* dDt;
+    unsigned* status;
+};
+
+constexpr int kStage = 73728;                           // Wt 16K | dO 16K | Qg 16K | K 16K | P 8K
+constexpr int kChainSmem = 2 * kStage + 32768 + 16384 + 1024;
+
+__global__ void __launch_bounds__(128) k_tc_chain_bwd(const __grid_constant__ CUtensorMap mapWt,
+                                                      const __grid_constant__ CUtensorMap mapdO,
+                                                      const __grid_constant__ CUtensorMap mapQg,
+                                                      const __grid_constant__ CUtensorMap mapK,
+                                                      const __grid_constant__ CUtensorMap mapP,
+                                                      const __grid_constant__ CUtensorMap mapdHs, ChainBwdParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char* sdH = smem + 2 * kStage;         // dh^T as A operand: K-major, 2 blocks of [128 lines][64]
+    unsigned char* sdD = sdH + 32768;               // dDelta^T: K-major [128 lines (dv)][64 tokens]
+    __shared__ uint64_t bar_load[2], bar_a, bar_b;
+    __shared__ uint32_t tmem_slot;
+    __shared__ float sg[2][C];
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int bh = blockIdx.x, b = bh / p.H, hh = bh % p.H;
+
+    if (tid == 0) {
+        mbar_init(&bar_load[0], 1); mbar_init(&bar_load[1], 1);
+        mbar_init(&bar_a, 1); mbar_init(&bar_b, 1);
+        mbar_init_fence();
+    }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tbase = tmem_slot;
+    const uint32_t tA1 = tbase, tA2 = tbase + 64, tH = tbase + 128;
+
+    // iteration `it` processes chunk n = N-1-it
+    auto issue_load = [&](int it) {
+        const int n = p.N - 1 - it;
+        unsigned char* st = smem + (it & 1) * kStage;
+        uint64_t* bar = &bar_load[it & 1];
+        mbar_expect_tx(bar, kStage);
+        const int yc = (int)(((size_t)bh * p.N + n) * D);
+        const int yt = (int)((size_t)bh * p.T + (size_t)n * C);
+        const int yi = (int)((size_t)b * p.T + (size_t)n * C);
+        tma_load_2d(st, &mapWt, 0, yc, bar);
+        tma_load_2d(st + 16384, &mapdO, hh * D, yi, bar);
+        tma_load_2d(st + 16384 + 8192, &mapdO, hh * D + 64, yi, bar);
+        tma_load_2d(st + 32768, &mapQg, 0, yt, bar);
+        tma_load_2d(st + 32768 + 8192, &mapQg, 64, yt, bar);
+        tma_load_2d(st + 49152, &mapK, hh * D, yi, bar);
+        tma_load_2d(st + 49152 + 8192, &mapK, hh * D + 64, yi, bar);
+        tma_load_2d(st + 65536, &mapP, 0, yt, bar);
+    };
+    if (tid == 0) { issue_load(0); if (p.N > 1) issue_load(1); }
+
+    float dh[D];      // row j of dh^T
+    if (p.dhT) {
+        const float* src = p.dhT + (size_t)bh * D * D + tid;
+#pragma unroll
+        for (int i = 0; i < D; ++i) dh[i] = src[(size_t)i * D];
+    } else {
+#pragma unroll
+        for (int i = 0; i < D; ++i) dh[i] = 0.f;
+    }
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk)
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch)
+            *reinterpret_cast<uint4*>(sdH + blk * 16384 + sw128_chunk(tid, ch)) = pack8(dh + blk * 64 + ch * 8);
+    if (tid < C) sg[0][tid] = p.g[(size_t)bh * p.T + (size_t)(p.N - 1) * C + tid];
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+
+    bool aborted = false;
+    int loads_waited = 0;
+    for (int it = 0; it < p.N; ++it) {
+        const int n = p.N - 1 - it;
+        unsigned char* st = smem + (it & 1) * kStage;
+        const float* gc = sg[it & 1];
+        bool fail = !mbar_wait(&bar_load[it & 1], (it >> 1) & 1);
+        if (__syncthreads_or(fail)) { aborted = true; break; }
+        loads_waited = it + 1;
+        if (tid == 0) {
+            // gradient w.r.t. the exit state of chunk n, bf16, as the operand tile (rows = d_v, cols = d_k)
+            const int yh = (int)(((size_t)bh * p.N + n) * D);
+            tma_store_2d(&mapdHs, sdH, 0, yh);
+            tma_store_2d(&mapdHs, sdH + 16384, 64, yh);
+            tma_store_commit();
+            tc_fence_after();
+            const uint32_t sdO = smem_u32(st + 16384);
+            // A1 = dO^T P  (A, B MN-major: lines = token r);  A2 = dh^T K^T (A, B K-major)
+            umma_product<true, true>(tA1, sdO, 8192, smem_u32(st + 65536), 8192, C, C, false);
+            umma_product<false, false>(tA2, smem_u32(sdH), 16384, smem_u32(st + 49152), 8192, C, D, false);
+            // H-accumulator = dO^T Qg (B MN-major: lines = token r, two blocks of d_k)
+            umma_product<true, true>(tH, sdO, 8192, smem_u32(st + 32768), 8192, D, C, false);
+            umma_commit(&bar_a);
+        }
+        fail = !mbar_wait(&bar_a, it & 1);
+        if (__syncthreads_or(fail)) { aborted = true; break; }
+        tc_fence_after();
+        {
+            const float gC = gc[C - 1];
+            bf16* drow = p.dDt + (((size_t)bh * p.N + n) * D + tid) * C;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                float a1[32], a2[32];
+                tmem_ld32(tmem_addr(tA1, warp * 32, half * 32), a1);
+                tmem_ld32(tmem_addr(tA2, warp * 32, half * 32), a2);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) a1[i] = fmaf(expf(gC - gc[half * 32 + i]), a2[i], a1[i]);
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    const uint4 pk = pack8(a1 + ch * 8);
+                    *reinterpret_cast<uint4*>(sdD + sw128_chunk(tid, half * 4 + ch)) = pk;
+                    *reinterpret_cast<uint4*>(drow + half * 32 + ch * 8) = pk;
+                }
+            }
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            // H-accumulator -= dDelta^T W<-   (A negated; B K-major: lines = d_k index, contraction over tokens)
+            umma_product<false, false>(tH, smem_u32(sdD), 16384, smem_u32(st), 16384, D, C, true, true);
+            umma_commit(&bar_b);
+        }
+        fail = !mbar_wait(&bar_b, it & 1);
+        if (tid == 0) tma_store_wait_read();
+        if (__syncthreads_or(fail)) { aborted = true; break; }
+        tc_fence_after();
+        if (tid == 0 && it + 2 < p.N) issue_load(it + 2);
+        {
+            const float gamC = expf(gc[C - 1]);
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                float v[32];
+                tmem_ld32(tmem_addr(tH, warp * 32, q4 * 32), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) dh[q4 * 32 + i] = fmaf(gamC, dh[q4 * 32 + i], v[i]);
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch)
+                    *reinterpret_cast<uint4*>(sdH + (q4 >> 1) * 16384 + sw128_chunk(tid, (q4 & 1) * 4 + ch)) =
+                        pack8(dh + q4 * 32 + ch * 8);
+            }
+        }
+        if (tid < C && n >= 1) sg[(it + 1) & 1][tid] = p.g[(size_t)bh * p.T + (size_t)(n - 1) * C + tid];
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+    }
+    if (aborted) {
+        if (tid == 0) {
+            *p.status = QD_ERR_TIMEOUT;
+            for (int it = loads_waited; it < p.N && it < loads_waited + 2; ++it) mbar_wait(&bar_load[it & 1], (it >> 1) & 1);
+        }
+    } else if (p.dh0) {
+        float* dst = p.dh0 + (size_t)bh * D * D + tid;
+#pragma unroll
+        for (int i = 0; i < D; ++i) dst[(size_t)i * D] = dh[i];
+    }
+    if (tid == 0) tma_store_wait_all();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tbase, 256);
+}
+
+// =================================================================================================
+struct ChunkBwdParams {
+    int T, H, N;
+    const bf16 *beta, *alpha, *lam;
+    const float* g;
+    bf16 *dq, *dk, *dv;
+    float *dbeta, *dalpha, *dlam;
+    unsigned* status;
+};
+
+// shared-memory map of k_tc_chunk_bwd (bytes from the 1024-aligned base)
+constexpr int oQ = 0, oK = 16384, oV = 32768, odO = 49152, oX = 65536, oMt = 81920, oP = 90112, oDt = 98304,
+              odDt = 114688, oH = 131072, odH = 163840, kBwdLoadBytes = 180224;   // all TMA-loaded tiles (X is built)
+constexpr int odPG = oV, odTb = oV + 8192, odW = odO, oN = oH, odXK = oH + 8192, oPP = oH + 16384,
+              oAA = odH + 1024;
+constexpr int kBwdSmem = 196608 + 1024;
+constexpr int LDAA = C + 1;
+
+__global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CUtensorMap mapQ,
+                                                      const __grid_constant__ CUtensorMap mapK,
+                                                      const __grid_constant__ CUtensorMap mapV,
+                                                      const __grid_constant__ CUtensorMap mapdO,
+                                                      const __grid_constant__ CUtensorMap mapMt,
+                                                      const __grid_constant__ CUtensorMap mapP,
+                                                      const __grid_constant__ CUtensorMap mapDt,
+                                                      const __grid_constant__ CUtensorMap mapdDt,
+                                                      const __grid_constant__ CUtensorMap mapHs,
+                                                      const __grid_constant__ CUtensorMap mapdHs, ChunkBwdParams p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* sm = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ uint64_t bar_load, bar_mma;
+    __shared__ uint32_t tmem_slot;
+    __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C], segc[C];
+    __shared__ float sred[3][4][C];          // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
+    __shared__ float sdg[C], swp[4];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int ch_id = blockIdx.x, n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
+    const size_t row0 = (size_t)b * p.T + (size_t)n * C;          // token row in the [B*T] view
+    const size_t wrow0 = (size_t)bh * p.T + (size_t)n * C;        // token row in the [BH*T] view
+
+    if (tid == 0) {
+        mbar_init(&bar_load, 1);
+        mbar_init(&bar_mma, 1);
+        mbar_init_fence();
+    }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_slot;
+    const uint32_t T0 = tb, T1 = tb + 64, T2 = tb + 128, T3 = tb + 192, T4 = tb + 256, T5 = tb + 320, T6 = tb + 384,
+                   T7 = tb + 448;
+    const uint32_t lane_base = (uint32_t)warp * 32;
+
+    if (tid == 0) {
+        mbar_expect_tx(&bar_load, kBwdLoadBytes);
+        const int yi = (int)row0, yt = (int)wrow0;
+        const int yc = (int)(((size_t)bh * p.N + n) * D), ym = (int)(((size_t)bh * p.N + n) * C);
+        for (int blk = 0; blk < 2; ++blk) {
+            tma_load_2d(sm + oQ + blk * 8192, &mapQ, hh * D + blk * 64, yi, &bar_load);
+            tma_load_2d(sm + oK + blk * 8192, &mapK, hh * D + blk * 64, yi, &bar_load);
+            tma_load_2d(sm + oV + blk * 8192, &mapV, hh * D + blk * 64, yi, &bar_load);
+            tma_load_2d(sm + odO + blk * 8192, &mapdO, hh * D + blk * 64, yi, &bar_load);
+            tma_load_2d(sm + oH + blk * 16384, &mapHs, blk * 64, yc, &bar_load);
+            tma_load_2d(sm + odH + blk * 16384, &mapdHs, blk * 64, yc, &bar_load);
+        }
+        tma_load_2d(sm + oMt, &mapMt, 0, ym, &bar_load);
+        tma_load_2d(sm + oP, &mapP, 0, yt, &bar_load);
+        tma_load_2d(sm + oDt, &mapDt, 0, yc, &bar_load);
+        tma_load_2d(sm + odDt, &mapdDt, 0, yc, &bar_load);
+    }
+    if (tid < C) {
+        const size_t cr = (row0 + tid) * p.H + hh;
+        sbeta[tid] = __bfloat162float(p.beta[cr]);
+        slam[tid] = p.lam ? __bfloat162float(p.lam[cr]) : 0.f;
+        salpha[tid] = p.alpha ? __bfloat162float(p.alpha[cr]) : 1.f;
+        const float gv = p.g[wrow0 + tid];
+        sg[tid] = gv;
+        sgam[tid] = expf(gv);
+    }
+    __syncthreads();
+    if (tid < C) segc[tid] = expf(sg[C - 1] - sg[tid]);
+
+    bool fail = !mbar_wait(&bar_load, 0);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        mbar_wait(&bar_load, 0);
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tb, 512);
+        return;
+    }
+    // ---- phase 0: X = K + lambda Q; <dh,h>_F; <dDelta_r, Delta_r> -----------------------------------
+    {
+        const int r = tid & 63, blk = tid >> 6;
+        const float lm = slam[r];
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+            const uint32_t off = blk * 8192 + sw128_chunk(r, ch);
+            float qv[8], kv[8];
+            load8(sm + oQ + off, qv);
+            load8(sm + oK + off, kv);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) kv[e] = fmaf(lm, qv[e], kv[e]);
+            *reinterpret_cast<uint4*>(sm + oX + off) = pack8(kv);
+        }
+    }
+    float dhh_part = 0.f;
+    {
+#pragma unroll
+        for (int blk = 0; blk < 2; ++blk)
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+                const uint32_t off = blk * 16384 + sw128_chunk(tid, ch);
+                float a[8], c8[8];
+                load8(sm + oH + off, a);
+                load8(sm + odH + off, c8);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) dhh_part = fmaf(a[e], c8[e], dhh_part);
+            }
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    // ---- phase 1 products ------------------------------------------------------------------------
+    const uint32_t aQ = smem_u32(sm + oQ), aK = smem_u32(sm + oK), aV = smem_u32(sm + oV), adO = smem_u32(sm + odO),
+                   aX = smem_u32(sm + oX), aMt = smem_u32(sm + oMt), aDt = smem_u32(sm + oDt),
+                   adDt = smem_u32(sm + odDt), aH = smem_u32(sm + oH), adH = smem_u32(sm + odH);
+    const uint32_t adPG = smem_u32(sm + odPG), adTb = smem_u32(sm + odTb), adW = smem_u32(sm + odW),
+                   aN = smem_u32(sm + oN), adXK = smem_u32(sm + odXK);
+    if (tid == 0) {
+        tc_fence_after();
+        umma_product<false, false>(T0, aX, 8192, aK, 8192, C, D, false);            // X K^T            [r][i]
+        umma_product<false, true>(T1, adO, 8192, aDt, 8192, C, D, false);           // dO Delta^T       [r][s]
+        umma_product<false, true>(T2, aV, 8192, adDt, 8192, C, D, false);           // V dDelta^T       [s][r]
+        umma_product<true, true>(T3, aH, 16384, adDt, 8192, C, D, false, true);     // -h dDelta^T      [i][r] = dW<-^T
+        umma_product<true, false>(T4, aH, 16384, adO, 8192, C, D, false);           // h dO^T           [i][r]
+        umma_product<true, true>(T5, adH, 16384, aDt, 8192, C, D, false);           // dh Delta^T       [i][s]
+        umma_product<false, false>(T6, adDt, 16384, aMt, 8192, C, C, false);        // dDelta^T M       [j][s]
+        umma_product<false, false>(T7, adH, 16384, aK, 8192, C, D, false);          // dh^T K^T         [j][s]
+        umma_commit(&bar_mma);
+    }
+    fail = !mbar_wait(&bar_mma, 0);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        if (warp == 0) tmem_dealloc(tb, 512);
+        return;
+    }
+    tc_fence_after();
+    float rPP = 0.f;
+    float* sPP = reinterpret_cast<float*>(sm + oPP);
+    {
+        // <(K-> dh)_s, Delta_s>: (K-> dh)^T[j][s] = gamma_C/gamma_s (dh^T K^T)[j][s] in fp32, Delta^T[j][s] from its tile;
+        // the sum over j runs across lanes
+        float kd[C];
+        ld64(tmem_addr(T7, lane_base, 0), kd);
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+            float dl[8];
+            load8(sm + oDt + sw128_chunk(tid, ch), dl);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) kd[ch * 8 + e] *= segc[ch * 8 + e] * dl[e];
+        }
+        col_reduce64(kd, lane);
+        const int col = col_of_lane(lane);
+        sred[0][warp][col] = kd[0];
+        sred[0][warp][col + 1] = kd[1];
+    }
+    if (tid < C) {
+        // dP row r: causal mask, dP o P (row sums here, column sums later), dP o Gamma as an operand tile
+        const int r = tid;
+        float v[C], pg[C];
+        ld64(tmem_addr(T1, lane_base, 0), v);
+        const float gr = sg[r];
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+            float pv[8];
+            load8(sm + oP + sw128_chunk(r, ch), pv);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int s = ch * 8 + e;
+                const float dp = (s <= r) ? v[s] : 0.f;
+                const float pp = dp * pv[e];
+                rPP += pp;
+                sPP[r * LDAA + s] = pp;
+                pg[s] = (s <= r) ? dp * expf(gr - sg[s]) : 0.f;
+            }
+        }
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + odPG + sw128_chunk(r, ch)) = pack8(pg + ch * 8);
+    }
+    {
+        float v[C];
+        ld64(tmem_addr(T3, lane_base, 0), v);                      // dW<-^T row i = tid
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + odW + sw128_chunk(tid, ch)) = pack8(v + ch * 8);
+        ld64(tmem_addr(T6, lane_base, 0), v);                      // dV^T row j = tid, to be scaled by beta_s
+        bf16* dst = p.dv + (row0 * p.H + hh) * D + tid;
+#pragma unroll
+        for (int s = 0; s < C; ++s) dst[(size_t)s * p.H * D] = __float2bfloat16_rn(sbeta[s] * v[s]);
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    // ---- phase 2 ---------------------------------------------------------------------------------
+    if (tid == 0) {
+        tc_fence_after();
+        umma_product<false, true>(T7, aX, 8192, adW, 8192, C, D, false);            // X dW<-^T         [s][r]
+        umma_product<false, false>(T6, adW, 16384, aMt, 8192, C, C, false);         // dW<-^T M         [i][s]
+        umma_commit(&bar_mma);
+    }
+    fail = !mbar_wait(&bar_mma, 1);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        if (warp == 0) tmem_dealloc(tb, 512);
+        return;
+    }
+    tc_fence_after();
+    float dbeta = 0.f, t2 = 0.f;
+    if (tid < C) {
+        // dT^T row s = tid: dT[r][s] for all r;  M[r][s] = line s of Mt
+        const int s = tid;
+        float a[C], bq[C];
+        ld64(tmem_addr(T2, lane_base, 0), a);
+        ld64(tmem_addr(T7, lane_base, 0), bq);
+        const float gs = sgam[s], bs = sbeta[s];
+        float mb = 0.f;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+            float m[8];
+            load8(sm + oMt + sw128_chunk(s, ch), m);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int r = ch * 8 + e;
+                const float dt = fmaf(gs, bq[r], a[r]);
+                dbeta = fmaf(dt, m[e], dbeta);
+                mb = fmaf(m[e], bq[r], mb);
+                a[r] = bs * dt;
+            }
+        }
+        t2 = gs * bs * mb;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + odTb + sw128_chunk(s, ch)) = pack8(a + ch * 8);
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    // ---- phase 3: N~ = dT diag(beta) M^T ----------------------------------------------------------
+    if (tid == 0) {
+        tc_fence_after();
+        umma_product<true, true>(T1, adTb, 8192, aMt, 8192, C, C, false);           // [r][u]
+        umma_commit(&bar_mma);
+    }
+    fail = !mbar_wait(&bar_mma, 0);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        if (warp == 0) tmem_dealloc(tb, 512);
+        return;
+    }
+    tc_fence_after();
+    if (tid < C) {
+        float v[C];
+        ld64(tmem_addr(T1, lane_base, 0), v);
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + oN + sw128_chunk(tid, ch)) = pack8(v + ch * 8);
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    // ---- phase 4: dA = -M^T N~ ---------------------------------------------------------------------
+    if (tid == 0) {
+        tc_fence_after();
+        umma_product<false, true>(T2, aMt, 8192, aN, 8192, C, C, false, true);      // [r][s]
+        umma_commit(&bar_mma);
+    }
+    fail = !mbar_wait(&bar_mma, 1);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        if (warp == 0) tmem_dealloc(tb, 512);
+        return;
+    }
+    tc_fence_after();
+    float rAA = 0.f;
+    float* sAA = reinterpret_cast<float*>(sm + oAA);
+    if (tid < C) {
+        const int r = tid;
+        float da[C], xk[C];
+        ld64(tmem_addr(T2, lane_base, 0), da);
+        ld64(tmem_addr(T0, lane_base, 0), xk);
+        const float gr = sg[r], br = sbeta[r];
+#pragma unroll
+        for (int s = 0; s < C; ++s) {
+            const bool on = s < r;
+            const float gm = on ? expf(gr - sg[s]) : 0.f;
+            const float d = on ? da[s] : 0.f;
+            const float dgx = d * gm * xk[s];
+            dbeta += dgx;
+            const float aa = br * dgx;
+            rAA += aa;
+            sAA[r * LDAA + s] = aa;
+            da[s] = d * br * gm;                                   // dXK
+        }
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + odXK + sw128_chunk(r, ch)) = pack8(da + ch * 8);
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    // ---- phase 5 ---------------------------------------------------------------------------------
+    if (tid == 0) {
+        tc_fence_after();
+        umma_product<true, false>(T7, aK, 8192, adXK, 8192, C, C, false);           // (dXK K)^T        [i][r]
+        umma_product<true, true>(T1, aX, 8192, adXK, 8192, C, C, false);            // (dXK^T X)^T      [i][s]
+        umma_product<true, true>(T1, aQ, 8192, adPG, 8192, C, C, true);             // + (dPG^T Q)^T
+        umma_product<true, false>(T2, aK, 8192, adPG, 8192, C, C, false);           // (dPG K)^T        [i][r]
+        umma_commit(&bar_mma);
+    }
+    fail = !mbar_wait(&bar_mma, 0);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        if (warp == 0) tmem_dealloc(tb, 512);
+        return;
+    }
+    tc_fence_after();
+    {
+        const int i = tid;                                          // d_k index
+        float dx[C], v[C], w[C];
+        ld64(tmem_addr(T6, lane_base, 0), dx);
+        ld64(tmem_addr(T7, lane_base, 0), v);
+#pragma unroll
+        for (int s = 0; s < C; ++s) dx[s] = fmaf(sgam[s] * sbeta[s], dx[s], v[s]);       // dX^T[i][s]
+        // dk
+        ld64(tmem_addr(T1, lane_base, 0), v);
+        ld64(tmem_addr(T5, lane_base, 0), w);
+        {
+            bf16* dst = p.dk + (row0 * p.H + hh) * D + i;
+#pragma unroll
+            for (int s = 0; s < C; ++s)
+                dst[(size_t)s * p.H * D] = __float2bfloat16_rn(v[s] + segc[s] * w[s] + dx[s]);
+        }
+        // dq, and the two row dot-products with Q that run across lanes
+        ld64(tmem_addr(T4, lane_base, 0), v);
+        ld64(tmem_addr(T2, lane_base, 0), w);
+        {
+            bf16* dst = p.dq + (row0 * p.H + hh) * D + i;
+            const unsigned char* qcol = sm + oQ + (i >> 6) * 8192;
+#pragma unroll
+            for (int r = 0; r < C; ++r) {
+                const float q1 = sgam[r] * v[r];
+                dst[(size_t)r * p.H * D] = __float2bfloat16_rn(q1 + w[r] + slam[r] * dx[r]);
+                const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(r, i & 63)));
+                v[r] = q1 * qv;
+                dx[r] = dx[r] * qv;
+            }
+        }
+        col_reduce64(dx, lane);
+        col_reduce64(v, lane);
+        const int col = col_of_lane(lane);
+        sred[1][warp][col] = dx[0]; sred[1][warp][col + 1] = dx[1];
+        sred[2][warp][col] = v[0];  sred[2][warp][col + 1] = v[1];
+    }
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 16);
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 8);
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 4);
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 2);
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 1);
+    if (lane == 0) swp[warp] = dhh_part;
+    __syncthreads();
+    // ---- decay gradient ----------------------------------------------------------------------------
+    if (tid < C) {
+        const int r = tid;
+        float kd = 0.f, dl = 0.f, t1 = 0.f, cAA = 0.f, cPP = 0.f;
+#pragma unroll
+        for (int w4 = 0; w4 < 4; ++w4) { kd += sred[0][w4][r]; dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
+        for (int u = r + 1; u < C; ++u) cAA += sAA[u * LDAA + r];
+        for (int u = r; u < C; ++u) cPP += sPP[u * LDAA + r];
+        sdg[r] = t1 + rPP - cPP + t2 + rAA - cAA - kd;
+        sred[0][0][r] = kd;                     // summed below into dg of the last token
+        p.dbeta[(row0 + r) * p.H + hh] = dbeta;
+        if (p.dlam) p.dlam[(row0 + r) * p.H + hh] = dl;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float tot = 0.f;
+        for (int r = 0; r < C; ++r) tot += sred[0][0][r];
+        sdg[C - 1] += sgam[C - 1] * (swp[0] + swp[1] + swp[2] + swp[3]) + tot;
+        float acc = 0.f;
+        for (int r = C - 1; r >= 0; --r) { acc += sdg[r]; sdg[r] = acc; }
+    }
+    __syncthreads();
+    if (tid < C && p.dalpha) p.dalpha[(row0 + tid) * p.H + hh] = sdg[tid] / salpha[tid];
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tb, 512);
+}
+
+template <class K>
+cudaError_t set_smem(K kern, size_t bytes) {
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+}  // namespace
+
+cudaError_t tc_chain_bwd(const ChunkArgs& a) {
+    const qd_shape& s = a.s;
+    const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
+    const uint64_t icols = (uint64_t)s.H * D, irows = (uint64_t)s.B * s.T;
+    CUtensorMap mWt, mdO, mQg, mK, mP, mdHs;
+    if (!make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, BH * N * D, 128, 128) ||
+        !make_tmap_bf16_2d(&mdO, a.dO, icols, irows, icols * 2, 64) ||
+        !make_tmap_bf16_2d(&mQg, a.ws + a.TL.Qg, D, BH * s.T, D * 2, 64) ||
+        !make_tmap_bf16_2d(&mK, a.k, icols, irows, icols * 2, 64) ||
+        !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * s.T, 128, 64) ||
+        !make_tmap_bf16_2d(&mdHs, a.ws + a.TL.dhsT, D, BH * N * D, D * 2, 128))
+        return cudaErrorInvalidValue;
+    ChainBwdParams p{};
+    p.T = s.T; p.H = s.H; p.N = (int)N;
+    p.g = (const float*)(a.ws + a.TL.g);
+    p.dhT = a.dhT; p.dh0 = a.dh0;
+    p.dDt = (bf16*)(a.ws + a.TL.dDt);
+    p.status = (unsigned*)(a.ws + a.TL.status);
+    cudaError_t e = set_smem(k_tc_chain_bwd, kChainSmem);
+    if (e != cudaSuccess) return e;
+    k_tc_chain_bwd<<<(unsigned)BH, 128, kChainSmem, a.stream>>>(mWt, mdO, mQg, mK, mP, mdHs, p);
+    return cudaGetLastError();
+}
+
+cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
+    const qd_shape& s = a.s;
+    const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
+    const uint64_t icols = (uint64_t)s.H * D, irows = (uint64_t)s.B * s.T;
+    CUtensorMap mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs;
+    if (!make_tmap_bf16_2d(&mQ, a.q, icols, irows, icols * 2, 64) ||
+        !make_tmap_bf16_2d(&mK, a.k, icols, irows, icols * 2, 64) ||
+        !make_tmap_bf16_2d(&mV, a.v, icols, irows, icols * 2, 64) ||
+        !make_tmap_bf16_2d(&mdO, a.dO, icols, irows, icols * 2, 64) ||
+        !make_tmap_bf16_2d(&mMt, a.ws + a.TL.Mt, 64, BH * s.T, 128, 64) ||
+        !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * s.T, 128, 64) ||
+        !make_tmap_bf16_2d(&mDt, a.ws + a.TL.Dt, 64, BH * N * D, 128, 128) ||
+        !make_tmap_bf16_2d(&mdDt, a.ws + a.TL.dDt, 64, BH * N * D, 128, 128) ||
+        !make_tmap_bf16_2d(&mHs, a.ws + a.TL.hsT, D, BH * N * D, D * 2, 128) ||
+        !make_tmap_bf16_2d(&mdHs, a.ws + a.TL.dhsT, D, BH * N * D, D * 2, 128))
+        return cudaErrorInvalidValue;
+    ChunkBwdParams p{};
+    p.T = s.T; p.H = s.H; p.N = (int)N;
+    p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
+    p.g = (const float*)(a.ws + a.TL.g);
+    p.dq = (bf16*)a.dq; p.dk = (bf16*)a.dk; p.dv = (bf16*)a.dv;
+    p.dbeta = a.dbeta; p.dalpha = a.dalpha; p.dlam = a.dlam;
+    p.status = (unsigned*)(a.ws + a.TL.status);
+    cudaError_t e = set_smem(k_tc_chunk_bwd, kBwdSmem);
+    if (e != cudaSuccess) return e;
+    k_tc_chunk_bwd<<<(unsigned)(BH * N), 128, kBwdSmem, a.stream>>>(mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs, p);
+    return cudaGetLastError();
+}
+
+}  // namespace qd

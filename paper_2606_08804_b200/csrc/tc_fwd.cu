@@ -43,6 +43,7 @@ struct PrepParams {
     const bf16 *beta, *alpha, *lam;
     float* g;
     bf16 *Qg, *P, *Wt, *Ut;
+    bf16* Mt;                  // optional: ((I+A)^-1)^T per chunk, [column i][row r]; kept for the backward
     unsigned* status;
 };
 
@@ -193,16 +194,18 @@ __global__ void __launch_bounds__(128) k_tc_prep(const __grid_constant__ CUtenso
         const float* M = sM + c * C * LDA;
         unsigned char* t0 = sT + c * 8192;
         unsigned char* t1 = sT + 16384 + c * 8192;
+        bf16* mt = p.Mt ? p.Mt + (((size_t)bh * p.N + 2 * pr + c) * C + r) * C : nullptr;
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) {
-            float a[8], bq[8];
+            float m0[8], a[8], bq[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const float m = M[(ch * 8 + e) * LDA + r] * beta;
-                a[e] = m; bq[e] = m * gam;
+                m0[e] = M[(ch * 8 + e) * LDA + r];
+                a[e] = m0[e] * beta; bq[e] = a[e] * gam;
             }
             *reinterpret_cast<uint4*>(t0 + sw128_chunk(r, ch)) = pack8(a);
             *reinterpret_cast<uint4*>(t1 + sw128_chunk(r, ch)) = pack8(bq);
+            if (mt) *reinterpret_cast<uint4*>(mt + ch * 8) = pack8(m0);
         }
     }
     fence_proxy_async();
@@ -253,6 +256,8 @@ struct ChainParams {
     const float* h0;
     bf16* o;
     float* hT;
+    bf16* Dt;                  // optional: Delta^T per chunk [dv][64]; kept for the backward
+    int save;                  // also store the bf16 entry state of every chunk through mapHs
     unsigned* status;
 };
 
@@ -263,7 +268,8 @@ __global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CU
                                                       const __grid_constant__ CUtensorMap mapUt,
                                                       const __grid_constant__ CUtensorMap mapQg,
                                                       const __grid_constant__ CUtensorMap mapK,
-                                                      const __grid_constant__ CUtensorMap mapP, ChainParams p) {
+                                                      const __grid_constant__ CUtensorMap mapP,
+                                                      const __grid_constant__ CUtensorMap mapHs, ChainParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char* sH = smem + 2 * kStage;          // h^T as A operand: K-major, 2 blocks of [128 lines][64]
@@ -334,6 +340,13 @@ __global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CU
         if (__syncthreads_or(fail)) { aborted = true; break; }
         loads_waited = n + 1;
         if (tid == 0) {
+            if (p.save) {
+                // entry state of chunk n, bf16, exactly the operand tile: rows = d_v index, cols = d_k index
+                const int yh = (int)(((size_t)bh * p.N + n) * D);
+                tma_store_2d(&mapHs, sH, 0, yh);
+                tma_store_2d(&mapHs, sH + 16384, 64, yh);
+                tma_store_commit();
+            }
             tc_fence_after();
             // Delta-accumulator = h^T Wt (B: MN-major, lines = d_k);  O-accumulator = h^T Qg^T (B: K-major)
             umma_product<false, true>(tD, smem_u32(sH), 16384, smem_u32(st), 8192, C, D, false);
@@ -362,8 +375,11 @@ __global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CU
                         d0[e] = u[e] - v[ch * 8 + e];
                         d1[e] = d0[e] * expf(gC - gc[half * 32 + ch * 8 + e]);
                     }
-                    *reinterpret_cast<uint4*>(sD + off) = pack8(d0);
+                    const uint4 pk = pack8(d0);
+                    *reinterpret_cast<uint4*>(sD + off) = pk;
                     *reinterpret_cast<uint4*>(sDs + off) = pack8(d1);
+                    if (p.Dt)
+                        *reinterpret_cast<uint4*>(p.Dt + (((size_t)bh * p.N + n) * D + tid) * C + half * 32 + ch * 8) = pk;
                 }
             }
         }
@@ -378,6 +394,7 @@ __global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CU
             umma_commit(&bar_b);
         }
         fail = !mbar_wait(&bar_b, n & 1);
+        if (tid == 0 && p.save) tma_store_wait_read();      // the state tile is about to be rewritten
         if (__syncthreads_or(fail)) { aborted = true; break; }
         tc_fence_after();
         // this stage's tiles are consumed: refill it with chunk n+2
@@ -426,6 +443,7 @@ __global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CU
 #pragma unroll
         for (int i = 0; i < D; ++i) dst[(size_t)i * D] = h[i];
     }
+    if (tid == 0 && p.save) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tbase, 256);
@@ -455,6 +473,13 @@ TcLayout tc_layout(const qd_shape& s) {
     L.Wt = take(BH * T * s.dk * 2);
     L.Ut = take(BH * T * s.dv * 2);
     L.fwd_end = off;
+    const size_t N = T / kChunk;
+    L.Mt = take(BH * T * kChunk * 2);
+    L.hsT = take(BH * N * s.dk * s.dv * 2);
+    L.Dt = take(BH * T * s.dv * 2);
+    L.dhsT = take(BH * N * s.dk * s.dv * 2);
+    L.dDt = take(BH * T * s.dv * 2);
+    L.bwd_end = off;
     return L;
 }
 
@@ -471,6 +496,7 @@ cudaError_t tc_prep(const ChunkArgs& a) {
     p.g = (float*)(a.ws + a.TL.g);
     p.Qg = (bf16*)(a.ws + a.TL.Qg); p.P = (bf16*)(a.ws + a.TL.P);
     p.Wt = (bf16*)(a.ws + a.TL.Wt); p.Ut = (bf16*)(a.ws + a.TL.Ut);
+    p.Mt = a.save ? (bf16*)(a.ws + a.TL.Mt) : nullptr;
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_prep, kPrepSmem);
     if (e != cudaSuccess) return e;
@@ -482,8 +508,9 @@ cudaError_t tc_prep(const ChunkArgs& a) {
 cudaError_t tc_chain_fwd(const ChunkArgs& a) {
     const qd_shape& s = a.s;
     const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
-    CUtensorMap mWt, mUt, mQg, mK, mP;
-    if (!make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, BH * N * D, 128, 128) ||
+    CUtensorMap mWt, mUt, mQg, mK, mP, mHs;
+    if (!make_tmap_bf16_2d(&mHs, a.ws + a.TL.hsT, D, BH * N * D, D * 2, 128) ||
+        !make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, BH * N * D, 128, 128) ||
         !make_tmap_bf16_2d(&mUt, a.ws + a.TL.Ut, 64, BH * N * D, 128, 128) ||
         !make_tmap_bf16_2d(&mQg, a.ws + a.TL.Qg, D, BH * s.T, D * 2, 64) ||
         !make_tmap_bf16_2d(&mK, a.k, (uint64_t)s.H * D, (uint64_t)s.B * s.T, (uint64_t)s.H * D * 2, 64) ||
@@ -493,10 +520,12 @@ cudaError_t tc_chain_fwd(const ChunkArgs& a) {
     p.T = s.T; p.H = s.H; p.N = (int)N;
     p.g = (const float*)(a.ws + a.TL.g);
     p.h0 = a.h0; p.o = (bf16*)a.o; p.hT = a.hT;
+    p.save = a.save ? 1 : 0;
+    p.Dt = a.save ? (bf16*)(a.ws + a.TL.Dt) : nullptr;
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_chain_fwd, kChainSmem);
     if (e != cudaSuccess) return e;
-    k_tc_chain_fwd<<<(unsigned)BH, 128, kChainSmem, a.stream>>>(mWt, mUt, mQg, mK, mP, p);
+    k_tc_chain_fwd<<<(unsigned)BH, 128, kChainSmem, a.stream>>>(mWt, mUt, mQg, mK, mP, mHs, p);
     return cudaGetLastError();
 }
 

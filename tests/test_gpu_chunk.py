@@ -159,8 +159,10 @@ def test_cfg3_long_context_full_size():
 @pytest.mark.parametrize("regime", gen.REGIMES)
 def test_tensor_core_forward_regimes(regime):
     # bf16, d = 128, T a multiple of 128: the tcgen05 kernels run the forward
-    cfg = replace(gen.CONFIGS["cfg1"], B=2, H=3, T=384, regime=regime, seed=17)
+    cfg = replace(gen.CONFIGS["cfg2"], B=2, H=3, T=384, regime=regime, seed=17)
     _fwd_check(cfg)
+    _bwd_check(cfg)
+    _bwd_check(cfg, reuse=True)
 
 
 def test_tensor_core_forward_single_pair_no_h0():
