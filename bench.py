@@ -234,20 +234,21 @@ def run_ours(args, cfg):
         for n, t in grads.items():
             out_host[n].copy_(t, non_blocking=True)
 
-    e2e_steps = max(1, min(args.steps, 10))
-    e2e_step()
+    e2e_steps = 0 if args.no_extras else max(1, min(args.steps, 10))
+    if e2e_steps:
+        e2e_step()
     barrier()
     e0.record()
     for _ in range(e2e_steps):
         e2e_step()
     e1.record()
     barrier()
-    ems = e0.elapsed_time(e1)
+    ems = e0.elapsed_time(e1) if e2e_steps else float("nan")
     if dist is not None:
         tms = torch.tensor([ems], device="cuda", dtype=torch.float64)
         dist.all_reduce(tms, op=dist.ReduceOp.MAX)
         ems = float(tms.item())
-    e2e_value = tokens_step / (ems / e2e_steps * 1e-3)
+    e2e_value = tokens_step / (ems / e2e_steps * 1e-3) if e2e_steps else None
 
     # ---- roofline of the dominant kernel and of the whole path -----------------------------------
     pk, pk_kind = peaks()
@@ -273,7 +274,7 @@ def run_ours(args, cfg):
     launches = int(sum(v[1] for v in stages.values()))
 
     # ---- decode step (separate configuration), in place over a long run of steps ------------------
-    decode = bench_decode(args, qd, gen, torch, pk, pk_kind) if rank == 0 else None
+    decode = bench_decode(args, qd, gen, torch, pk, pk_kind) if (rank == 0 and not args.no_extras) else None
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -285,7 +286,7 @@ def run_ours(args, cfg):
                     "steps": e2e_steps},
             "gpu_launches": launches, "roofline": roofline, "roofline_path": path, "decode": decode}
     if rank == 0:
-        if world == 1:
+        if world == 1 and not args.no_extras:
             cores = os.cpu_count() or 1
             nseq = max(1, min(B * H, 4 * cores))
             v, dt, thr = oracle_sample(cfg, nseq)
@@ -341,9 +342,14 @@ def main():
     ap.add_argument("--only", default="all", choices=["all", "decode"],
                     help="'decode': time only the decode step (small runs for profiler captures)")
     ap.add_argument("--decode-steps", type=int, default=200)
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "small"],
+                    help="cfg2: headline (default); cfg3: long context; small: B=2 of cfg2 for profiler captures")
+    ap.add_argument("--no-extras", action="store_true", help="skip the end-to-end, decode and CPU-baseline legs")
     args = ap.parse_args()
     from paper_2606_08804_b200 import inputs as gen
-    cfg = gen.CONFIGS["cfg2"]
+    cfg = gen.CONFIGS["cfg3" if args.workload == "cfg3" else "cfg2"]
+    if args.workload == "small":
+        cfg = replace(cfg, B=2)
     if args.only == "decode":
         import torch
         from paper_2606_08804_b200 import binding as qd
