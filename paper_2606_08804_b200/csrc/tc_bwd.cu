@@ -241,7 +241,6 @@ struct ChunkBwdParams {
     int T, H, N;
     const bf16 *beta, *alpha, *lam;
     const float* g;
-    bf16 *dq, *dk, *dv;
     float *dbeta, *dalpha, *dlam;
     unsigned* status;
 };
@@ -249,30 +248,54 @@ struct ChunkBwdParams {
 // shared-memory map of k_tc_chunk_bwd (bytes from the 1024-aligned base)
 constexpr int oQ = 0, oK = 16384, oV = 32768, odO = 49152, oX = 65536, oMt = 81920, oP = 90112, oDt = 98304,
               odDt = 114688, oH = 131072, odH = 163840, kBwdLoadBytes = 180224;   // all TMA-loaded tiles (X is built)
+// tiles built later reuse regions whose contents are dead by then
 constexpr int odPG = oV, odTb = oV + 8192, odW = odO, oN = oH, odXK = oH + 8192, oPP = oH + 16384,
-              oAA = odH + 1024;
+              oAA = odH + 1024, oStDv = odDt, oStDk = oDt, oStDq = odDt;
 constexpr int kBwdSmem = 196608 + 1024;
 constexpr int LDAA = C + 1;
+constexpr int kBwdThreads = 256;
 
-__global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CUtensorMap mapQ,
-                                                      const __grid_constant__ CUtensorMap mapK,
-                                                      const __grid_constant__ CUtensorMap mapV,
-                                                      const __grid_constant__ CUtensorMap mapdO,
-                                                      const __grid_constant__ CUtensorMap mapMt,
-                                                      const __grid_constant__ CUtensorMap mapP,
-                                                      const __grid_constant__ CUtensorMap mapDt,
-                                                      const __grid_constant__ CUtensorMap mapdDt,
-                                                      const __grid_constant__ CUtensorMap mapHs,
-                                                      const __grid_constant__ CUtensorMap mapdHs, ChunkBwdParams p) {
+// 32 TMEM columns of this thread's lane
+__device__ __forceinline__ void ld32(uint32_t taddr, float* v) {
+    tmem_ld32(taddr, v);
+    tmem_ld_wait();
+}
+// Column sums across the 32 lanes of a warp for 32 columns: on return v[0] is the warp-wide sum of
+// column col32_of_lane(lane).
+__device__ __forceinline__ void col_reduce32(float* v, int lane) {
+    fold<32>(v, lane, 16); fold<16>(v, lane, 8); fold<8>(v, lane, 4); fold<4>(v, lane, 2); fold<2>(v, lane, 1);
+}
+__device__ __forceinline__ int col32_of_lane(int lane) {
+    return ((lane & 16) ? 16 : 0) + ((lane & 8) ? 8 : 0) + ((lane & 4) ? 4 : 0) + ((lane & 2) ? 2 : 0) + ((lane & 1) ? 1 : 0);
+}
+
+// Two warpgroups: warpgroup w (threads 128w..128w+127) owns TMEM columns [32w, 32w+32) of every
+// 64-column accumulator; inside a warpgroup thread l owns TMEM lane l.
+__global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_constant__ CUtensorMap mapQ,
+                                                              const __grid_constant__ CUtensorMap mapK,
+                                                              const __grid_constant__ CUtensorMap mapV,
+                                                              const __grid_constant__ CUtensorMap mapdO,
+                                                              const __grid_constant__ CUtensorMap mapMt,
+                                                              const __grid_constant__ CUtensorMap mapP,
+                                                              const __grid_constant__ CUtensorMap mapDt,
+                                                              const __grid_constant__ CUtensorMap mapdDt,
+                                                              const __grid_constant__ CUtensorMap mapHs,
+                                                              const __grid_constant__ CUtensorMap mapdHs,
+                                                              const __grid_constant__ CUtensorMap mapdQ,
+                                                              const __grid_constant__ CUtensorMap mapdK,
+                                                              const __grid_constant__ CUtensorMap mapdV,
+                                                              ChunkBwdParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ uint64_t bar_load, bar_mma;
     __shared__ uint32_t tmem_slot;
     __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C], segc[C];
-    __shared__ float sred[3][4][C];          // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
-    __shared__ float sdg[C], swp[4];
+    __shared__ float sred[3][4][C];   // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
+    __shared__ float srow[4][2][C];   // per-row partial sums of the two column halves: rPP, d beta, t2, rAA
+    __shared__ float sdg[C], swp[8];
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tid = threadIdx.x, wg = tid >> 7, l = tid & 127, lane = tid & 31, wq = (tid >> 5) & 3;
+    const int c0 = wg * 32;                                       // my columns of a 64-column accumulator
     const int ch_id = blockIdx.x, n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
     const size_t row0 = (size_t)b * p.T + (size_t)n * C;          // token row in the [B*T] view
     const size_t wrow0 = (size_t)bh * p.T + (size_t)n * C;        // token row in the [BH*T] view
@@ -282,14 +305,15 @@ __global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CU
         mbar_init(&bar_mma, 1);
         mbar_init_fence();
     }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
+    if (tid < 32) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tb = tmem_slot;
     const uint32_t T0 = tb, T1 = tb + 64, T2 = tb + 128, T3 = tb + 192, T4 = tb + 256, T5 = tb + 320, T6 = tb + 384,
                    T7 = tb + 448;
-    const uint32_t lane_base = (uint32_t)warp * 32;
+    const uint32_t lane_base = (uint32_t)wq * 32;
+    auto my = [&](uint32_t t) { return tmem_addr(t, lane_base, (uint32_t)c0); };
 
     if (tid == 0) {
         mbar_expect_tx(&bar_load, kBwdLoadBytes);
@@ -315,26 +339,26 @@ __global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CU
         salpha[tid] = p.alpha ? __bfloat162float(p.alpha[cr]) : 1.f;
         const float gv = p.g[wrow0 + tid];
         sg[tid] = gv;
-        sgam[tid] = expf(gv);
+        sgam[tid] = __expf(gv);
     }
     __syncthreads();
-    if (tid < C) segc[tid] = expf(sg[C - 1] - sg[tid]);
+    if (tid < C) segc[tid] = __expf(sg[C - 1] - sg[tid]);
 
     bool fail = !mbar_wait(&bar_load, 0);
     if (__syncthreads_or(fail)) {
         if (tid == 0) *p.status = QD_ERR_TIMEOUT;
         mbar_wait(&bar_load, 0);
         __syncthreads();
-        if (warp == 0) tmem_dealloc(tb, 512);
+        if (tid < 32) tmem_dealloc(tb, 512);
         return;
     }
-    // ---- phase 0: X = K + lambda Q; <dh,h>_F; <dDelta_r, Delta_r> -----------------------------------
+    // ---- phase 0: X = K + lambda Q; partial <dh,h>_F ------------------------------------------------
     {
-        const int r = tid & 63, blk = tid >> 6;
+        const int r = tid & 63, qd4 = tid >> 6;          // four threads per row: block qd4>>1, chunks (qd4&1)*4..+3
         const float lm = slam[r];
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-            const uint32_t off = blk * 8192 + sw128_chunk(r, ch);
+        for (int cc = 0; cc < 4; ++cc) {
+            const uint32_t off = (qd4 >> 1) * 8192 + sw128_chunk(r, (qd4 & 1) * 4 + cc);
             float qv[8], kv[8];
             load8(sm + oQ + off, qv);
             load8(sm + oK + off, kv);
@@ -344,18 +368,14 @@ __global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CU
         }
     }
     float dhh_part = 0.f;
-    {
 #pragma unroll
-        for (int blk = 0; blk < 2; ++blk)
+    for (int ch = 0; ch < 8; ++ch) {
+        const uint32_t off = wg * 16384 + sw128_chunk(l, ch);
+        float a[8], c8[8];
+        load8(sm + oH + off, a);
+        load8(sm + odH + off, c8);
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-                const uint32_t off = blk * 16384 + sw128_chunk(tid, ch);
-                float a[8], c8[8];
-                load8(sm + oH + off, a);
-                load8(sm + odH + off, c8);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) dhh_part = fmaf(a[e], c8[e], dhh_part);
-            }
+        for (int e = 0; e < 8; ++e) dhh_part = fmaf(a[e], c8[e], dhh_part);
     }
     fence_proxy_async();
     tc_fence_before();
@@ -381,67 +401,70 @@ __global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CU
     fail = !mbar_wait(&bar_mma, 0);
     if (__syncthreads_or(fail)) {
         if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        if (warp == 0) tmem_dealloc(tb, 512);
+        if (tid < 32) tmem_dealloc(tb, 512);
         return;
     }
     tc_fence_after();
-    float rPP = 0.f;
     float* sPP = reinterpret_cast<float*>(sm + oPP);
     {
-        // <(K-> dh)_s, Delta_s>: (K-> dh)^T[j][s] = gamma_C/gamma_s (dh^T K^T)[j][s] in fp32, Delta^T[j][s] from its tile;
-        // the sum over j runs across lanes
-        float kd[C];
-        ld64(tmem_addr(T7, lane_base, 0), kd);
+        // <(K-> dh)_s, Delta_s>: (K-> dh)^T[j][s] = gamma_C/gamma_s (dh^T K^T)[j][s] in fp32, Delta^T[j][s] from
+        // its tile; the sum over j runs across lanes
+        float kd[32];
+        ld32(my(T7), kd);
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
+        for (int cc = 0; cc < 4; ++cc) {
             float dl[8];
-            load8(sm + oDt + sw128_chunk(tid, ch), dl);
+            load8(sm + oDt + sw128_chunk(l, wg * 4 + cc), dl);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) kd[ch * 8 + e] *= segc[ch * 8 + e] * dl[e];
+            for (int e = 0; e < 8; ++e) kd[cc * 8 + e] *= segc[c0 + cc * 8 + e] * dl[e];
         }
-        col_reduce64(kd, lane);
-        const int col = col_of_lane(lane);
-        sred[0][warp][col] = kd[0];
-        sred[0][warp][col + 1] = kd[1];
+        col_reduce32(kd, lane);
+        sred[0][wq][c0 + col32_of_lane(lane)] = kd[0];
     }
-    if (tid < C) {
-        // dP row r: causal mask, dP o P (row sums here, column sums later), dP o Gamma as an operand tile
-        const int r = tid;
-        float v[C], pg[C];
-        ld64(tmem_addr(T1, lane_base, 0), v);
+    if (l < C) {
+        // dP row r, my 32 columns: causal mask, dP o P (row and column sums), dP o Gamma as an operand tile
+        const int r = l;
+        float v[32];
+        ld32(my(T1), v);
         const float gr = sg[r];
+        float rPP = 0.f;
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-            float pv[8];
-            load8(sm + oP + sw128_chunk(r, ch), pv);
+        for (int cc = 0; cc < 4; ++cc) {
+            float pv[8], pg[8];
+            load8(sm + oP + sw128_chunk(r, wg * 4 + cc), pv);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const int s = ch * 8 + e;
-                const float dp = (s <= r) ? v[s] : 0.f;
+                const int s = c0 + cc * 8 + e;
+                const float dp = (s <= r) ? v[cc * 8 + e] : 0.f;
                 const float pp = dp * pv[e];
                 rPP += pp;
                 sPP[r * LDAA + s] = pp;
-                pg[s] = (s <= r) ? dp * expf(gr - sg[s]) : 0.f;
+                pg[e] = (s <= r) ? dp * __expf(gr - sg[s]) : 0.f;
             }
+            *reinterpret_cast<uint4*>(sm + odPG + sw128_chunk(r, wg * 4 + cc)) = pack8(pg);
         }
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + odPG + sw128_chunk(r, ch)) = pack8(pg + ch * 8);
+        srow[0][wg][r] = rPP;
     }
     {
-        float v[C];
-        ld64(tmem_addr(T3, lane_base, 0), v);                      // dW<-^T row i = tid
+        float v[32];
+        ld32(my(T3), v);                                            // dW<-^T row i = l, my 32 tokens
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + odW + sw128_chunk(tid, ch)) = pack8(v + ch * 8);
-        ld64(tmem_addr(T6, lane_base, 0), v);                      // dV^T row j = tid, to be scaled by beta_s
-        bf16* dst = p.dv + (row0 * p.H + hh) * D + tid;
+        for (int cc = 0; cc < 4; ++cc)
+            *reinterpret_cast<uint4*>(sm + odW + sw128_chunk(l, wg * 4 + cc)) = pack8(v + cc * 8);
+        ld32(my(T6), v);                                            // dV^T row j = l, scaled by beta_s -> staging tile
+        unsigned char* stg = sm + oStDv + (l >> 6) * 8192;
 #pragma unroll
-        for (int s = 0; s < C; ++s) dst[(size_t)s * p.H * D] = __float2bfloat16_rn(sbeta[s] * v[s]);
+        for (int i = 0; i < 32; ++i)
+            *reinterpret_cast<bf16*>(stg + sw128_off(c0 + i, l & 63)) = __float2bfloat16_rn(sbeta[c0 + i] * v[i]);
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
     // ---- phase 2 ---------------------------------------------------------------------------------
     if (tid == 0) {
+        tma_store_2d(&mapdV, sm + oStDv, hh * D, (int)row0);
+        tma_store_2d(&mapdV, sm + oStDv + 8192, hh * D + 64, (int)row0);
+        tma_store_commit();
         tc_fence_after();
         umma_product<false, true>(T7, aX, 8192, adW, 8192, C, D, false);            // X dW<-^T         [s][r]
         umma_product<false, false>(T6, adW, 16384, aMt, 8192, C, C, false);         // dW<-^T M         [i][s]
@@ -449,36 +472,34 @@ __global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CU
     }
     fail = !mbar_wait(&bar_mma, 1);
     if (__syncthreads_or(fail)) {
-        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        if (warp == 0) tmem_dealloc(tb, 512);
+        if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
+        if (tid < 32) tmem_dealloc(tb, 512);
         return;
     }
     tc_fence_after();
-    float dbeta = 0.f, t2 = 0.f;
-    if (tid < C) {
-        // dT^T row s = tid: dT[r][s] for all r;  M[r][s] = line s of Mt
-        const int s = tid;
-        float a[C], bq[C];
-        ld64(tmem_addr(T2, lane_base, 0), a);
-        ld64(tmem_addr(T7, lane_base, 0), bq);
+    if (l < C) {
+        // dT^T row s = l, my 32 values of r;  M[r][s] = line s of Mt
+        const int s = l;
+        float a[32], bq[32];
+        ld32(my(T2), a);
+        ld32(my(T7), bq);
         const float gs = sgam[s], bs = sbeta[s];
-        float mb = 0.f;
+        float mb = 0.f, db = 0.f;
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-            float m[8];
-            load8(sm + oMt + sw128_chunk(s, ch), m);
+        for (int cc = 0; cc < 4; ++cc) {
+            float m[8], tb8[8];
+            load8(sm + oMt + sw128_chunk(s, wg * 4 + cc), m);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const int r = ch * 8 + e;
-                const float dt = fmaf(gs, bq[r], a[r]);
-                dbeta = fmaf(dt, m[e], dbeta);
-                mb = fmaf(m[e], bq[r], mb);
-                a[r] = bs * dt;
+                const float dt = fmaf(gs, bq[cc * 8 + e], a[cc * 8 + e]);
+                db = fmaf(dt, m[e], db);
+                mb = fmaf(m[e], bq[cc * 8 + e], mb);
+                tb8[e] = bs * dt;
             }
+            *reinterpret_cast<uint4*>(sm + odTb + sw128_chunk(s, wg * 4 + cc)) = pack8(tb8);
         }
-        t2 = gs * bs * mb;
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + odTb + sw128_chunk(s, ch)) = pack8(a + ch * 8);
+        srow[1][wg][s] = db;
+        srow[2][wg][s] = gs * bs * mb;
     }
     fence_proxy_async();
     tc_fence_before();
@@ -491,16 +512,17 @@ __global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CU
     }
     fail = !mbar_wait(&bar_mma, 0);
     if (__syncthreads_or(fail)) {
-        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        if (warp == 0) tmem_dealloc(tb, 512);
+        if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
+        if (tid < 32) tmem_dealloc(tb, 512);
         return;
     }
     tc_fence_after();
-    if (tid < C) {
-        float v[C];
-        ld64(tmem_addr(T1, lane_base, 0), v);
+    if (l < C) {
+        float v[32];
+        ld32(my(T1), v);
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + oN + sw128_chunk(tid, ch)) = pack8(v + ch * 8);
+        for (int cc = 0; cc < 4; ++cc)
+            *reinterpret_cast<uint4*>(sm + oN + sw128_chunk(l, wg * 4 + cc)) = pack8(v + cc * 8);
     }
     fence_proxy_async();
     tc_fence_before();
@@ -513,33 +535,37 @@ __global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CU
     }
     fail = !mbar_wait(&bar_mma, 1);
     if (__syncthreads_or(fail)) {
-        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        if (warp == 0) tmem_dealloc(tb, 512);
+        if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
+        if (tid < 32) tmem_dealloc(tb, 512);
         return;
     }
     tc_fence_after();
-    float rAA = 0.f;
     float* sAA = reinterpret_cast<float*>(sm + oAA);
-    if (tid < C) {
-        const int r = tid;
-        float da[C], xk[C];
-        ld64(tmem_addr(T2, lane_base, 0), da);
-        ld64(tmem_addr(T0, lane_base, 0), xk);
+    if (l < C) {
+        const int r = l;
+        float da[32], xk[32];
+        ld32(my(T2), da);
+        ld32(my(T0), xk);
         const float gr = sg[r], br = sbeta[r];
+        float rAA = 0.f, db = 0.f;
 #pragma unroll
-        for (int s = 0; s < C; ++s) {
+        for (int i = 0; i < 32; ++i) {
+            const int s = c0 + i;
             const bool on = s < r;
-            const float gm = on ? expf(gr - sg[s]) : 0.f;
-            const float d = on ? da[s] : 0.f;
-            const float dgx = d * gm * xk[s];
-            dbeta += dgx;
+            const float gm = on ? __expf(gr - sg[s]) : 0.f;
+            const float d = on ? da[i] : 0.f;
+            const float dgx = d * gm * xk[i];
+            db += dgx;
             const float aa = br * dgx;
             rAA += aa;
             sAA[r * LDAA + s] = aa;
-            da[s] = d * br * gm;                                   // dXK
+            da[i] = d * br * gm;                                   // dXK
         }
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) *reinterpret_cast<uint4*>(sm + odXK + sw128_chunk(r, ch)) = pack8(da + ch * 8);
+        for (int cc = 0; cc < 4; ++cc)
+            *reinterpret_cast<uint4*>(sm + odXK + sw128_chunk(r, wg * 4 + cc)) = pack8(da + cc * 8);
+        srow[1][wg][r] += db;
+        srow[3][wg][r] = rAA;
     }
     fence_proxy_async();
     tc_fence_before();
@@ -552,58 +578,67 @@ __global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CU
         umma_product<true, true>(T1, aQ, 8192, adPG, 8192, C, C, true);             // + (dPG^T Q)^T
         umma_product<true, false>(T2, aK, 8192, adPG, 8192, C, C, false);           // (dPG K)^T        [i][r]
         umma_commit(&bar_mma);
+        tma_store_wait_read();                                      // the dv staging tile may be reused now
     }
     fail = !mbar_wait(&bar_mma, 0);
     if (__syncthreads_or(fail)) {
-        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        if (warp == 0) tmem_dealloc(tb, 512);
+        if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
+        if (tid < 32) tmem_dealloc(tb, 512);
         return;
     }
     tc_fence_after();
     {
-        const int i = tid;                                          // d_k index
-        float dx[C], v[C], w[C];
-        ld64(tmem_addr(T6, lane_base, 0), dx);
-        ld64(tmem_addr(T7, lane_base, 0), v);
+        const int i = l;                                            // d_k index; my 32 tokens c0..c0+31
+        float dx[32], v[32], w[32];
+        ld32(my(T6), dx);
+        ld32(my(T7), v);
 #pragma unroll
-        for (int s = 0; s < C; ++s) dx[s] = fmaf(sgam[s] * sbeta[s], dx[s], v[s]);       // dX^T[i][s]
-        // dk
-        ld64(tmem_addr(T1, lane_base, 0), v);
-        ld64(tmem_addr(T5, lane_base, 0), w);
+        for (int s = 0; s < 32; ++s) dx[s] = fmaf(sgam[c0 + s] * sbeta[c0 + s], dx[s], v[s]);       // dX^T[i][s]
+        ld32(my(T1), v);
+        ld32(my(T5), w);
         {
-            bf16* dst = p.dk + (row0 * p.H + hh) * D + i;
+            unsigned char* stg = sm + oStDk + (i >> 6) * 8192;
 #pragma unroll
-            for (int s = 0; s < C; ++s)
-                dst[(size_t)s * p.H * D] = __float2bfloat16_rn(v[s] + segc[s] * w[s] + dx[s]);
+            for (int s = 0; s < 32; ++s)
+                *reinterpret_cast<bf16*>(stg + sw128_off(c0 + s, i & 63)) =
+                    __float2bfloat16_rn(v[s] + segc[c0 + s] * w[s] + dx[s]);
         }
-        // dq, and the two row dot-products with Q that run across lanes
-        ld64(tmem_addr(T4, lane_base, 0), v);
-        ld64(tmem_addr(T2, lane_base, 0), w);
+        ld32(my(T4), v);
+        ld32(my(T2), w);
         {
-            bf16* dst = p.dq + (row0 * p.H + hh) * D + i;
+            unsigned char* stg = sm + oStDq + (i >> 6) * 8192;
             const unsigned char* qcol = sm + oQ + (i >> 6) * 8192;
 #pragma unroll
-            for (int r = 0; r < C; ++r) {
-                const float q1 = sgam[r] * v[r];
-                dst[(size_t)r * p.H * D] = __float2bfloat16_rn(q1 + w[r] + slam[r] * dx[r]);
-                const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(r, i & 63)));
+            for (int r = 0; r < 32; ++r) {
+                const float q1 = sgam[c0 + r] * v[r];
+                *reinterpret_cast<bf16*>(stg + sw128_off(c0 + r, i & 63)) =
+                    __float2bfloat16_rn(q1 + w[r] + slam[c0 + r] * dx[r]);
+                const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(c0 + r, i & 63)));
                 v[r] = q1 * qv;
                 dx[r] = dx[r] * qv;
             }
         }
-        col_reduce64(dx, lane);
-        col_reduce64(v, lane);
-        const int col = col_of_lane(lane);
-        sred[1][warp][col] = dx[0]; sred[1][warp][col + 1] = dx[1];
-        sred[2][warp][col] = v[0];  sred[2][warp][col + 1] = v[1];
+        col_reduce32(dx, lane);
+        col_reduce32(v, lane);
+        const int col = c0 + col32_of_lane(lane);
+        sred[1][wq][col] = dx[0];
+        sred[2][wq][col] = v[0];
     }
     dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 16);
     dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 8);
     dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 4);
     dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 2);
     dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 1);
-    if (lane == 0) swp[warp] = dhh_part;
+    if (lane == 0) swp[tid >> 5] = dhh_part;
+    fence_proxy_async();
     __syncthreads();
+    if (tid == 0) {
+        tma_store_2d(&mapdK, sm + oStDk, hh * D, (int)row0);
+        tma_store_2d(&mapdK, sm + oStDk + 8192, hh * D + 64, (int)row0);
+        tma_store_2d(&mapdQ, sm + oStDq, hh * D, (int)row0);
+        tma_store_2d(&mapdQ, sm + oStDq + 8192, hh * D + 64, (int)row0);
+        tma_store_commit();
+    }
     // ---- decay gradient ----------------------------------------------------------------------------
     if (tid < C) {
         const int r = tid;
@@ -612,24 +647,28 @@ __global__ void __launch_bounds__(128) k_tc_chunk_bwd(const __grid_constant__ CU
         for (int w4 = 0; w4 < 4; ++w4) { kd += sred[0][w4][r]; dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
         for (int u = r + 1; u < C; ++u) cAA += sAA[u * LDAA + r];
         for (int u = r; u < C; ++u) cPP += sPP[u * LDAA + r];
+        const float rPP = srow[0][0][r] + srow[0][1][r], t2 = srow[2][0][r] + srow[2][1][r];
+        const float rAA = srow[3][0][r] + srow[3][1][r];
         sdg[r] = t1 + rPP - cPP + t2 + rAA - cAA - kd;
         sred[0][0][r] = kd;                     // summed below into dg of the last token
-        p.dbeta[(row0 + r) * p.H + hh] = dbeta;
+        p.dbeta[(row0 + r) * p.H + hh] = srow[1][0][r] + srow[1][1][r];
         if (p.dlam) p.dlam[(row0 + r) * p.H + hh] = dl;
     }
     __syncthreads();
     if (tid == 0) {
-        float tot = 0.f;
+        float tot = 0.f, dhh = 0.f;
         for (int r = 0; r < C; ++r) tot += sred[0][0][r];
-        sdg[C - 1] += sgam[C - 1] * (swp[0] + swp[1] + swp[2] + swp[3]) + tot;
+        for (int w8 = 0; w8 < 8; ++w8) dhh += swp[w8];
+        sdg[C - 1] += sgam[C - 1] * dhh + tot;
         float acc = 0.f;
         for (int r = C - 1; r >= 0; --r) { acc += sdg[r]; sdg[r] = acc; }
     }
     __syncthreads();
     if (tid < C && p.dalpha) p.dalpha[(row0 + tid) * p.H + hh] = sdg[tid] / salpha[tid];
+    if (tid == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tb, 512);
+    if (tid < 32) tmem_dealloc(tb, 512);
 }
 
 template <class K>
@@ -667,8 +706,11 @@ cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
     const qd_shape& s = a.s;
     const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
     const uint64_t icols = (uint64_t)s.H * D, irows = (uint64_t)s.B * s.T;
-    CUtensorMap mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs;
-    if (!make_tmap_bf16_2d(&mQ, a.q, icols, irows, icols * 2, 64) ||
+    CUtensorMap mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs, mdQ, mdK, mdV;
+    if (!make_tmap_bf16_2d(&mdQ, a.dq, icols, irows, icols * 2, 64) ||
+        !make_tmap_bf16_2d(&mdK, a.dk, icols, irows, icols * 2, 64) ||
+        !make_tmap_bf16_2d(&mdV, a.dv, icols, irows, icols * 2, 64) ||
+        !make_tmap_bf16_2d(&mQ, a.q, icols, irows, icols * 2, 64) ||
         !make_tmap_bf16_2d(&mK, a.k, icols, irows, icols * 2, 64) ||
         !make_tmap_bf16_2d(&mV, a.v, icols, irows, icols * 2, 64) ||
         !make_tmap_bf16_2d(&mdO, a.dO, icols, irows, icols * 2, 64) ||
@@ -683,12 +725,12 @@ cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
     p.T = s.T; p.H = s.H; p.N = (int)N;
     p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
     p.g = (const float*)(a.ws + a.TL.g);
-    p.dq = (bf16*)a.dq; p.dk = (bf16*)a.dk; p.dv = (bf16*)a.dv;
     p.dbeta = a.dbeta; p.dalpha = a.dalpha; p.dlam = a.dlam;
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_chunk_bwd, kBwdSmem);
     if (e != cudaSuccess) return e;
-    k_tc_chunk_bwd<<<(unsigned)(BH * N), 128, kBwdSmem, a.stream>>>(mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs, p);
+    k_tc_chunk_bwd<<<(unsigned)(BH * N), kBwdThreads, kBwdSmem, a.stream>>>(mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs,
+                                                                               mdQ, mdK, mdV, p);
     return cudaGetLastError();
 }
 
