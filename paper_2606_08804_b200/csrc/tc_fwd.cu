@@ -47,17 +47,22 @@ struct PrepParams {
     unsigned* status;
 };
 
-constexpr int kPrepSmem = 4 * 32768 + 2 * C * LDA * 4 + 1024;
+// 96 KB: Q (later X, in place) | K (later A in fp32, then the T tiles) | V.  Two CTAs fit on one SM.
+constexpr int kPrepSmem = 3 * 32768 + 1024;
 
-__global__ void __launch_bounds__(128) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
-                                                 const __grid_constant__ CUtensorMap mapK,
-                                                 const __grid_constant__ CUtensorMap mapV, PrepParams p) {
+// A (fp32, 64 x 64 per chunk) is kept unpadded; 16-byte groups of a row are XOR-swizzled with the
+// row index so that row-wise 16-byte stores by 32 different rows do not collide on banks.
+__device__ __forceinline__ int a_off(int r, int q4) { return r * C + ((q4 ^ (r & 15)) << 2); }
+
+__global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
+                                                    const __grid_constant__ CUtensorMap mapK,
+                                                    const __grid_constant__ CUtensorMap mapV, PrepParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    unsigned char *sQ = smem, *sK = smem + 32768, *sV = smem + 65536, *sX = smem + 98304;
-    float* sA = reinterpret_cast<float*>(smem);                 // [2][64][65], aliases sQ/sK once the Grams are read
-    float* sM = reinterpret_cast<float*>(smem + 131072);        // [2][64][65]
-    unsigned char* sT = smem;                                   // [2] T_c, [2] T_c diag(gamma): 8 KB each, alias sA
+    unsigned char *sQ = smem, *sK = smem + 32768, *sV = smem + 65536;
+    unsigned char* sX = sQ;                                     // X overwrites Q once Q K^T has been formed
+    float* sA = reinterpret_cast<float*>(sK);                   // [2][64][64], aliases K once both Grams are read
+    unsigned char* sT = sK;                                     // [2] T_c, [2] T_c diag(gamma): 8 KB each, alias A
     __shared__ uint64_t bar_load, bar_mma;
     __shared__ uint32_t tmem_slot;
     __shared__ float sg[128], swsum[4];
@@ -105,45 +110,65 @@ __global__ void __launch_bounds__(128) k_tc_prep(const __grid_constant__ CUtenso
     if (warp & 1) g += swsum[warp - 1];
     sg[tid] = g;
     p.g[wtok] = g;
-    const float gam = expf(g);
+    const float gam = __expf(g);
 
     bool fail = !mbar_wait(&bar_load, 0);
     if (__syncthreads_or(fail)) {
         if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        // loads may still be in flight: give them one more bounded chance before leaving
-        mbar_wait(&bar_load, 0);
+        mbar_wait(&bar_load, 0);           // loads may still be in flight: one more bounded chance
         __syncthreads();
         if (warp == 0) tmem_dealloc(tbase, 256);
         return;
     }
-    // X = K + lambda Q (row `tid`, in the K-major swizzled layout); Qg = gamma Q to the workspace
+    if (tid == 0) {
+        tc_fence_after();
+        // G2 = Q K^T -> columns [128,256)
+        umma_product<false, false>(tbase + 128, smem_u32(sQ), 16384, smem_u32(sK), 16384, 128, 128, false);
+        umma_commit(&bar_mma);
+    }
+    // meanwhile: Qg = gamma Q to the workspace (row `tid`)
     {
         bf16* qg = p.Qg + wtok * D;
 #pragma unroll
         for (int blk = 0; blk < 2; ++blk)
 #pragma unroll
             for (int ch = 0; ch < 8; ++ch) {
-                const uint32_t off = blk * 16384 + sw128_chunk(tid, ch);
-                float qv[8], kv[8], xv[8], gv[8];
-                load8(sQ + off, qv);
-                load8(sK + off, kv);
+                float qv[8];
+                load8(sQ + blk * 16384 + sw128_chunk(tid, ch), qv);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) { xv[e] = fmaf(lam, qv[e], kv[e]); gv[e] = gam * qv[e]; }
-                *reinterpret_cast<uint4*>(sX + off) = pack8(xv);
-                *reinterpret_cast<uint4*>(qg + blk * 64 + ch * 8) = pack8(gv);
+                for (int e = 0; e < 8; ++e) qv[e] *= gam;
+                *reinterpret_cast<uint4*>(qg + blk * 64 + ch * 8) = pack8(qv);
             }
     }
+    fail = !mbar_wait(&bar_mma, 0);
+    if (__syncthreads_or(fail)) {
+        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+        if (warp == 0) tmem_dealloc(tbase, 256);
+        return;
+    }
+    // X = K + lambda Q, in place over Q (row `tid`, K-major swizzled layout)
+#pragma unroll
+    for (int blk = 0; blk < 2; ++blk)
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+            const uint32_t off = blk * 16384 + sw128_chunk(tid, ch);
+            float qv[8], kv[8];
+            load8(sQ + off, qv);
+            load8(sK + off, kv);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) kv[e] = fmaf(lam, qv[e], kv[e]);
+            *reinterpret_cast<uint4*>(sX + off) = pack8(kv);
+        }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
     if (tid == 0) {
         tc_fence_after();
-        // G1 = X K^T -> columns [0,128);  G2 = Q K^T -> columns [128,256)
+        // G1 = X K^T -> columns [0,128)
         umma_product<false, false>(tbase, smem_u32(sX), 16384, smem_u32(sK), 16384, 128, 128, false);
-        umma_product<false, false>(tbase + 128, smem_u32(sQ), 16384, smem_u32(sK), 16384, 128, 128, false);
         umma_commit(&bar_mma);
     }
-    fail = !mbar_wait(&bar_mma, 0);
+    fail = !mbar_wait(&bar_mma, 1);
     if (__syncthreads_or(fail)) {
         if (tid == 0) *p.status = QD_ERR_TIMEOUT;
         if (warp == 0) tmem_dealloc(tbase, 256);
@@ -152,7 +177,7 @@ __global__ void __launch_bounds__(128) k_tc_prep(const __grid_constant__ CUtenso
     tc_fence_after();
     // A = strictLower(beta_r Gamma_ri (x_r . k_i)) -> shared fp32;  P = Gamma_ri (q_r . k_i), i <= r -> workspace
     {
-        float* arow = sA + c * C * LDA + r * LDA;
+        float* Ac = sA + c * C * C;
         bf16* prow = p.P + wtok * C;
         const float* gc = sg + c * C;
 #pragma unroll
@@ -161,51 +186,60 @@ __global__ void __launch_bounds__(128) k_tc_prep(const __grid_constant__ CUtenso
             tmem_ld32(tmem_addr(tbase, warp * 32, c * C + half * 32), v1);
             tmem_ld32(tmem_addr(tbase, warp * 32, 128 + c * C + half * 32), v2);
             tmem_ld_wait();
-            float pv[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const int col = half * 32 + i;
-                const float dec = (col <= r) ? expf(g - gc[col]) : 0.f;
-                arow[col] = (col < r) ? beta * dec * v1[i] : 0.f;
-                pv[i] = dec * v2[i];
+                const float dec = (col <= r) ? __expf(g - gc[col]) : 0.f;
+                v1[i] = (col < r) ? beta * dec * v1[i] : 0.f;
+                v2[i] = dec * v2[i];
             }
 #pragma unroll
-            for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(prow + half * 32 + i * 8) = pack8(pv + i * 8);
+            for (int q4 = 0; q4 < 8; ++q4)
+                *reinterpret_cast<float4*>(Ac + a_off(r, half * 8 + q4)) =
+                    make_float4(v1[q4 * 4], v1[q4 * 4 + 1], v1[q4 * 4 + 2], v1[q4 * 4 + 3]);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(prow + half * 32 + i * 8) = pack8(v2 + i * 8);
         }
     }
     tc_fence_before();
     __syncthreads();
-    // M_c = (I + A_c)^-1: thread (c, j) solves column j by forward substitution
+    // M_c = (I + A_c)^-1: thread (c, j) solves column j by forward substitution, column in registers.
+    // Rows above j come out as exact zeros, row j as one.
+    float m[C];
     {
-        const float* A = sA + c * C * LDA;
-        float* M = sM + c * C * LDA;
+        const float* Ac = sA + c * C * C;
         const int j = r;
-        for (int rr = 0; rr < j; ++rr) M[rr * LDA + j] = 0.f;
-        M[j * LDA + j] = 1.f;
-        for (int rr = j + 1; rr < C; ++rr) {
-            float acc = 0.f;
-            for (int i = j; i < rr; ++i) acc = fmaf(A[rr * LDA + i], M[i * LDA + j], acc);
-            M[rr * LDA + j] = -acc;
+#pragma unroll
+        for (int rr = 0; rr < C; ++rr) m[rr] = 0.f;
+#pragma unroll
+        for (int rr = 0; rr < C; ++rr) {
+            float a0 = (rr == j) ? 1.f : 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+            for (int q4 = 0; q4 < (rr + 3) / 4; ++q4) {
+                const float4 av = *reinterpret_cast<const float4*>(Ac + a_off(rr, q4));
+                a0 = fmaf(-av.x, m[q4 * 4], a0);
+                a1 = fmaf(-av.y, m[q4 * 4 + 1], a1);
+                a2 = fmaf(-av.z, m[q4 * 4 + 2], a2);
+                a3 = fmaf(-av.w, m[q4 * 4 + 3], a3);
+            }
+            m[rr] = (a0 + a1) + (a2 + a3);
         }
     }
     __syncthreads();
     // T_c = M_c diag(beta), T_c diag(gamma): thread (c, i) owns column i and writes line i (MN-major tile)
     {
-        const float* M = sM + c * C * LDA;
         unsigned char* t0 = sT + c * 8192;
         unsigned char* t1 = sT + 16384 + c * 8192;
         bf16* mt = p.Mt ? p.Mt + (((size_t)bh * p.N + 2 * pr + c) * C + r) * C : nullptr;
+        const float bg = beta * gam;
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) {
-            float m0[8], a[8], bq[8];
+            float a[8], bq[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                m0[e] = M[(ch * 8 + e) * LDA + r];
-                a[e] = m0[e] * beta; bq[e] = a[e] * gam;
-            }
+            for (int e = 0; e < 8; ++e) { a[e] = m[ch * 8 + e] * beta; bq[e] = m[ch * 8 + e] * bg; }
             *reinterpret_cast<uint4*>(t0 + sw128_chunk(r, ch)) = pack8(a);
             *reinterpret_cast<uint4*>(t1 + sw128_chunk(r, ch)) = pack8(bq);
-            if (mt) *reinterpret_cast<uint4*>(mt + ch * 8) = pack8(m0);
+            if (mt) *reinterpret_cast<uint4*>(mt + ch * 8) = pack8(m + ch * 8);
         }
     }
     fence_proxy_async();
@@ -222,7 +256,7 @@ __global__ void __launch_bounds__(128) k_tc_prep(const __grid_constant__ CUtenso
         }
         umma_commit(&bar_mma);
     }
-    fail = !mbar_wait(&bar_mma, 1);
+    fail = !mbar_wait(&bar_mma, 0);
     if (__syncthreads_or(fail)) {
         if (tid == 0) *p.status = QD_ERR_TIMEOUT;
         if (warp == 0) tmem_dealloc(tbase, 256);
