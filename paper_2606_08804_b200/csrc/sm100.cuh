@@ -106,6 +106,13 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
+    uint32_t* r = reinterpret_cast<uint32_t*>(v);
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                 : "r"(taddr)
+                 : "memory");
+}
 // address of (lane, column) relative to an allocation base
 __device__ __forceinline__ uint32_t tmem_addr(uint32_t base, uint32_t lane, uint32_t col) {
     return base + (lane << 16) + col;
@@ -174,6 +181,21 @@ __device__ __forceinline__ uint32_t sw128_off(uint32_t line, uint32_t e) {
 }
 // Byte offset of 16-byte chunk c (0..7) of a line.
 __device__ __forceinline__ uint32_t sw128_chunk(uint32_t line, uint32_t c) { return line * 128u + (((c ^ line) & 7u) << 4); }
+
+// Shared-memory stores issued as volatile asm WITHOUT a memory clobber: the compiler keeps their
+// order among themselves and relative to barriers, but is free to hoist ordinary shared-memory
+// loads above them (it cannot otherwise prove that a tile store does not alias a coefficient
+// array, and serialises every load behind the preceding store).  Only use for data that the
+// storing thread does not read back before the next barrier.
+__device__ __forceinline__ void sts128(void* p, uint4 v) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_u32(p)), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w));
+}
+__device__ __forceinline__ void sts16(void* p, __nv_bfloat16 v) {
+    asm volatile("st.shared.b16 [%0], %1;" ::"r"(smem_u32(p)), "h"(*reinterpret_cast<unsigned short*>(&v)));
+}
+__device__ __forceinline__ void sts32(void* p, float v) {
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(smem_u32(p)), "f"(v));
+}
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);

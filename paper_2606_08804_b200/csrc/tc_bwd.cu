@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(128) k_tc_chain_bwd(const __grid_constant__ CU
     for (int blk = 0; blk < 2; ++blk)
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch)
-            *reinterpret_cast<uint4*>(sdH + blk * 16384 + sw128_chunk(tid, ch)) = pack8(dh + blk * 64 + ch * 8);
+            sts128(sdH + blk * 16384 + sw128_chunk(tid, ch), pack8(dh + blk * 64 + ch * 8));
     if (tid < C) sg[0][tid] = p.g[(size_t)bh * p.T + (size_t)(p.N - 1) * C + tid];
     fence_proxy_async();
     tc_fence_before();
@@ -181,7 +181,7 @@ __global__ void __launch_bounds__(128) k_tc_chain_bwd(const __grid_constant__ CU
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
                     const uint4 pk = pack8(a1 + ch * 8);
-                    *reinterpret_cast<uint4*>(sdD + sw128_chunk(tid, half * 4 + ch)) = pk;
+                    sts128(sdD + sw128_chunk(tid, half * 4 + ch), pk);
                     *reinterpret_cast<uint4*>(drow + half * 32 + ch * 8) = pk;
                 }
             }
@@ -211,8 +211,7 @@ __global__ void __launch_bounds__(128) k_tc_chain_bwd(const __grid_constant__ CU
                 for (int i = 0; i < 32; ++i) dh[q4 * 32 + i] = fmaf(gamC, dh[q4 * 32 + i], v[i]);
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch)
-                    *reinterpret_cast<uint4*>(sdH + (q4 >> 1) * 16384 + sw128_chunk(tid, (q4 & 1) * 4 + ch)) =
-                        pack8(dh + q4 * 32 + ch * 8);
+                    sts128(sdH + (q4 >> 1) * 16384 + sw128_chunk(tid, (q4 & 1) * 4 + ch), pack8(dh + q4 * 32 + ch * 8));
             }
         }
         if (tid < C && n >= 1) sg[(it + 1) & 1][tid] = p.g[(size_t)bh * p.T + (size_t)(n - 1) * C + tid];
@@ -237,6 +236,7 @@ __global__ void __launch_bounds__(128) k_tc_chain_bwd(const __grid_constant__ CU
 }
 
 // =================================================================================================
+// =================================================================================================
 struct ChunkBwdParams {
     int T, H, N;
     const bf16 *beta, *alpha, *lam;
@@ -253,7 +253,17 @@ constexpr int odPG = oV, odTb = oV + 8192, odW = odO, oN = oH, odXK = oH + 8192,
               oAA = odH + 1024, oStDv = odDt, oStDk = oDt, oStDq = odDt;
 constexpr int kBwdSmem = 196608 + 1024;
 constexpr int LDAA = C + 1;
-constexpr int kBwdThreads = 256;
+constexpr int kNWG = 4;                       // warpgroups; each owns 64/kNWG columns of every 64-column accumulator
+constexpr int kCW = C / kNWG, kG8 = kCW / 8;    // columns per warpgroup, groups of 8 columns
+constexpr int kBwdThreads = 128 * kNWG;
+
+// Optional phase timestamps (build with -DQD_PHASE_CLOCKS -DQD_CLK_CTA=<block>): thread 0 of that CTA
+// writes clock64() values into bytes 64.. of the workspace status section.
+#ifdef QD_PHASE_CLOCKS
+#define QD_CLK(i) do { if (blockIdx.x == QD_CLK_CTA && threadIdx.x == 0) ((long long*)((char*)p.status + 64))[i] = clock64(); } while (0)
+#else
+#define QD_CLK(i) do { } while (0)
+#endif
 
 // 32 TMEM columns of this thread's lane
 __device__ __forceinline__ void ld32(uint32_t taddr, float* v) {
@@ -268,6 +278,18 @@ __device__ __forceinline__ void col_reduce32(float* v, int lane) {
 __device__ __forceinline__ int col32_of_lane(int lane) {
     return ((lane & 16) ? 16 : 0) + ((lane & 8) ? 8 : 0) + ((lane & 4) ? 4 : 0) + ((lane & 2) ? 2 : 0) + ((lane & 1) ? 1 : 0);
 }
+// Column sums across the 32 lanes of a warp for 8 columns: returns, in every lane, the warp-wide sum of
+// column col8_of_lane(lane) (four lanes hold each column).
+__device__ __forceinline__ float col_reduce8(float* v, int lane) {
+    fold<8>(v, lane, 16); fold<4>(v, lane, 8); fold<2>(v, lane, 4);
+    float x = v[0];
+    x += __shfl_xor_sync(0xffffffffu, x, 2);
+    x += __shfl_xor_sync(0xffffffffu, x, 1);
+    return x;
+}
+__device__ __forceinline__ int col8_of_lane(int lane) { return ((lane & 16) ? 4 : 0) + ((lane & 8) ? 2 : 0) + ((lane & 4) ? 1 : 0); }
+// 8 TMEM columns of this thread's lane (no wait)
+__device__ __forceinline__ void ld8(uint32_t taddr, float* v) { tmem_ld8(taddr, v); }
 
 // Two warpgroups: warpgroup w (threads 128w..128w+127) owns TMEM columns [32w, 32w+32) of every
 // 64-column accumulator; inside a warpgroup thread l owns TMEM lane l.
@@ -291,11 +313,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     __shared__ uint32_t tmem_slot;
     __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C], segc[C];
     __shared__ float sred[3][4][C];   // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
-    __shared__ float srow[4][2][C];   // per-row partial sums of the two column halves: rPP, d beta, t2, rAA
-    __shared__ float sdg[C], swp[8];
+    __shared__ float srow[4][kNWG][C];   // per-row partial sums over each warpgroup's columns: rPP, d beta, t2, rAA
+    __shared__ float sdg[C], skd[C], swp[kBwdThreads / 32], scol[2][kBwdThreads / 64][C];
 
     const int tid = threadIdx.x, wg = tid >> 7, l = tid & 127, lane = tid & 31, wq = (tid >> 5) & 3;
-    const int c0 = wg * 32;                                       // my columns of a 64-column accumulator
+    const int c0 = wg * kCW;                                      // my columns of a 64-column accumulator
     const int ch_id = blockIdx.x, n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
     const size_t row0 = (size_t)b * p.T + (size_t)n * C;          // token row in the [B*T] view
     const size_t wrow0 = (size_t)bh * p.T + (size_t)n * C;        // token row in the [BH*T] view
@@ -315,6 +337,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     const uint32_t lane_base = (uint32_t)wq * 32;
     auto my = [&](uint32_t t) { return tmem_addr(t, lane_base, (uint32_t)c0); };
 
+    QD_CLK(0);
     if (tid == 0) {
         mbar_expect_tx(&bar_load, kBwdLoadBytes);
         const int yi = (int)row0, yt = (int)wrow0;
@@ -352,25 +375,29 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         if (tid < 32) tmem_dealloc(tb, 512);
         return;
     }
+    QD_CLK(1);
     // ---- phase 0: X = K + lambda Q; partial <dh,h>_F ------------------------------------------------
     {
-        const int r = tid & 63, qd4 = tid >> 6;          // four threads per row: block qd4>>1, chunks (qd4&1)*4..+3
+        constexpr int kPer = 16 / (kBwdThreads / 64);     // 16-byte chunks of a row per thread
+        const int r = tid & 63, part = tid >> 6;
         const float lm = slam[r];
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-            const uint32_t off = (qd4 >> 1) * 8192 + sw128_chunk(r, (qd4 & 1) * 4 + cc);
+        for (int cc = 0; cc < kPer; ++cc) {
+            const int ci = part * kPer + cc;              // chunk 0..15 of the row: block ci>>3, chunk ci&7
+            const uint32_t off = (ci >> 3) * 8192 + sw128_chunk(r, ci & 7);
             float qv[8], kv[8];
             load8(sm + oQ + off, qv);
             load8(sm + oK + off, kv);
 #pragma unroll
             for (int e = 0; e < 8; ++e) kv[e] = fmaf(lm, qv[e], kv[e]);
-            *reinterpret_cast<uint4*>(sm + oX + off) = pack8(kv);
+            sts128(sm + oX + off, pack8(kv));
         }
     }
     float dhh_part = 0.f;
 #pragma unroll
-    for (int ch = 0; ch < 8; ++ch) {
-        const uint32_t off = wg * 16384 + sw128_chunk(l, ch);
+    for (int cc = 0; cc < 16 / kNWG; ++cc) {
+        const int ci = wg * (16 / kNWG) + cc;                // chunk 0..15 of line l
+        const uint32_t off = (ci >> 3) * 16384 + sw128_chunk(l, ci & 7);
         float a[8], c8[8];
         load8(sm + oH + off, a);
         load8(sm + odH + off, c8);
@@ -380,6 +407,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    QD_CLK(2);
     // ---- phase 1 products ------------------------------------------------------------------------
     const uint32_t aQ = smem_u32(sm + oQ), aK = smem_u32(sm + oK), aV = smem_u32(sm + oV), adO = smem_u32(sm + odO),
                    aX = smem_u32(sm + oX), aMt = smem_u32(sm + oMt), aDt = smem_u32(sm + oDt),
@@ -405,61 +433,59 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         return;
     }
     tc_fence_after();
+    QD_CLK(3);
     float* sPP = reinterpret_cast<float*>(sm + oPP);
     {
-        // <(K-> dh)_s, Delta_s>: (K-> dh)^T[j][s] = gamma_C/gamma_s (dh^T K^T)[j][s] in fp32, Delta^T[j][s] from
-        // its tile; the sum over j runs across lanes
-        float kd[32];
-        ld32(my(T7), kd);
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-            float dl[8];
-            load8(sm + oDt + sw128_chunk(l, wg * 4 + cc), dl);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) kd[cc * 8 + e] *= segc[c0 + cc * 8 + e] * dl[e];
-        }
-        col_reduce32(kd, lane);
-        sred[0][wq][c0 + col32_of_lane(lane)] = kd[0];
-    }
-    if (l < C) {
-        // dP row r, my 32 columns: causal mask, dP o P (row and column sums), dP o Gamma as an operand tile
-        const int r = l;
-        float v[32];
-        ld32(my(T1), v);
-        const float gr = sg[r];
+        // my 32 columns in four groups of 8 (one 16-byte bf16 chunk each)
         float rPP = 0.f;
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-            float pv[8], pg[8];
-            load8(sm + oP + sw128_chunk(r, wg * 4 + cc), pv);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int s = c0 + cc * 8 + e;
-                const float dp = (s <= r) ? v[cc * 8 + e] : 0.f;
-                const float pp = dp * pv[e];
-                rPP += pp;
-                sPP[r * LDAA + s] = pp;
-                pg[e] = (s <= r) ? dp * __expf(gr - sg[s]) : 0.f;
-            }
-            *reinterpret_cast<uint4*>(sm + odPG + sw128_chunk(r, wg * 4 + cc)) = pack8(pg);
-        }
-        srow[0][wg][r] = rPP;
-    }
-    {
-        float v[32];
-        ld32(my(T3), v);                                            // dW<-^T row i = l, my 32 tokens
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc)
-            *reinterpret_cast<uint4*>(sm + odW + sw128_chunk(l, wg * 4 + cc)) = pack8(v + cc * 8);
-        ld32(my(T6), v);                                            // dV^T row j = l, scaled by beta_s -> staging tile
         unsigned char* stg = sm + oStDv + (l >> 6) * 8192;
+#pragma unroll 1
+        for (int g8 = 0; g8 < kG8; ++g8) {
+            const int cb = c0 + g8 * 8, ck = wg * kG8 + g8;
+            float kd[8], dw[8], dvv[8];
+            ld8(my(T7) + g8 * 8, kd);
+            ld8(my(T3) + g8 * 8, dw);
+            ld8(my(T6) + g8 * 8, dvv);
+            tmem_ld_wait();
+            // <(K-> dh)_s, Delta_s>: (K-> dh)^T[j][s] = gamma_C/gamma_s (dh^T K^T)[j][s] in fp32, times Delta^T[j][s];
+            // the sum over j runs across lanes
+            float dl[8];
+            load8(sm + oDt + sw128_chunk(l, ck), dl);
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-            *reinterpret_cast<bf16*>(stg + sw128_off(c0 + i, l & 63)) = __float2bfloat16_rn(sbeta[c0 + i] * v[i]);
+            for (int e = 0; e < 8; ++e) kd[e] *= segc[cb + e] * dl[e];
+            const float ksum = col_reduce8(kd, lane);
+            if ((lane & 3) == 0) sred[0][wq][cb + col8_of_lane(lane)] = ksum;
+            // dW<-^T row i = l as an operand tile; dV^T row j = l scaled by beta_s into the staging tile
+            sts128(sm + odW + sw128_chunk(l, ck), pack8(dw));
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                sts16(stg + sw128_off(cb + e, l & 63), __float2bfloat16_rn(sbeta[cb + e] * dvv[e]));
+            if (l < C) {
+                // dP row r = l: causal mask, dP o P (row and column sums), dP o Gamma as an operand tile
+                const int r = l;
+                float v[8], pv[8], pg[8];
+                ld8(my(T1) + g8 * 8, v);
+                tmem_ld_wait();
+                load8(sm + oP + sw128_chunk(r, ck), pv);
+                const float gr = sg[r];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int s = cb + e;
+                    const float dp = (s <= r) ? v[e] : 0.f;
+                    const float pp = dp * pv[e];
+                    rPP += pp;
+                    sts32(&sPP[r * LDAA + s], pp);
+                    pg[e] = (s <= r) ? dp * __expf(gr - sg[s]) : 0.f;
+                }
+                sts128(sm + odPG + sw128_chunk(r, ck), pack8(pg));
+            }
+        }
+        if (l < C) srow[0][wg][l] = rPP;
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    QD_CLK(4);
     // ---- phase 2 ---------------------------------------------------------------------------------
     if (tid == 0) {
         tma_store_2d(&mapdV, sm + oStDv, hh * D, (int)row0);
@@ -477,26 +503,28 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         return;
     }
     tc_fence_after();
+    QD_CLK(5);
     if (l < C) {
         // dT^T row s = l, my 32 values of r;  M[r][s] = line s of Mt
         const int s = l;
-        float a[32], bq[32];
-        ld32(my(T2), a);
-        ld32(my(T7), bq);
         const float gs = sgam[s], bs = sbeta[s];
         float mb = 0.f, db = 0.f;
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-            float m[8], tb8[8];
-            load8(sm + oMt + sw128_chunk(s, wg * 4 + cc), m);
+#pragma unroll 1
+        for (int g8 = 0; g8 < kG8; ++g8) {
+            const int ck = wg * kG8 + g8;
+            float a[8], bq[8], m[8], tb8[8];
+            ld8(my(T2) + g8 * 8, a);
+            ld8(my(T7) + g8 * 8, bq);
+            tmem_ld_wait();
+            load8(sm + oMt + sw128_chunk(s, ck), m);
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                const float dt = fmaf(gs, bq[cc * 8 + e], a[cc * 8 + e]);
+                const float dt = fmaf(gs, bq[e], a[e]);
                 db = fmaf(dt, m[e], db);
-                mb = fmaf(m[e], bq[cc * 8 + e], mb);
+                mb = fmaf(m[e], bq[e], mb);
                 tb8[e] = bs * dt;
             }
-            *reinterpret_cast<uint4*>(sm + odTb + sw128_chunk(s, wg * 4 + cc)) = pack8(tb8);
+            sts128(sm + odTb + sw128_chunk(s, ck), pack8(tb8));
         }
         srow[1][wg][s] = db;
         srow[2][wg][s] = gs * bs * mb;
@@ -504,6 +532,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    QD_CLK(6);
     // ---- phase 3: N~ = dT diag(beta) M^T ----------------------------------------------------------
     if (tid == 0) {
         tc_fence_after();
@@ -518,15 +547,18 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     }
     tc_fence_after();
     if (l < C) {
-        float v[32];
-        ld32(my(T1), v);
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc)
-            *reinterpret_cast<uint4*>(sm + oN + sw128_chunk(l, wg * 4 + cc)) = pack8(v + cc * 8);
+#pragma unroll 1
+        for (int g8 = 0; g8 < kG8; ++g8) {
+            float v[8];
+            ld8(my(T1) + g8 * 8, v);
+            tmem_ld_wait();
+            sts128(sm + oN + sw128_chunk(l, wg * kG8 + g8), pack8(v));
+        }
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    QD_CLK(8);
     // ---- phase 4: dA = -M^T N~ ---------------------------------------------------------------------
     if (tid == 0) {
         tc_fence_after();
@@ -540,36 +572,41 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         return;
     }
     tc_fence_after();
+    QD_CLK(9);
     float* sAA = reinterpret_cast<float*>(sm + oAA);
     if (l < C) {
         const int r = l;
-        float da[32], xk[32];
-        ld32(my(T2), da);
-        ld32(my(T0), xk);
         const float gr = sg[r], br = sbeta[r];
         float rAA = 0.f, db = 0.f;
+#pragma unroll 1
+        for (int g8 = 0; g8 < kG8; ++g8) {
+            const int cb = c0 + g8 * 8;
+            float da[8], xk[8];
+            ld8(my(T2) + g8 * 8, da);
+            ld8(my(T0) + g8 * 8, xk);
+            tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            const int s = c0 + i;
-            const bool on = s < r;
-            const float gm = on ? __expf(gr - sg[s]) : 0.f;
-            const float d = on ? da[i] : 0.f;
-            const float dgx = d * gm * xk[i];
-            db += dgx;
-            const float aa = br * dgx;
-            rAA += aa;
-            sAA[r * LDAA + s] = aa;
-            da[i] = d * br * gm;                                   // dXK
+            for (int e = 0; e < 8; ++e) {
+                const int s = cb + e;
+                const bool on = s < r;
+                const float gm = on ? __expf(gr - sg[s]) : 0.f;
+                const float d = on ? da[e] : 0.f;
+                const float dgx = d * gm * xk[e];
+                db += dgx;
+                const float aa = br * dgx;
+                rAA += aa;
+                sts32(&sAA[r * LDAA + s], aa);
+                da[e] = d * br * gm;                               // dXK
+            }
+            sts128(sm + odXK + sw128_chunk(r, wg * kG8 + g8), pack8(da));
         }
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc)
-            *reinterpret_cast<uint4*>(sm + odXK + sw128_chunk(r, wg * 4 + cc)) = pack8(da + cc * 8);
         srow[1][wg][r] += db;
         srow[3][wg][r] = rAA;
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    QD_CLK(10);
     // ---- phase 5 ---------------------------------------------------------------------------------
     if (tid == 0) {
         tc_fence_after();
@@ -587,42 +624,41 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         return;
     }
     tc_fence_after();
+    QD_CLK(11);
     {
-        const int i = l;                                            // d_k index; my 32 tokens c0..c0+31
-        float dx[32], v[32], w[32];
-        ld32(my(T6), dx);
-        ld32(my(T7), v);
+        const int i = l;                                            // d_k index; my 32 tokens c0..c0+31 in groups of 8
+        unsigned char* stk = sm + oStDk + (i >> 6) * 8192;
+        unsigned char* stq = sm + oStDq + (i >> 6) * 8192;
+        const unsigned char* qcol = sm + oQ + (i >> 6) * 8192;
+#pragma unroll 1
+        for (int g8 = 0; g8 < kG8; ++g8) {
+            const int cb = c0 + g8 * 8;
+            float dx[8], v[8], w[8], u[8], z[8], y[8];
+            ld8(my(T6) + g8 * 8, dx);
+            ld8(my(T7) + g8 * 8, v);
+            ld8(my(T1) + g8 * 8, w);
+            ld8(my(T5) + g8 * 8, u);
+            ld8(my(T4) + g8 * 8, z);
+            ld8(my(T2) + g8 * 8, y);
+            tmem_ld_wait();
 #pragma unroll
-        for (int s = 0; s < 32; ++s) dx[s] = fmaf(sgam[c0 + s] * sbeta[c0 + s], dx[s], v[s]);       // dX^T[i][s]
-        ld32(my(T1), v);
-        ld32(my(T5), w);
-        {
-            unsigned char* stg = sm + oStDk + (i >> 6) * 8192;
-#pragma unroll
-            for (int s = 0; s < 32; ++s)
-                *reinterpret_cast<bf16*>(stg + sw128_off(c0 + s, i & 63)) =
-                    __float2bfloat16_rn(v[s] + segc[c0 + s] * w[s] + dx[s]);
-        }
-        ld32(my(T4), v);
-        ld32(my(T2), w);
-        {
-            unsigned char* stg = sm + oStDq + (i >> 6) * 8192;
-            const unsigned char* qcol = sm + oQ + (i >> 6) * 8192;
-#pragma unroll
-            for (int r = 0; r < 32; ++r) {
-                const float q1 = sgam[c0 + r] * v[r];
-                *reinterpret_cast<bf16*>(stg + sw128_off(c0 + r, i & 63)) =
-                    __float2bfloat16_rn(q1 + w[r] + slam[c0 + r] * dx[r]);
-                const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(c0 + r, i & 63)));
-                v[r] = q1 * qv;
-                dx[r] = dx[r] * qv;
+            for (int e = 0; e < 8; ++e) {
+                const int t = cb + e;
+                const float dxe = fmaf(sgam[t] * sbeta[t], dx[e], v[e]);                   // dX^T[i][t]
+                sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(w[e] + segc[t] * u[e] + dxe));
+                const float q1 = sgam[t] * z[e];
+                sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(q1 + y[e] + slam[t] * dxe));
+                const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(t, i & 63)));
+                z[e] = q1 * qv;
+                dx[e] = dxe * qv;
+            }
+            const float dls = col_reduce8(dx, lane), t1s = col_reduce8(z, lane);
+            if ((lane & 3) == 0) {
+                const int col = cb + col8_of_lane(lane);
+                sred[1][wq][col] = dls;
+                sred[2][wq][col] = t1s;
             }
         }
-        col_reduce32(dx, lane);
-        col_reduce32(v, lane);
-        const int col = c0 + col32_of_lane(lane);
-        sred[1][wq][col] = dx[0];
-        sred[2][wq][col] = v[0];
     }
     dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 16);
     dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 8);
@@ -639,33 +675,65 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         tma_store_2d(&mapdQ, sm + oStDq + 8192, hh * D + 64, (int)row0);
         tma_store_commit();
     }
+    QD_CLK(12);
     // ---- decay gradient ----------------------------------------------------------------------------
+    {
+        // column sums of dA o A and dP o P: kBwdThreads/64 threads per column
+        const int r = tid & 63, part = tid >> 6;
+        float cA = 0.f, cP = 0.f;
+#pragma unroll
+        constexpr int kRows = C / (kBwdThreads / 64);
+#pragma unroll
+        for (int k = 0; k < kRows; ++k) {
+            cA += sAA[(part * kRows + k) * LDAA + r];
+            cP += sPP[(part * kRows + k) * LDAA + r];
+        }
+        scol[0][part][r] = cA;
+        scol[1][part][r] = cP;
+    }
+    __syncthreads();
     if (tid < C) {
         const int r = tid;
         float kd = 0.f, dl = 0.f, t1 = 0.f, cAA = 0.f, cPP = 0.f;
 #pragma unroll
         for (int w4 = 0; w4 < 4; ++w4) { kd += sred[0][w4][r]; dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
-        for (int u = r + 1; u < C; ++u) cAA += sAA[u * LDAA + r];
-        for (int u = r; u < C; ++u) cPP += sPP[u * LDAA + r];
-        const float rPP = srow[0][0][r] + srow[0][1][r], t2 = srow[2][0][r] + srow[2][1][r];
-        const float rAA = srow[3][0][r] + srow[3][1][r];
+#pragma unroll
+        for (int w4 = 0; w4 < kBwdThreads / 64; ++w4) { cAA += scol[0][w4][r]; cPP += scol[1][w4][r]; }
+        float rPP = 0.f, t2 = 0.f, rAA = 0.f, dbt = 0.f;
+#pragma unroll
+        for (int w4 = 0; w4 < kNWG; ++w4) { rPP += srow[0][w4][r]; dbt += srow[1][w4][r]; t2 += srow[2][w4][r]; rAA += srow[3][w4][r]; }
         sdg[r] = t1 + rPP - cPP + t2 + rAA - cAA - kd;
-        sred[0][0][r] = kd;                     // summed below into dg of the last token
-        p.dbeta[(row0 + r) * p.H + hh] = srow[1][0][r] + srow[1][1][r];
+        skd[r] = kd;                            // summed below into dg of the last token
+        p.dbeta[(row0 + r) * p.H + hh] = dbt;
         if (p.dlam) p.dlam[(row0 + r) * p.H + hh] = dl;
     }
     __syncthreads();
-    if (tid == 0) {
-        float tot = 0.f, dhh = 0.f;
-        for (int r = 0; r < C; ++r) tot += sred[0][0][r];
-        for (int w8 = 0; w8 < 8; ++w8) dhh += swp[w8];
-        sdg[C - 1] += sgam[C - 1] * dhh + tot;
-        float acc = 0.f;
-        for (int r = C - 1; r >= 0; --r) { acc += sdg[r]; sdg[r] = acc; }
+    if (tid < 32) {
+        // warp 0: lane owns tokens 2*lane, 2*lane+1; d log alpha_i = sum_{r >= i} dg_r (suffix sums)
+        const float a = sdg[2 * lane];
+        float b2 = sdg[2 * lane + 1];
+        float kds = skd[2 * lane] + skd[2 * lane + 1];
+        float dhh = lane < kBwdThreads / 32 ? swp[lane] : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            kds += __shfl_xor_sync(0xffffffffu, kds, o);
+            dhh += __shfl_xor_sync(0xffffffffu, dhh, o);
+        }
+        if (lane == 31) b2 += sgam[C - 1] * dhh + kds;
+        float sfx = a + b2;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float t = __shfl_down_sync(0xffffffffu, sfx, o);
+            if (lane + o < 32) sfx += t;
+        }
+        if (p.dalpha) {
+            p.dalpha[(row0 + 2 * lane) * p.H + hh] = sfx / salpha[2 * lane];
+            p.dalpha[(row0 + 2 * lane + 1) * p.H + hh] = (sfx - a) / salpha[2 * lane + 1];
+        }
     }
-    __syncthreads();
-    if (tid < C && p.dalpha) p.dalpha[(row0 + tid) * p.H + hh] = sdg[tid] / salpha[tid];
+    QD_CLK(13);
     if (tid == 0) tma_store_wait_all();
+    QD_CLK(14);
     tc_fence_before();
     __syncthreads();
     if (tid < 32) tmem_dealloc(tb, 512);

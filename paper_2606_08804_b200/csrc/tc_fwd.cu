@@ -52,7 +52,17 @@ constexpr int kPrepSmem = 3 * 32768 + 1024;
 
 // A (fp32, 64 x 64 per chunk) is kept unpadded; 16-byte groups of a row are XOR-swizzled with the
 // row index so that row-wise 16-byte stores by 32 different rows do not collide on banks.
-__device__ __forceinline__ int a_off(int r, int q4) { return r * C + ((q4 ^ (r & 15)) << 2); }
+// A (fp32, 64 x 64 per chunk) is kept transposed and unpadded: element (column i, row r) of A^T at
+// i*64 + r, with the 16-byte group index of r XOR-ed with (i & 15) so that reading one column as
+// float4 and writing one row element-wise are both free of bank conflicts.
+__device__ __forceinline__ int at_off(int i, int r) { return i * C + ((((r >> 2) ^ i) & 15) << 2) + (r & 3); }
+
+// Optional phase timestamps (build with -DQD_PHASE_CLOCKS): CTA 0, thread 0 -> bytes 64.. of the status section.
+#ifdef QD_PHASE_CLOCKS
+#define QD_PCLK(i) do { if (blockIdx.x == QD_CLK_CTA && threadIdx.x == 0) ((long long*)((char*)p.status + 64))[i] = clock64(); } while (0)
+#else
+#define QD_PCLK(i) do { } while (0)
+#endif
 
 __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
                                                     const __grid_constant__ CUtensorMap mapK,
@@ -85,6 +95,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     tc_fence_after();
     const uint32_t tbase = tmem_slot;
 
+    QD_PCLK(0);
     if (tid == 0) {
         mbar_expect_tx(&bar_load, 3 * 32768);
         const int y = (int)((size_t)b * p.T + (size_t)pr * 128);
@@ -120,6 +131,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         if (warp == 0) tmem_dealloc(tbase, 256);
         return;
     }
+    QD_PCLK(1);
     if (tid == 0) {
         tc_fence_after();
         // G2 = Q K^T -> columns [128,256)
@@ -146,6 +158,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         if (warp == 0) tmem_dealloc(tbase, 256);
         return;
     }
+    QD_PCLK(2);
     // X = K + lambda Q, in place over Q (row `tid`, K-major swizzled layout)
 #pragma unroll
     for (int blk = 0; blk < 2; ++blk)
@@ -157,11 +170,12 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
             load8(sK + off, kv);
 #pragma unroll
             for (int e = 0; e < 8; ++e) kv[e] = fmaf(lam, qv[e], kv[e]);
-            *reinterpret_cast<uint4*>(sX + off) = pack8(kv);
+            sts128(sX + off, pack8(kv));
         }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    QD_PCLK(3);
     if (tid == 0) {
         tc_fence_after();
         // G1 = X K^T -> columns [0,128)
@@ -175,6 +189,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         return;
     }
     tc_fence_after();
+    QD_PCLK(4);
     // A = strictLower(beta_r Gamma_ri (x_r . k_i)) -> shared fp32;  P = Gamma_ri (q_r . k_i), i <= r -> workspace
     {
         float* Ac = sA + c * C * C;
@@ -193,39 +208,50 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
                 v1[i] = (col < r) ? beta * dec * v1[i] : 0.f;
                 v2[i] = dec * v2[i];
             }
+            // A^T: entry (column i, row r) so that a column of A is contiguous over r
 #pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4)
-                *reinterpret_cast<float4*>(Ac + a_off(r, half * 8 + q4)) =
-                    make_float4(v1[q4 * 4], v1[q4 * 4 + 1], v1[q4 * 4 + 2], v1[q4 * 4 + 3]);
+            for (int i = 0; i < 32; ++i) Ac[at_off(half * 32 + i, r)] = v1[i];
 #pragma unroll
             for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(prow + half * 32 + i * 8) = pack8(v2 + i * 8);
         }
     }
     tc_fence_before();
     __syncthreads();
+    QD_PCLK(5);
     // M_c = (I + A_c)^-1: thread (c, j) solves column j by forward substitution, column in registers.
     // Rows above j come out as exact zeros, row j as one.
     float m[C];
     {
+        // right-looking substitution: once m[i] is final, every later row gets its update
+        // m[r] -= A[r][i] m[i]; the updates of one step are independent of each other, and the
+        // loads of A do not depend on the recurrence.
         const float* Ac = sA + c * C * C;
         const int j = r;
+#ifdef QD_REP
+#pragma unroll 1
+        for (int rep = 0; rep < QD_REP; ++rep) {
+#endif
 #pragma unroll
-        for (int rr = 0; rr < C; ++rr) m[rr] = 0.f;
+        for (int rr = 0; rr < C; ++rr) m[rr] = (rr == j) ? 1.f : 0.f;
 #pragma unroll
-        for (int rr = 0; rr < C; ++rr) {
-            float a0 = (rr == j) ? 1.f : 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        for (int i = 0; i < C - 1; ++i) {
+            const float mi = m[i];
 #pragma unroll
-            for (int q4 = 0; q4 < (rr + 3) / 4; ++q4) {
-                const float4 av = *reinterpret_cast<const float4*>(Ac + a_off(rr, q4));
-                a0 = fmaf(-av.x, m[q4 * 4], a0);
-                a1 = fmaf(-av.y, m[q4 * 4 + 1], a1);
-                a2 = fmaf(-av.z, m[q4 * 4 + 2], a2);
-                a3 = fmaf(-av.w, m[q4 * 4 + 3], a3);
+            for (int q4 = (i + 1) / 4; q4 < C / 4; ++q4) {
+                const float4 av = *reinterpret_cast<const float4*>(Ac + i * C + (((q4 ^ i) & 15) << 2));
+                // rows 4*q4 .. 4*q4+3; entries with row <= i are zero (A is strictly lower)
+                m[q4 * 4] = fmaf(-av.x, mi, m[q4 * 4]);
+                m[q4 * 4 + 1] = fmaf(-av.y, mi, m[q4 * 4 + 1]);
+                m[q4 * 4 + 2] = fmaf(-av.z, mi, m[q4 * 4 + 2]);
+                m[q4 * 4 + 3] = fmaf(-av.w, mi, m[q4 * 4 + 3]);
             }
-            m[rr] = (a0 + a1) + (a2 + a3);
         }
+#ifdef QD_REP
+        }
+#endif
     }
     __syncthreads();
+    QD_PCLK(6);
     // T_c = M_c diag(beta), T_c diag(gamma): thread (c, i) owns column i and writes line i (MN-major tile)
     {
         unsigned char* t0 = sT + c * 8192;
@@ -237,14 +263,15 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
             float a[8], bq[8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) { a[e] = m[ch * 8 + e] * beta; bq[e] = m[ch * 8 + e] * bg; }
-            *reinterpret_cast<uint4*>(t0 + sw128_chunk(r, ch)) = pack8(a);
-            *reinterpret_cast<uint4*>(t1 + sw128_chunk(r, ch)) = pack8(bq);
+            sts128(t0 + sw128_chunk(r, ch), pack8(a));
+            sts128(t1 + sw128_chunk(r, ch), pack8(bq));
             if (mt) *reinterpret_cast<uint4*>(mt + ch * 8) = pack8(m + ch * 8);
         }
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
+    QD_PCLK(7);
     if (tid == 0) {
         tc_fence_after();
         for (int cc = 0; cc < 2; ++cc) {
@@ -263,6 +290,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         return;
     }
     tc_fence_after();
+    QD_PCLK(8);
     // rows `tid` (a d_v resp. d_k index) of Ut and Wt, both chunks
 #pragma unroll
     for (int which = 0; which < 2; ++which) {
@@ -278,6 +306,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
             for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(row + i * 8) = pack8(v + i * 8);
         }
     }
+    QD_PCLK(9);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tbase, 256);
@@ -359,7 +388,7 @@ __global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CU
     for (int blk = 0; blk < 2; ++blk)
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch)
-            *reinterpret_cast<uint4*>(sH + blk * 16384 + sw128_chunk(tid, ch)) = pack8(h + blk * 64 + ch * 8);
+            sts128(sH + blk * 16384 + sw128_chunk(tid, ch), pack8(h + blk * 64 + ch * 8));
     if (tid < C) sg[0][tid] = p.g[(size_t)bh * p.T + tid];
     fence_proxy_async();
     tc_fence_before();
@@ -410,8 +439,8 @@ __global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CU
                         d1[e] = d0[e] * expf(gC - gc[half * 32 + ch * 8 + e]);
                     }
                     const uint4 pk = pack8(d0);
-                    *reinterpret_cast<uint4*>(sD + off) = pk;
-                    *reinterpret_cast<uint4*>(sDs + off) = pack8(d1);
+                    sts128(sD + off, pk);
+                    sts128(sDs + off, pack8(d1));
                     if (p.Dt)
                         *reinterpret_cast<uint4*>(p.Dt + (((size_t)bh * p.N + n) * D + tid) * C + half * 32 + ch * 8) = pk;
                 }
@@ -445,8 +474,7 @@ __global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CU
                 for (int i = 0; i < 32; ++i) h[q4 * 32 + i] = fmaf(gamC, h[q4 * 32 + i], v[i]);
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch)
-                    *reinterpret_cast<uint4*>(sH + (q4 >> 1) * 16384 + sw128_chunk(tid, (q4 & 1) * 4 + ch)) =
-                        pack8(h + q4 * 32 + ch * 8);
+                    sts128(sH + (q4 >> 1) * 16384 + sw128_chunk(tid, (q4 & 1) * 4 + ch), pack8(h + q4 * 32 + ch * 8));
             }
         }
         // O^T row j -> o[b, t0 + r, hh, j]
