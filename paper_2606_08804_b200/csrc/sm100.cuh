@@ -64,6 +64,9 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void*
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// wait until at most N of this thread's most recent bulk groups still have to read their source
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read_n() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -165,13 +168,14 @@ template <bool A_MN, bool B_MN>
 __device__ __forceinline__ void umma_product(uint32_t d_tmem, uint32_t a_saddr, uint32_t a_blk, uint32_t b_saddr,
                                              uint32_t b_blk, int N, int K, bool accumulate, bool a_neg = false) {
     const uint32_t idesc = make_idesc(128, N, A_MN, B_MN, a_neg);
+    // base descriptors once; a K step only moves the 14-bit start-address field (units of 16 bytes)
+    const uint64_t a0 = A_MN ? desc_mnmajor(a_saddr, a_blk) : desc_kmajor(a_saddr);
+    const uint64_t b0 = B_MN ? desc_mnmajor(b_saddr, b_blk) : desc_kmajor(b_saddr);
+#pragma unroll
     for (int k = 0; k < K; k += 16) {
-        uint64_t ad, bd;
-        if (A_MN) ad = desc_mnmajor(a_saddr + (uint32_t)k * 128u, a_blk);
-        else ad = desc_kmajor(a_saddr + (uint32_t)(k >> 6) * a_blk + (uint32_t)(k & 63) * 2u);
-        if (B_MN) bd = desc_mnmajor(b_saddr + (uint32_t)k * 128u, b_blk);
-        else bd = desc_kmajor(b_saddr + (uint32_t)(k >> 6) * b_blk + (uint32_t)(k & 63) * 2u);
-        umma_ss(d_tmem, ad, bd, idesc, accumulate || k > 0);
+        const uint32_t ao = A_MN ? (uint32_t)k * 128u : (uint32_t)(k >> 6) * a_blk + (uint32_t)(k & 63) * 2u;
+        const uint32_t bo = B_MN ? (uint32_t)k * 128u : (uint32_t)(k >> 6) * b_blk + (uint32_t)(k & 63) * 2u;
+        umma_ss(d_tmem, a0 + (uint64_t)(ao >> 4), b0 + (uint64_t)(bo >> 4), idesc, accumulate || k > 0);
     }
 }
 

@@ -65,177 +65,203 @@ struct ChainBwdParams {
     const float* g;
     const float* dhT;
     float* dh0;
-    bf16* dDt;
     unsigned* status;
 };
 
 constexpr int kStage = 73728;                           // Wt 16K | dO 16K | Qg 16K | K 16K | P 8K
 constexpr int kChainSmem = 2 * kStage + 32768 + 16384 + 1024;
+constexpr int kChainThreads = 288;                 // 8 compute warps + 1 issue warp
 
-__global__ void __launch_bounds__(128) k_tc_chain_bwd(const __grid_constant__ CUtensorMap mapWt,
-                                                      const __grid_constant__ CUtensorMap mapdO,
-                                                      const __grid_constant__ CUtensorMap mapQg,
-                                                      const __grid_constant__ CUtensorMap mapK,
-                                                      const __grid_constant__ CUtensorMap mapP,
-                                                      const __grid_constant__ CUtensorMap mapdHs, ChainBwdParams p) {
+// named barriers between the 256 compute threads (arrive) and the issue warp (sync)
+constexpr int kBarH = 1, kBarD = 2, kBarCount = kChainThreads;
+__device__ __forceinline__ void nb_arrive(int id) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(kBarCount) : "memory"); }
+__device__ __forceinline__ void nb_sync(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(kBarCount) : "memory"); }
+
+// Reverse state chain.  Per chunk the dependency is
+//   dh ready -> A2 = dh^T K^T -> dDelta^T -> H-accumulator -= dDelta^T W<- -> dh update;
+// A1 = dO^T P and the dO^T Qg part of the H-accumulator do not depend on dh.
+// Compute warpgroup w owns tokens [32w, 32w+32) of the 64-column accumulators and d_k columns
+// [64w, 64w+64) of dh^T; thread l of a warpgroup owns TMEM lane l = d_v index.
+__global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_constant__ CUtensorMap mapWt,
+                                                                const __grid_constant__ CUtensorMap mapdO,
+                                                                const __grid_constant__ CUtensorMap mapQg,
+                                                                const __grid_constant__ CUtensorMap mapK,
+                                                                const __grid_constant__ CUtensorMap mapP,
+                                                                const __grid_constant__ CUtensorMap mapdHs,
+                                                                const __grid_constant__ CUtensorMap mapdDt,
+                                                                ChainBwdParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char* sdH = smem + 2 * kStage;         // dh^T as A operand: K-major, 2 blocks of [128 lines][64]
     unsigned char* sdD = sdH + 32768;               // dDelta^T: K-major [128 lines (dv)][64 tokens]
-    __shared__ uint64_t bar_load[2], bar_a, bar_b;
+    __shared__ uint64_t bar_load[2], bar_a, bar_b, bar_e;
     __shared__ uint32_t tmem_slot;
-    __shared__ float sg[2][C];
+    __shared__ volatile int s_abort;
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, wg = tid >> 7, l = tid & 127, wq = (tid >> 5) & 3;
     const int bh = blockIdx.x, b = bh / p.H, hh = bh % p.H;
+    const bool compute = tid < 256;
 
     if (tid == 0) {
         mbar_init(&bar_load[0], 1); mbar_init(&bar_load[1], 1);
-        mbar_init(&bar_a, 1); mbar_init(&bar_b, 1);
+        mbar_init(&bar_a, 2); mbar_init(&bar_b, 2); mbar_init(&bar_e, 1);
         mbar_init_fence();
+        s_abort = 0;
     }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    if (tid < 32) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tbase = tmem_slot;
     const uint32_t tA1 = tbase, tA2 = tbase + 64, tH = tbase + 128;
+    const uint32_t lane_base = (uint32_t)wq * 32;
 
-    // iteration `it` processes chunk n = N-1-it
-    auto issue_load = [&](int it) {
-        const int n = p.N - 1 - it;
-        unsigned char* st = smem + (it & 1) * kStage;
-        uint64_t* bar = &bar_load[it & 1];
-        mbar_expect_tx(bar, kStage);
-        const int yc = (int)(((size_t)bh * p.N + n) * D);
-        const int yt = (int)((size_t)bh * p.T + (size_t)n * C);
-        const int yi = (int)((size_t)b * p.T + (size_t)n * C);
-        tma_load_2d(st, &mapWt, 0, yc, bar);
-        tma_load_2d(st + 16384, &mapdO, hh * D, yi, bar);
-        tma_load_2d(st + 16384 + 8192, &mapdO, hh * D + 64, yi, bar);
-        tma_load_2d(st + 32768, &mapQg, 0, yt, bar);
-        tma_load_2d(st + 32768 + 8192, &mapQg, 64, yt, bar);
-        tma_load_2d(st + 49152, &mapK, hh * D, yi, bar);
-        tma_load_2d(st + 49152 + 8192, &mapK, hh * D + 64, yi, bar);
-        tma_load_2d(st + 65536, &mapP, 0, yt, bar);
+    // bounded wait; once any wait has expired every later wait returns at once (the kernel drains)
+    auto wait = [&](uint64_t* bar, uint32_t parity) {
+        if (s_abort) return;
+        if (!mbar_wait(bar, parity)) { s_abort = 1; *p.status = QD_ERR_TIMEOUT; }
     };
-    if (tid == 0) { issue_load(0); if (p.N > 1) issue_load(1); }
+    const float* gseq = p.g + (size_t)bh * p.T;
 
-    float dh[D];      // row j of dh^T
-    if (p.dhT) {
-        const float* src = p.dhT + (size_t)bh * D * D + tid;
+    if (compute) {
+        // ---------------------------------- compute warps ----------------------------------
+        float dh[64];     // dh^T[j = l][64 wg .. 64 wg + 63]
+        if (p.dhT) {
+            const float* src = p.dhT + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
 #pragma unroll
-        for (int i = 0; i < D; ++i) dh[i] = src[(size_t)i * D];
-    } else {
+            for (int i = 0; i < 64; ++i) dh[i] = src[(size_t)i * D];
+        } else {
 #pragma unroll
-        for (int i = 0; i < D; ++i) dh[i] = 0.f;
-    }
-#pragma unroll
-    for (int blk = 0; blk < 2; ++blk)
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch)
-            sts128(sdH + blk * 16384 + sw128_chunk(tid, ch), pack8(dh + blk * 64 + ch * 8));
-    if (tid < C) sg[0][tid] = p.g[(size_t)bh * p.T + (size_t)(p.N - 1) * C + tid];
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-
-    bool aborted = false;
-    int loads_waited = 0;
-    for (int it = 0; it < p.N; ++it) {
-        const int n = p.N - 1 - it;
-        unsigned char* st = smem + (it & 1) * kStage;
-        const float* gc = sg[it & 1];
-        bool fail = !mbar_wait(&bar_load[it & 1], (it >> 1) & 1);
-        if (__syncthreads_or(fail)) { aborted = true; break; }
-        loads_waited = it + 1;
-        if (tid == 0) {
-            // gradient w.r.t. the exit state of chunk n, bf16, as the operand tile (rows = d_v, cols = d_k)
-            const int yh = (int)(((size_t)bh * p.N + n) * D);
-            tma_store_2d(&mapdHs, sdH, 0, yh);
-            tma_store_2d(&mapdHs, sdH + 16384, 64, yh);
-            tma_store_commit();
-            tc_fence_after();
-            const uint32_t sdO = smem_u32(st + 16384);
-            // A1 = dO^T P  (A, B MN-major: lines = token r);  A2 = dh^T K^T (A, B K-major)
-            umma_product<true, true>(tA1, sdO, 8192, smem_u32(st + 65536), 8192, C, C, false);
-            umma_product<false, false>(tA2, smem_u32(sdH), 16384, smem_u32(st + 49152), 8192, C, D, false);
-            // H-accumulator = dO^T Qg (B MN-major: lines = token r, two blocks of d_k)
-            umma_product<true, true>(tH, sdO, 8192, smem_u32(st + 32768), 8192, D, C, false);
-            umma_commit(&bar_a);
+            for (int i = 0; i < 64; ++i) dh[i] = 0.f;
         }
-        fail = !mbar_wait(&bar_a, it & 1);
-        if (__syncthreads_or(fail)) { aborted = true; break; }
-        tc_fence_after();
-        {
-            const float gC = gc[C - 1];
-            bf16* drow = p.dDt + (((size_t)bh * p.N + n) * D + tid) * C;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                float a1[32], a2[32];
-                tmem_ld32(tmem_addr(tA1, warp * 32, half * 32), a1);
-                tmem_ld32(tmem_addr(tA2, warp * 32, half * 32), a2);
-                tmem_ld_wait();
+        for (int ch = 0; ch < 8; ++ch) sts128(sdH + wg * 16384 + sw128_chunk(l, ch), pack8(dh + ch * 8));
+        fence_proxy_async();
+        nb_arrive(kBarH);
+
+        for (int it = 0; it < p.N; ++it) {
+            const int n = p.N - 1 - it;
+            const float gC = gseq[(size_t)n * C + C - 1];
+            float sc[32];
+            {
+                const float4* gp = reinterpret_cast<const float4*>(gseq + (size_t)n * C + wg * 32);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) a1[i] = fmaf(expf(gC - gc[half * 32 + i]), a2[i], a1[i]);
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    const uint4 pk = pack8(a1 + ch * 8);
-                    sts128(sdD + sw128_chunk(tid, half * 4 + ch), pk);
-                    *reinterpret_cast<uint4*>(drow + half * 32 + ch * 8) = pk;
+                for (int q = 0; q < 8; ++q) {
+                    const float4 t = gp[q];
+                    sc[q * 4] = t.x; sc[q * 4 + 1] = t.y; sc[q * 4 + 2] = t.z; sc[q * 4 + 3] = t.w;
                 }
             }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
-            tc_fence_after();
-            // H-accumulator -= dDelta^T W<-   (A negated; B K-major: lines = d_k index, contraction over tokens)
-            umma_product<false, false>(tH, smem_u32(sdD), 16384, smem_u32(st), 16384, D, C, true, true);
-            umma_commit(&bar_b);
-        }
-        fail = !mbar_wait(&bar_b, it & 1);
-        if (tid == 0) tma_store_wait_read();
-        if (__syncthreads_or(fail)) { aborted = true; break; }
-        tc_fence_after();
-        if (tid == 0 && it + 2 < p.N) issue_load(it + 2);
-        {
-            const float gamC = expf(gc[C - 1]);
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                float v[32];
-                tmem_ld32(tmem_addr(tH, warp * 32, q4 * 32), v);
+            for (int i = 0; i < 32; ++i) sc[i] = __expf(gC - sc[i]);
+            const float gamC = __expf(gC);
+            wait(&bar_a, it & 1);
+            tc_fence_after();
+            // dDelta^T = A1 + gamma_C/gamma_s A2, my 32 tokens
+            {
+                float a1[32], a2[32];
+                tmem_ld32(tmem_addr(tA1, lane_base, wg * 32), a1);
+                tmem_ld32(tmem_addr(tA2, lane_base, wg * 32), a2);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) dh[q4 * 32 + i] = fmaf(gamC, dh[q4 * 32 + i], v[i]);
+                for (int i = 0; i < 32; ++i) a1[i] = fmaf(sc[i], a2[i], a1[i]);
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch)
-                    sts128(sdH + (q4 >> 1) * 16384 + sw128_chunk(tid, (q4 & 1) * 4 + ch), pack8(dh + q4 * 32 + ch * 8));
+                for (int cc = 0; cc < 4; ++cc) sts128(sdD + sw128_chunk(l, wg * 4 + cc), pack8(a1 + cc * 8));
+            }
+            tc_fence_before();
+            fence_proxy_async();
+            nb_arrive(kBarD);
+            wait(&bar_b, it & 1);
+            tc_fence_after();
+#pragma unroll
+            for (int q2 = 0; q2 < 2; ++q2) {
+                float v[32];
+                tmem_ld32(tmem_addr(tH, lane_base, wg * 64 + q2 * 32), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) dh[q2 * 32 + i] = fmaf(gamC, dh[q2 * 32 + i], v[i]);
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+                    sts128(sdH + wg * 16384 + sw128_chunk(l, q2 * 4 + cc), pack8(dh + q2 * 32 + cc * 8));
+            }
+            tc_fence_before();
+            fence_proxy_async();
+            nb_arrive(kBarH);
+        }
+        if (p.dh0 && !s_abort) {
+            float* dst = p.dh0 + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
+#pragma unroll
+            for (int i = 0; i < 64; ++i) dst[(size_t)i * D] = dh[i];
+        }
+    } else {
+        // ---------------------------------- issue warp ----------------------------------
+        const bool lead = (tid & 31) == 0;
+        // iteration `it` processes chunk n = N-1-it
+        auto issue_load = [&](int it) {
+            const int n = p.N - 1 - it;
+            unsigned char* st = smem + (it & 1) * kStage;
+            uint64_t* bar = &bar_load[it & 1];
+            mbar_expect_tx(bar, kStage);
+            const int yc = (int)(((size_t)bh * p.N + n) * D);
+            const int yt = (int)((size_t)bh * p.T + (size_t)n * C);
+            const int yi = (int)((size_t)b * p.T + (size_t)n * C);
+            tma_load_2d(st, &mapWt, 0, yc, bar);
+            tma_load_2d(st + 16384, &mapdO, hh * D, yi, bar);
+            tma_load_2d(st + 16384 + 8192, &mapdO, hh * D + 64, yi, bar);
+            tma_load_2d(st + 32768, &mapQg, 0, yt, bar);
+            tma_load_2d(st + 32768 + 8192, &mapQg, 64, yt, bar);
+            tma_load_2d(st + 49152, &mapK, hh * D, yi, bar);
+            tma_load_2d(st + 49152 + 8192, &mapK, hh * D + 64, yi, bar);
+            tma_load_2d(st + 65536, &mapP, 0, yt, bar);
+        };
+        if (lead) { issue_load(0); if (p.N > 1) issue_load(1); }
+        for (int it = 0; it < p.N; ++it) {
+            const int n = p.N - 1 - it;
+            const uint32_t st = smem_u32(smem + (it & 1) * kStage);
+            if (lead) wait(&bar_load[it & 1], (it >> 1) & 1);
+            nb_sync(kBarH);                               // dh^T operand (exit state of chunk n) is in place
+            if (lead) {
+                tc_fence_after();
+                const uint32_t sdO = st + 16384;
+                // A2 = dh^T K^T (A, B K-major) -- the critical product;  A1 = dO^T P (A, B MN-major: lines = token r)
+                umma_product<false, false>(tA2, smem_u32(sdH), 16384, st + 49152, 8192, C, D, false);
+                umma_product<true, true>(tA1, sdO, 8192, st + 65536, 8192, C, C, false);
+                umma_commit(&bar_a);
+                // H-accumulator = dO^T Qg (B MN-major: lines = token r, two blocks of d_k)
+                umma_product<true, true>(tH, sdO, 8192, st + 32768, 8192, D, C, false);
+                tma_store_wait_read_n<0>();               // dDelta^T tile of the previous chunk has been read
+                mbar_arrive(&bar_a);
+                // gradient w.r.t. the exit state of chunk n, bf16, as the operand tile (rows = d_v, cols = d_k)
+                const int yh = (int)(((size_t)bh * p.N + n) * D);
+                tma_store_2d(&mapdHs, sdH, 0, yh);
+                tma_store_2d(&mapdHs, sdH + 16384, 64, yh);
+                tma_store_commit();
+            }
+            nb_sync(kBarD);                               // dDelta^T operand of chunk n is in place
+            if (lead) {
+                tc_fence_after();
+                // H-accumulator -= dDelta^T W<-   (A negated; B K-major: lines = d_k index, contraction over tokens)
+                umma_product<false, false>(tH, smem_u32(sdD), 16384, st, 16384, D, C, true, true);
+                umma_commit(&bar_b);
+                umma_commit(&bar_e);
+                tma_store_2d(&mapdDt, sdD, 0, (int)(((size_t)bh * p.N + n) * D));
+                tma_store_commit();
+                tma_store_wait_read_n<1>();               // the dh^T tile may be rewritten
+                mbar_arrive(&bar_b);
+                wait(&bar_e, it & 1);                     // every product of this chunk has finished
+                if (it + 2 < p.N && !s_abort) issue_load(it + 2);
             }
         }
-        if (tid < C && n >= 1) sg[(it + 1) & 1][tid] = p.g[(size_t)bh * p.T + (size_t)(n - 1) * C + tid];
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-    }
-    if (aborted) {
-        if (tid == 0) {
-            *p.status = QD_ERR_TIMEOUT;
-            for (int it = loads_waited; it < p.N && it < loads_waited + 2; ++it) mbar_wait(&bar_load[it & 1], (it >> 1) & 1);
+        nb_sync(kBarH);                                   // final arrival of the compute warps
+        if (lead) {
+            tma_store_wait_all();
+            if (s_abort) { mbar_wait(&bar_load[0], 0); mbar_wait(&bar_load[1], 0); }
         }
-    } else if (p.dh0) {
-        float* dst = p.dh0 + (size_t)bh * D * D + tid;
-#pragma unroll
-        for (int i = 0; i < D; ++i) dst[(size_t)i * D] = dh[i];
     }
-    if (tid == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tbase, 256);
+    if (tid < 32) tmem_dealloc(tbase, 256);
 }
 
-// =================================================================================================
 // =================================================================================================
 struct ChunkBwdParams {
     int T, H, N;
@@ -750,23 +776,23 @@ cudaError_t tc_chain_bwd(const ChunkArgs& a) {
     const qd_shape& s = a.s;
     const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
     const uint64_t icols = (uint64_t)s.H * D, irows = (uint64_t)s.B * s.T;
-    CUtensorMap mWt, mdO, mQg, mK, mP, mdHs;
+    CUtensorMap mWt, mdO, mQg, mK, mP, mdHs, mdDt;
     if (!make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, BH * N * D, 128, 128) ||
         !make_tmap_bf16_2d(&mdO, a.dO, icols, irows, icols * 2, 64) ||
         !make_tmap_bf16_2d(&mQg, a.ws + a.TL.Qg, D, BH * s.T, D * 2, 64) ||
         !make_tmap_bf16_2d(&mK, a.k, icols, irows, icols * 2, 64) ||
         !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * s.T, 128, 64) ||
-        !make_tmap_bf16_2d(&mdHs, a.ws + a.TL.dhsT, D, BH * N * D, D * 2, 128))
+        !make_tmap_bf16_2d(&mdHs, a.ws + a.TL.dhsT, D, BH * N * D, D * 2, 128) ||
+        !make_tmap_bf16_2d(&mdDt, a.ws + a.TL.dDt, 64, BH * N * D, 128, 128))
         return cudaErrorInvalidValue;
     ChainBwdParams p{};
     p.T = s.T; p.H = s.H; p.N = (int)N;
     p.g = (const float*)(a.ws + a.TL.g);
     p.dhT = a.dhT; p.dh0 = a.dh0;
-    p.dDt = (bf16*)(a.ws + a.TL.dDt);
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_chain_bwd, kChainSmem);
     if (e != cudaSuccess) return e;
-    k_tc_chain_bwd<<<(unsigned)BH, 128, kChainSmem, a.stream>>>(mWt, mdO, mQg, mK, mP, mdHs, p);
+    k_tc_chain_bwd<<<(unsigned)BH, kChainThreads, kChainSmem, a.stream>>>(mWt, mdO, mQg, mK, mP, mdHs, mdDt, p);
     return cudaGetLastError();
 }
 

@@ -317,198 +317,263 @@ struct ChainParams {
     int T, H, N;
     const float* g;
     const float* h0;
-    bf16* o;
     float* hT;
-    bf16* Dt;                  // optional: Delta^T per chunk [dv][64]; kept for the backward
-    int save;                  // also store the bf16 entry state of every chunk through mapHs
+    int save;                  // also store, per chunk, the bf16 entry state (mapHs) and Delta^T (mapDt)
     unsigned* status;
 };
 
-constexpr int kStage = 73728;                           // Wt 16K | Ut 16K | Qg 16K | K 16K | P 8K
-constexpr int kChainSmem = 2 * kStage + 65536 + 1024;   // + hT operand 32K, Delta^T 16K, scaled Delta^T 16K
+constexpr int kStage = 73728;                                   // Wt 16K | Ut 16K | Qg 16K | K 16K | P 8K
+constexpr int kChainSmem = 2 * kStage + 65536 + 16384 + 1024;   // + h^T 32K, Delta^T 16K, scaled Delta^T 16K, O 16K
+constexpr int kChainThreads = 288;                 // 8 compute warps + 1 issue warp
+constexpr int kIssueWarp = 8;                      // its lane 0 issues every MMA and TMA copy
 
-__global__ void __launch_bounds__(128) k_tc_chain_fwd(const __grid_constant__ CUtensorMap mapWt,
-                                                      const __grid_constant__ CUtensorMap mapUt,
-                                                      const __grid_constant__ CUtensorMap mapQg,
-                                                      const __grid_constant__ CUtensorMap mapK,
-                                                      const __grid_constant__ CUtensorMap mapP,
-                                                      const __grid_constant__ CUtensorMap mapHs, ChainParams p) {
+// named barriers between the 256 compute threads (arrive) and the issue warp (sync)
+constexpr int kBarH = 1, kBarD = 2, kBarO = 3, kBarCount = kChainThreads;
+__device__ __forceinline__ void nb_arrive(int id) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(kBarCount) : "memory"); }
+__device__ __forceinline__ void nb_sync(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(kBarCount) : "memory"); }
+
+// Forward state chain.  The only true dependency per chunk is
+//   h ready -> Delta-accumulator = h^T Wt -> Delta^T -> H-accumulator = (scaled Delta^T) K -> h update;
+// the output products (h^T Qg^T + Delta^T P^T) and the output epilogue run in its shadow.
+// Compute warpgroup w owns tokens [32w, 32w+32) of the 64-column accumulators and d_k columns
+// [64w, 64w+64) of the state; thread l of a warpgroup owns TMEM lane l = d_v index.
+__global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_constant__ CUtensorMap mapWt,
+                                                                const __grid_constant__ CUtensorMap mapUt,
+                                                                const __grid_constant__ CUtensorMap mapQg,
+                                                                const __grid_constant__ CUtensorMap mapK,
+                                                                const __grid_constant__ CUtensorMap mapP,
+                                                                const __grid_constant__ CUtensorMap mapHs,
+                                                                const __grid_constant__ CUtensorMap mapDt,
+                                                                const __grid_constant__ CUtensorMap mapO,
+                                                                ChainParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char* sH = smem + 2 * kStage;          // h^T as A operand: K-major, 2 blocks of [128 lines][64]
     unsigned char* sD = sH + 32768;                 // Delta^T: K-major [128 lines (dv)][64 tokens]
     unsigned char* sDs = sD + 16384;                // Delta^T scaled by gamma_C/gamma_r per token
-    __shared__ uint64_t bar_load[2], bar_a, bar_b;
+    unsigned char* sO = sDs + 16384;                // output tile [64 tokens][128 dv], 2 blocks of [64 lines][64]
+    __shared__ uint64_t bar_load[2], bar_a, bar_b, bar_o, bar_e;
     __shared__ uint32_t tmem_slot;
-    __shared__ float sg[2][C];
+    __shared__ volatile int s_abort;
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, wg = tid >> 7, l = tid & 127, wq = (tid >> 5) & 3;
     const int bh = blockIdx.x, b = bh / p.H, hh = bh % p.H;
+    const bool compute = tid < 256;
 
     if (tid == 0) {
         mbar_init(&bar_load[0], 1); mbar_init(&bar_load[1], 1);
-        mbar_init(&bar_a, 1); mbar_init(&bar_b, 1);
+        mbar_init(&bar_a, 2); mbar_init(&bar_b, 2); mbar_init(&bar_o, 2); mbar_init(&bar_e, 1);
         mbar_init_fence();
+        s_abort = 0;
     }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    if (tid < 32) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tbase = tmem_slot;
     const uint32_t tD = tbase, tO = tbase + 64, tH = tbase + 128;
+    const uint32_t lane_base = (uint32_t)wq * 32;
 
-    auto issue_load = [&](int n) {
-        unsigned char* st = smem + (n & 1) * kStage;
-        uint64_t* bar = &bar_load[n & 1];
-        mbar_expect_tx(bar, kStage);
-        const int yc = (int)(((size_t)bh * p.N + n) * D);
-        const int yt = (int)((size_t)bh * p.T + (size_t)n * C);
-        tma_load_2d(st, &mapWt, 0, yc, bar);
-        tma_load_2d(st + 16384, &mapUt, 0, yc, bar);
-        tma_load_2d(st + 32768, &mapQg, 0, yt, bar);
-        tma_load_2d(st + 32768 + 8192, &mapQg, 64, yt, bar);
-        const int yk = (int)((size_t)b * p.T + (size_t)n * C);
-        tma_load_2d(st + 49152, &mapK, hh * D, yk, bar);
-        tma_load_2d(st + 49152 + 8192, &mapK, hh * D + 64, yk, bar);
-        tma_load_2d(st + 65536, &mapP, 0, yt, bar);
+    // bounded wait; once any wait has expired every later wait returns at once (the kernel drains)
+    auto wait = [&](uint64_t* bar, uint32_t parity) {
+        if (s_abort) return;
+        if (!mbar_wait(bar, parity)) { s_abort = 1; *p.status = QD_ERR_TIMEOUT; }
     };
-    if (tid == 0) { issue_load(0); if (p.N > 1) issue_load(1); }
+    const float* gseq = p.g + (size_t)bh * p.T;
 
-    // state: thread j holds row j of h^T (= column j of h), fp32
-    float h[D];
-    if (p.h0) {
-        const float* src = p.h0 + (size_t)bh * D * D + tid;
+    if (compute) {
+        // ---------------------------------- compute warps ----------------------------------
+        float h[64];      // h^T[j = l][64 wg .. 64 wg + 63], fp32
+        if (p.h0) {
+            const float* src = p.h0 + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
 #pragma unroll
-        for (int i = 0; i < D; ++i) h[i] = src[(size_t)i * D];
-    } else {
+            for (int i = 0; i < 64; ++i) h[i] = src[(size_t)i * D];
+        } else {
 #pragma unroll
-        for (int i = 0; i < D; ++i) h[i] = 0.f;
-    }
-#pragma unroll
-    for (int blk = 0; blk < 2; ++blk)
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch)
-            sts128(sH + blk * 16384 + sw128_chunk(tid, ch), pack8(h + blk * 64 + ch * 8));
-    if (tid < C) sg[0][tid] = p.g[(size_t)bh * p.T + tid];
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-
-    bool aborted = false;
-    int loads_waited = 0;
-    for (int n = 0; n < p.N; ++n) {
-        unsigned char* st = smem + (n & 1) * kStage;
-        const float* gc = sg[n & 1];
-        bool fail = !mbar_wait(&bar_load[n & 1], (n >> 1) & 1);
-        if (__syncthreads_or(fail)) { aborted = true; break; }
-        loads_waited = n + 1;
-        if (tid == 0) {
-            if (p.save) {
-                // entry state of chunk n, bf16, exactly the operand tile: rows = d_v index, cols = d_k index
-                const int yh = (int)(((size_t)bh * p.N + n) * D);
-                tma_store_2d(&mapHs, sH, 0, yh);
-                tma_store_2d(&mapHs, sH + 16384, 64, yh);
-                tma_store_commit();
-            }
-            tc_fence_after();
-            // Delta-accumulator = h^T Wt (B: MN-major, lines = d_k);  O-accumulator = h^T Qg^T (B: K-major)
-            umma_product<false, true>(tD, smem_u32(sH), 16384, smem_u32(st), 8192, C, D, false);
-            umma_product<false, false>(tO, smem_u32(sH), 16384, smem_u32(st + 32768), 8192, C, D, false);
-            umma_commit(&bar_a);
+            for (int i = 0; i < 64; ++i) h[i] = 0.f;
         }
-        fail = !mbar_wait(&bar_a, n & 1);
-        if (__syncthreads_or(fail)) { aborted = true; break; }
-        tc_fence_after();
-        // Delta^T = Ut - acc ; two bf16 copies (plain, and scaled by gamma_C/gamma_r) as A operands
-        {
-            const float gC = gc[C - 1];
-            const unsigned char* ut = st + 16384;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
+        for (int ch = 0; ch < 8; ++ch) sts128(sH + wg * 16384 + sw128_chunk(l, ch), pack8(h + ch * 8));
+        // byte offsets of my (fixed) column inside a staging line, for the 8 possible (token & 7)
+        uint32_t xoff[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            xoff[e] = (uint32_t)e * 128u + (((((uint32_t)l & 63u) >> 3) ^ (uint32_t)e) << 4) + ((uint32_t)l & 7u) * 2u;
+        fence_proxy_async();
+        nb_arrive(kBarH);
+
+        auto o_stage = [&]() {
+            // O^T row j = l, my 32 tokens -> staging tile (token-major); stored by TMA afterwards
+            unsigned char* stg = sO + (l >> 6) * 8192 + (wg * 32) * 128;
+            float v[32];
+            tmem_ld32(tmem_addr(tO, lane_base, wg * 32), v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sts16(stg + (i >> 3) * 1024 + xoff[i & 7], __float2bfloat16_rn(v[i]));
+            tc_fence_before();
+            fence_proxy_async();
+            nb_arrive(kBarO);
+        };
+
+        for (int n = 0; n < p.N; ++n) {
+            const unsigned char* st = smem + (n & 1) * kStage;
+            const float gC = gseq[(size_t)n * C + C - 1];
+            // decay ratios of my 32 tokens (global loads issued early)
+            float sc[32];
+            {
+                const float4* gp = reinterpret_cast<const float4*>(gseq + (size_t)n * C + wg * 32);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float4 t = gp[q];
+                    sc[q * 4] = t.x; sc[q * 4 + 1] = t.y; sc[q * 4 + 2] = t.z; sc[q * 4 + 3] = t.w;
+                }
+            }
+            if (n > 0) { wait(&bar_o, (n - 1) & 1); tc_fence_after(); o_stage(); }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sc[i] = __expf(gC - sc[i]);
+            wait(&bar_load[n & 1], (n >> 1) & 1);
+            wait(&bar_a, n & 1);
+            tc_fence_after();
+            // Delta^T = Ut - acc, my 32 tokens; two bf16 copies (plain, and scaled by gamma_C/gamma_r) as A operands
+            {
+                const unsigned char* ut = st + 16384;
                 float v[32];
-                tmem_ld32(tmem_addr(tD, warp * 32, half * 32), v);
+                tmem_ld32(tmem_addr(tD, lane_base, wg * 32), v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    float u[8], d0[8], d1[8];
-                    const uint32_t off = sw128_chunk(tid, half * 4 + ch);
+                for (int cc = 0; cc < 4; ++cc) {
+                    float u[8], d1[8];
+                    const uint32_t off = sw128_chunk(l, wg * 4 + cc);
                     load8(ut + off, u);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
-                        d0[e] = u[e] - v[ch * 8 + e];
-                        d1[e] = d0[e] * expf(gC - gc[half * 32 + ch * 8 + e]);
+                        u[e] -= v[cc * 8 + e];
+                        d1[e] = u[e] * sc[cc * 8 + e];
                     }
-                    const uint4 pk = pack8(d0);
-                    sts128(sD + off, pk);
+                    sts128(sD + off, pack8(u));
                     sts128(sDs + off, pack8(d1));
-                    if (p.Dt)
-                        *reinterpret_cast<uint4*>(p.Dt + (((size_t)bh * p.N + n) * D + tid) * C + half * 32 + ch * 8) = pk;
                 }
             }
-        }
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
-        if (tid == 0) {
+            tc_fence_before();
+            fence_proxy_async();
+            nb_arrive(kBarD);
+            // h^T <- gamma_C h^T + acc (my 64 d_k columns), refresh the bf16 operand copy
+            const float gamC = __expf(gC);
+            wait(&bar_b, n & 1);
             tc_fence_after();
-            // O += Delta^T P^T (B: K-major [r][s]);   H-accumulator = scaled Delta^T K (B: MN-major, lines = tokens)
-            umma_product<false, false>(tO, smem_u32(sD), 16384, smem_u32(st + 65536), 8192, C, C, true);
-            umma_product<false, true>(tH, smem_u32(sDs), 16384, smem_u32(st + 49152), 8192, D, C, false);
-            umma_commit(&bar_b);
+#pragma unroll
+            for (int q2 = 0; q2 < 2; ++q2) {
+                float v[32];
+                tmem_ld32(tmem_addr(tH, lane_base, wg * 64 + q2 * 32), v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) h[q2 * 32 + i] = fmaf(gamC, h[q2 * 32 + i], v[i]);
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc)
+                    sts128(sH + wg * 16384 + sw128_chunk(l, q2 * 4 + cc), pack8(h + q2 * 32 + cc * 8));
+            }
+            tc_fence_before();
+            fence_proxy_async();
+            nb_arrive(kBarH);
         }
-        fail = !mbar_wait(&bar_b, n & 1);
-        if (tid == 0 && p.save) tma_store_wait_read();      // the state tile is about to be rewritten
-        if (__syncthreads_or(fail)) { aborted = true; break; }
+        wait(&bar_o, (p.N - 1) & 1);
         tc_fence_after();
-        // this stage's tiles are consumed: refill it with chunk n+2
-        if (tid == 0 && n + 2 < p.N) issue_load(n + 2);
-        // h^T <- gamma_C h^T + acc, refresh the bf16 operand copy
-        {
-            const float gamC = expf(gc[C - 1]);
+        o_stage();
+        if (p.hT && !s_abort) {
+            float* dst = p.hT + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                float v[32];
-                tmem_ld32(tmem_addr(tH, warp * 32, q4 * 32), v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) h[q4 * 32 + i] = fmaf(gamC, h[q4 * 32 + i], v[i]);
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch)
-                    sts128(sH + (q4 >> 1) * 16384 + sw128_chunk(tid, (q4 & 1) * 4 + ch), pack8(h + q4 * 32 + ch * 8));
+            for (int i = 0; i < 64; ++i) dst[(size_t)i * D] = h[i];
+        }
+    } else {
+        // ---------------------------------- issue warp ----------------------------------
+        const bool lead = (tid & 31) == 0;
+        auto issue_load = [&](int n) {
+            unsigned char* st = smem + (n & 1) * kStage;
+            uint64_t* bar = &bar_load[n & 1];
+            mbar_expect_tx(bar, kStage);
+            const int yc = (int)(((size_t)bh * p.N + n) * D);
+            const int yt = (int)((size_t)bh * p.T + (size_t)n * C);
+            tma_load_2d(st, &mapWt, 0, yc, bar);
+            tma_load_2d(st + 16384, &mapUt, 0, yc, bar);
+            tma_load_2d(st + 32768, &mapQg, 0, yt, bar);
+            tma_load_2d(st + 32768 + 8192, &mapQg, 64, yt, bar);
+            const int yk = (int)((size_t)b * p.T + (size_t)n * C);
+            tma_load_2d(st + 49152, &mapK, hh * D, yk, bar);
+            tma_load_2d(st + 49152 + 8192, &mapK, hh * D + 64, yk, bar);
+            tma_load_2d(st + 65536, &mapP, 0, yt, bar);
+        };
+        if (lead) { issue_load(0); if (p.N > 1) issue_load(1); }
+        for (int n = 0; n < p.N; ++n) {
+            const uint32_t st = smem_u32(smem + (n & 1) * kStage);
+            if (lead) wait(&bar_load[n & 1], (n >> 1) & 1);
+            nb_sync(kBarH);                               // h^T operand of chunk n is in place
+            if (lead) {
+                tc_fence_after();
+                // Delta-accumulator = h^T Wt (B: MN-major, lines = d_k)
+                umma_product<false, true>(tD, smem_u32(sH), 16384, st, 8192, C, D, false);
+                umma_commit(&bar_a);
+                tma_store_wait_read_n<0>();               // Delta^T and output tiles of earlier chunks have been read
+                mbar_arrive(&bar_a);
+                if (p.save) {
+                    // entry state of chunk n, bf16, exactly the operand tile: rows = d_v index, cols = d_k index
+                    const int yh = (int)(((size_t)bh * p.N + n) * D);
+                    tma_store_2d(&mapHs, sH, 0, yh);
+                    tma_store_2d(&mapHs, sH + 16384, 64, yh);
+                }
+                tma_store_commit();                       // group: entry state of chunk n
+            }
+            if (n > 0) {
+                nb_sync(kBarO);                           // output tile of chunk n-1 staged, O-accumulator free
+                if (lead) {
+                    const int yo = (int)((size_t)b * p.T + (size_t)(n - 1) * C);
+                    tma_store_2d(&mapO, sO, hh * D, yo);
+                    tma_store_2d(&mapO, sO + 8192, hh * D + 64, yo);
+                    tma_store_commit();                   // group: output of chunk n-1
+                }
+            }
+            if (lead) {
+                tc_fence_after();
+                // O-accumulator = h^T Qg^T (B: K-major); reads the state tile, so it must precede the release
+                // of that tile (the commit behind the H product below covers it)
+                umma_product<false, false>(tO, smem_u32(sH), 16384, st + 32768, 8192, C, D, false);
+            }
+            nb_sync(kBarD);                               // Delta^T operands of chunk n are in place
+            if (lead) {
+                tc_fence_after();
+                // H-accumulator = scaled Delta^T K (B: MN-major, lines = tokens): the critical product first
+                umma_product<false, true>(tH, smem_u32(sDs), 16384, st + 49152, 8192, D, C, false);
+                umma_commit(&bar_b);
+                // O-accumulator += Delta^T P^T (B: K-major [r][s])
+                umma_product<false, false>(tO, smem_u32(sD), 16384, st + 65536, 8192, C, C, true);
+                umma_commit(&bar_o);
+                umma_commit(&bar_e);
+                if (p.save) tma_store_2d(&mapDt, sD, 0, (int)(((size_t)bh * p.N + n) * D));
+                tma_store_commit();                       // group: Delta^T of chunk n (possibly empty)
+                tma_store_wait_read_n<1>();               // entry-state and output tiles may be rewritten
+                mbar_arrive(&bar_b);
+                mbar_arrive(&bar_o);
+                // every product of chunk n has finished: its stage can take chunk n+2
+                wait(&bar_e, n & 1);
+                if (n + 2 < p.N && !s_abort) issue_load(n + 2);
             }
         }
-        // O^T row j -> o[b, t0 + r, hh, j]
-        {
-            bf16* orow = p.o + (((size_t)b * p.T + (size_t)n * C) * p.H + hh) * D + tid;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                float v[32];
-                tmem_ld32(tmem_addr(tO, warp * 32, half * 32), v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) orow[(size_t)(half * 32 + i) * p.H * D] = __float2bfloat16_rn(v[i]);
+        nb_sync(kBarH);                                   // final arrival of the compute warps (state of chunk N)
+        nb_sync(kBarO);                                   // output tile of the last chunk staged
+        if (lead) {
+            const int yo = (int)((size_t)b * p.T + (size_t)(p.N - 1) * C);
+            tma_store_2d(&mapO, sO, hh * D, yo);
+            tma_store_2d(&mapO, sO + 8192, hh * D + 64, yo);
+            tma_store_commit();
+            tma_store_wait_all();
+            if (s_abort) {
+                // loads that were issued but never consumed may still be in flight: one more bounded chance
+                mbar_wait(&bar_load[0], 0); mbar_wait(&bar_load[1], 0);
             }
         }
-        if (tid < C && n + 1 < p.N) sg[(n + 1) & 1][tid] = p.g[(size_t)bh * p.T + (size_t)(n + 1) * C + tid];
-        fence_proxy_async();
-        tc_fence_before();
-        __syncthreads();
     }
-    if (aborted) {
-        if (tid == 0) {
-            *p.status = QD_ERR_TIMEOUT;
-            // loads already issued for chunks loads_waited .. min(N, loads_waited + 2) - 1 may be in flight
-            for (int n = loads_waited; n < p.N && n < loads_waited + 2; ++n) mbar_wait(&bar_load[n & 1], (n >> 1) & 1);
-        }
-    } else if (p.hT) {
-        float* dst = p.hT + (size_t)bh * D * D + tid;
-#pragma unroll
-        for (int i = 0; i < D; ++i) dst[(size_t)i * D] = h[i];
-    }
-    if (tid == 0 && p.save) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tbase, 256);
+    if (tid < 32) tmem_dealloc(tbase, 256);
 }
 
 template <class K>
@@ -570,24 +635,26 @@ cudaError_t tc_prep(const ChunkArgs& a) {
 cudaError_t tc_chain_fwd(const ChunkArgs& a) {
     const qd_shape& s = a.s;
     const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
-    CUtensorMap mWt, mUt, mQg, mK, mP, mHs;
+    const uint64_t icols = (uint64_t)s.H * D, irows = (uint64_t)s.B * s.T;
+    CUtensorMap mWt, mUt, mQg, mK, mP, mHs, mDt, mO;
     if (!make_tmap_bf16_2d(&mHs, a.ws + a.TL.hsT, D, BH * N * D, D * 2, 128) ||
+        !make_tmap_bf16_2d(&mDt, a.ws + a.TL.Dt, 64, BH * N * D, 128, 128) ||
+        !make_tmap_bf16_2d(&mO, a.o, icols, irows, icols * 2, 64) ||
         !make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, BH * N * D, 128, 128) ||
         !make_tmap_bf16_2d(&mUt, a.ws + a.TL.Ut, 64, BH * N * D, 128, 128) ||
         !make_tmap_bf16_2d(&mQg, a.ws + a.TL.Qg, D, BH * s.T, D * 2, 64) ||
-        !make_tmap_bf16_2d(&mK, a.k, (uint64_t)s.H * D, (uint64_t)s.B * s.T, (uint64_t)s.H * D * 2, 64) ||
+        !make_tmap_bf16_2d(&mK, a.k, icols, irows, icols * 2, 64) ||
         !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * s.T, 128, 64))
         return cudaErrorInvalidValue;
     ChainParams p{};
     p.T = s.T; p.H = s.H; p.N = (int)N;
     p.g = (const float*)(a.ws + a.TL.g);
-    p.h0 = a.h0; p.o = (bf16*)a.o; p.hT = a.hT;
+    p.h0 = a.h0; p.hT = a.hT;
     p.save = a.save ? 1 : 0;
-    p.Dt = a.save ? (bf16*)(a.ws + a.TL.Dt) : nullptr;
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_chain_fwd, kChainSmem);
     if (e != cudaSuccess) return e;
-    k_tc_chain_fwd<<<(unsigned)BH, 128, kChainSmem, a.stream>>>(mWt, mUt, mQg, mK, mP, mHs, p);
+    k_tc_chain_fwd<<<(unsigned)BH, kChainThreads, kChainSmem, a.stream>>>(mWt, mUt, mQg, mK, mP, mHs, mDt, mO, p);
     return cudaGetLastError();
 }
 
