@@ -70,16 +70,18 @@ struct ChainBwdParams {
 
 constexpr int kStage = 73728;                           // Wt 16K | dO 16K | Qg 16K | K 16K | P 8K
 constexpr int kChainSmem = 2 * kStage + 32768 + 16384 + 1024;
-constexpr int kChainThreads = 288;                 // 8 compute warps + 1 issue warp
+constexpr int kChainThreads = 320;                 // 8 compute warps, 1 MMA-issue warp, 1 TMA warp
+constexpr int kMmaWarp = 8;
 
-// named barriers between the 256 compute threads (arrive) and the issue warp (sync)
-constexpr int kBarH = 1, kBarD = 2, kBarCount = kChainThreads;
-__device__ __forceinline__ void nb_arrive(int id) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(kBarCount) : "memory"); }
-__device__ __forceinline__ void nb_sync(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(kBarCount) : "memory"); }
+// named barriers: compute threads arrive, the MMA and TMA warps wait
+constexpr int kBarH = 1, kBarD = 2;
+__device__ __forceinline__ void nb_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+__device__ __forceinline__ void nb_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 
 // Reverse state chain.  Per chunk the dependency is
 //   dh ready -> A2 = dh^T K^T -> dDelta^T -> H-accumulator -= dDelta^T W<- -> dh update;
-// A1 = dO^T P and the dO^T Qg part of the H-accumulator do not depend on dh.
+// A1 = dO^T P and the dO^T Qg part of the H-accumulator do not depend on dh; every TMA copy is
+// issued by its own warp.
 // Compute warpgroup w owns tokens [32w, 32w+32) of the 64-column accumulators and d_k columns
 // [64w, 64w+64) of dh^T; thread l of a warpgroup owns TMEM lane l = d_v index.
 __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_constant__ CUtensorMap mapWt,
@@ -98,9 +100,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int s_abort;
 
-    const int tid = threadIdx.x, wg = tid >> 7, l = tid & 127, wq = (tid >> 5) & 3;
+    const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, l = tid & 127, wq = warp & 3;
     const int bh = blockIdx.x, b = bh / p.H, hh = bh % p.H;
-    const bool compute = tid < 256;
 
     if (tid == 0) {
         mbar_init(&bar_load[0], 1); mbar_init(&bar_load[1], 1);
@@ -123,7 +124,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
     };
     const float* gseq = p.g + (size_t)bh * p.T;
 
-    if (compute) {
+    if (warp < 8) {
         // ---------------------------------- compute warps ----------------------------------
         float dh[64];     // dh^T[j = l][64 wg .. 64 wg + 63]
         if (p.dhT) {
@@ -137,7 +138,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) sts128(sdH + wg * 16384 + sw128_chunk(l, ch), pack8(dh + ch * 8));
         fence_proxy_async();
-        nb_arrive(kBarH);
+        nb_arrive(kBarH, 320);
 
         for (int it = 0; it < p.N; ++it) {
             const int n = p.N - 1 - it;
@@ -169,7 +170,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarD);
+            nb_arrive(kBarD, 320);
             wait(&bar_b, it & 1);
             tc_fence_after();
 #pragma unroll
@@ -185,15 +186,43 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarH);
+            nb_arrive(kBarH, 320);
         }
         if (p.dh0 && !s_abort) {
             float* dst = p.dh0 + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
 #pragma unroll
             for (int i = 0; i < 64; ++i) dst[(size_t)i * D] = dh[i];
         }
+    } else if (warp == kMmaWarp) {
+        // ---------------------------------- MMA-issue warp ----------------------------------
+        const bool lead = (tid & 31) == 0;
+        const uint32_t adH = smem_u32(sdH), adD = smem_u32(sdD);
+        for (int it = 0; it < p.N; ++it) {
+            const uint32_t st = smem_u32(smem + (it & 1) * kStage);
+            if (lead) wait(&bar_load[it & 1], (it >> 1) & 1);
+            nb_sync(kBarH, 320);                          // dh^T operand (exit state of this chunk) is in place
+            if (lead) {
+                tc_fence_after();
+                const uint32_t sdO = st + 16384;
+                // A2 = dh^T K^T (A, B K-major) -- the critical product;  A1 = dO^T P (A, B MN-major: lines = token r)
+                umma_product<false, false>(tA2, adH, 16384, st + 49152, 8192, C, D, false);
+                umma_product<true, true>(tA1, sdO, 8192, st + 65536, 8192, C, C, false);
+                umma_commit(&bar_a);
+                // H-accumulator = dO^T Qg (B MN-major: lines = token r, two blocks of d_k)
+                umma_product<true, true>(tH, sdO, 8192, st + 32768, 8192, D, C, false);
+            }
+            nb_sync(kBarD, 320);                          // dDelta^T operand is in place
+            if (lead) {
+                tc_fence_after();
+                // H-accumulator -= dDelta^T W<-   (A negated; B K-major: lines = d_k index, contraction over tokens)
+                umma_product<false, false>(tH, adD, 16384, st, 16384, D, C, true, true);
+                umma_commit(&bar_b);
+                umma_commit(&bar_e);
+            }
+        }
+        nb_sync(kBarH, 320);                              // final arrival of the compute warps
     } else {
-        // ---------------------------------- issue warp ----------------------------------
+        // ---------------------------------- TMA warp ----------------------------------
         const bool lead = (tid & 31) == 0;
         // iteration `it` processes chunk n = N-1-it
         auto issue_load = [&](int it) {
@@ -216,42 +245,29 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
         if (lead) { issue_load(0); if (p.N > 1) issue_load(1); }
         for (int it = 0; it < p.N; ++it) {
             const int n = p.N - 1 - it;
-            const uint32_t st = smem_u32(smem + (it & 1) * kStage);
-            if (lead) wait(&bar_load[it & 1], (it >> 1) & 1);
-            nb_sync(kBarH);                               // dh^T operand (exit state of chunk n) is in place
             if (lead) {
-                tc_fence_after();
-                const uint32_t sdO = st + 16384;
-                // A2 = dh^T K^T (A, B K-major) -- the critical product;  A1 = dO^T P (A, B MN-major: lines = token r)
-                umma_product<false, false>(tA2, smem_u32(sdH), 16384, st + 49152, 8192, C, D, false);
-                umma_product<true, true>(tA1, sdO, 8192, st + 65536, 8192, C, C, false);
-                umma_commit(&bar_a);
-                // H-accumulator = dO^T Qg (B MN-major: lines = token r, two blocks of d_k)
-                umma_product<true, true>(tH, sdO, 8192, st + 32768, 8192, D, C, false);
                 tma_store_wait_read_n<0>();               // dDelta^T tile of the previous chunk has been read
                 mbar_arrive(&bar_a);
+            }
+            nb_sync(kBarH, 320);                          // dh^T operand (exit state of chunk n) is in place
+            if (lead) {
                 // gradient w.r.t. the exit state of chunk n, bf16, as the operand tile (rows = d_v, cols = d_k)
                 const int yh = (int)(((size_t)bh * p.N + n) * D);
                 tma_store_2d(&mapdHs, sdH, 0, yh);
                 tma_store_2d(&mapdHs, sdH + 16384, 64, yh);
                 tma_store_commit();
             }
-            nb_sync(kBarD);                               // dDelta^T operand of chunk n is in place
+            nb_sync(kBarD, 320);                          // dDelta^T of chunk n is in place
             if (lead) {
-                tc_fence_after();
-                // H-accumulator -= dDelta^T W<-   (A negated; B K-major: lines = d_k index, contraction over tokens)
-                umma_product<false, false>(tH, smem_u32(sdD), 16384, st, 16384, D, C, true, true);
-                umma_commit(&bar_b);
-                umma_commit(&bar_e);
                 tma_store_2d(&mapdDt, sdD, 0, (int)(((size_t)bh * p.N + n) * D));
                 tma_store_commit();
-                tma_store_wait_read_n<1>();               // the dh^T tile may be rewritten
+                tma_store_wait_read_n<1>();               // the dh^T tile has been read: it may be rewritten
                 mbar_arrive(&bar_b);
-                wait(&bar_e, it & 1);                     // every product of this chunk has finished
+                wait(&bar_e, it & 1);                     // every product of this chunk has finished: refill its stage
                 if (it + 2 < p.N && !s_abort) issue_load(it + 2);
             }
         }
-        nb_sync(kBarH);                                   // final arrival of the compute warps
+        nb_sync(kBarH, 320);                              // final arrival of the compute warps
         if (lead) {
             tma_store_wait_all();
             if (s_abort) { mbar_wait(&bar_load[0], 0); mbar_wait(&bar_load[1], 0); }

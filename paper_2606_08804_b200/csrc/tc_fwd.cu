@@ -324,17 +324,18 @@ struct ChainParams {
 
 constexpr int kStage = 73728;                                   // Wt 16K | Ut 16K | Qg 16K | K 16K | P 8K
 constexpr int kChainSmem = 2 * kStage + 65536 + 16384 + 1024;   // + h^T 32K, Delta^T 16K, scaled Delta^T 16K, O 16K
-constexpr int kChainThreads = 288;                 // 8 compute warps + 1 issue warp
-constexpr int kIssueWarp = 8;                      // its lane 0 issues every MMA and TMA copy
+constexpr int kChainThreads = 320;                 // 8 compute warps, 1 MMA-issue warp, 1 TMA warp
+constexpr int kMmaWarp = 8, kTmaWarp = 9;
 
-// named barriers between the 256 compute threads (arrive) and the issue warp (sync)
-constexpr int kBarH = 1, kBarD = 2, kBarO = 3, kBarCount = kChainThreads;
-__device__ __forceinline__ void nb_arrive(int id) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(kBarCount) : "memory"); }
-__device__ __forceinline__ void nb_sync(int id) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(kBarCount) : "memory"); }
+// named barriers: compute threads arrive, the MMA and/or TMA warp wait
+constexpr int kBarH = 1, kBarD = 2, kBarO = 3;
+__device__ __forceinline__ void nb_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+__device__ __forceinline__ void nb_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 
 // Forward state chain.  The only true dependency per chunk is
 //   h ready -> Delta-accumulator = h^T Wt -> Delta^T -> H-accumulator = (scaled Delta^T) K -> h update;
-// the output products (h^T Qg^T + Delta^T P^T) and the output epilogue run in its shadow.
+// the output products (h^T Qg^T + Delta^T P^T, double-buffered accumulator), the output epilogue and
+// every TMA copy run in its shadow on their own warps.
 // Compute warpgroup w owns tokens [32w, 32w+32) of the 64-column accumulators and d_k columns
 // [64w, 64w+64) of the state; thread l of a warpgroup owns TMEM lane l = d_v index.
 __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_constant__ CUtensorMap mapWt,
@@ -356,9 +357,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int s_abort;
 
-    const int tid = threadIdx.x, wg = tid >> 7, l = tid & 127, wq = (tid >> 5) & 3;
+    const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, l = tid & 127, wq = warp & 3;
     const int bh = blockIdx.x, b = bh / p.H, hh = bh % p.H;
-    const bool compute = tid < 256;
 
     if (tid == 0) {
         mbar_init(&bar_load[0], 1); mbar_init(&bar_load[1], 1);
@@ -366,12 +366,12 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         mbar_init_fence();
         s_abort = 0;
     }
-    if (tid < 32) { tmem_alloc(&tmem_slot, 256); tmem_relinquish(); }
+    if (tid < 32) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tbase = tmem_slot;
-    const uint32_t tD = tbase, tO = tbase + 64, tH = tbase + 128;
+    const uint32_t tD = tbase, tH = tbase + 128, tO0 = tbase + 256;      // O-accumulators: tO0 + 64 * (n & 1)
     const uint32_t lane_base = (uint32_t)wq * 32;
 
     // bounded wait; once any wait has expired every later wait returns at once (the kernel drains)
@@ -381,7 +381,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
     };
     const float* gseq = p.g + (size_t)bh * p.T;
 
-    if (compute) {
+    if (warp < 8) {
         // ---------------------------------- compute warps ----------------------------------
         float h[64];      // h^T[j = l][64 wg .. 64 wg + 63], fp32
         if (p.h0) {
@@ -400,25 +400,33 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         for (int e = 0; e < 8; ++e)
             xoff[e] = (uint32_t)e * 128u + (((((uint32_t)l & 63u) >> 3) ^ (uint32_t)e) << 4) + ((uint32_t)l & 7u) * 2u;
         fence_proxy_async();
-        nb_arrive(kBarH);
+        nb_arrive(kBarH, 320);
 
-        auto o_stage = [&]() {
-            // O^T row j = l, my 32 tokens -> staging tile (token-major); stored by TMA afterwards
+        auto o_stage = [&](int m) {
+            // output of chunk m: O^T row j = l, my 32 tokens -> staging tile (token-major); stored by the TMA warp
             unsigned char* stg = sO + (l >> 6) * 8192 + (wg * 32) * 128;
             float v[32];
-            tmem_ld32(tmem_addr(tO, lane_base, wg * 32), v);
+            tmem_ld32(tmem_addr(tO0 + 64 * (m & 1), lane_base, wg * 32), v);
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 32; ++i) sts16(stg + (i >> 3) * 1024 + xoff[i & 7], __float2bfloat16_rn(v[i]));
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarO);
+            nb_arrive(kBarO, 288);
         };
 
+#ifdef QD_PHASE_CLOCKS
+#define QD_C(i) do { if (blockIdx.x == 5 && tid == 0 && n == 10) ((long long*)((char*)p.status + 64))[i] = clock64(); } while (0)
+#define QD_M(i) do { if (blockIdx.x == 5 && lead && n == 10) ((long long*)((char*)p.status + 64))[12 + (i)] = clock64(); } while (0)
+#else
+#define QD_C(i) do { } while (0)
+#define QD_M(i) do { } while (0)
+#endif
         for (int n = 0; n < p.N; ++n) {
+            QD_C(0);
             const unsigned char* st = smem + (n & 1) * kStage;
             const float gC = gseq[(size_t)n * C + C - 1];
-            // decay ratios of my 32 tokens (global loads issued early)
+            // decay ratios of my 32 tokens
             float sc[32];
             {
                 const float4* gp = reinterpret_cast<const float4*>(gseq + (size_t)n * C + wg * 32);
@@ -428,11 +436,13 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                     sc[q * 4] = t.x; sc[q * 4 + 1] = t.y; sc[q * 4 + 2] = t.z; sc[q * 4 + 3] = t.w;
                 }
             }
-            if (n > 0) { wait(&bar_o, (n - 1) & 1); tc_fence_after(); o_stage(); }
 #pragma unroll
             for (int i = 0; i < 32; ++i) sc[i] = __expf(gC - sc[i]);
+            const float gamC = __expf(gC);
+            QD_C(1);
             wait(&bar_load[n & 1], (n >> 1) & 1);
             wait(&bar_a, n & 1);
+            QD_C(2);
             tc_fence_after();
             // Delta^T = Ut - acc, my 32 tokens; two bf16 copies (plain, and scaled by gamma_C/gamma_r) as A operands
             {
@@ -456,10 +466,14 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarD);
+            nb_arrive(kBarD, 320);
+            QD_C(3);
+            // in the shadow of the H product: output epilogue of the previous chunk
+            if (n > 0) { wait(&bar_o, (n - 1) & 1); tc_fence_after(); o_stage(n - 1); }
+            QD_C(4);
             // h^T <- gamma_C h^T + acc (my 64 d_k columns), refresh the bf16 operand copy
-            const float gamC = __expf(gC);
             wait(&bar_b, n & 1);
+            QD_C(5);
             tc_fence_after();
 #pragma unroll
             for (int q2 = 0; q2 < 2; ++q2) {
@@ -474,18 +488,57 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarH);
+            nb_arrive(kBarH, 320);
+            QD_C(6);
         }
         wait(&bar_o, (p.N - 1) & 1);
         tc_fence_after();
-        o_stage();
+        o_stage(p.N - 1);
         if (p.hT && !s_abort) {
             float* dst = p.hT + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
 #pragma unroll
             for (int i = 0; i < 64; ++i) dst[(size_t)i * D] = h[i];
         }
+    } else if (warp == kMmaWarp) {
+        // ---------------------------------- MMA-issue warp ----------------------------------
+        const bool lead = (tid & 31) == 0;
+        const uint32_t aH = smem_u32(sH), aD = smem_u32(sD), aDs = smem_u32(sDs);
+        for (int n = 0; n < p.N; ++n) {
+            const uint32_t st = smem_u32(smem + (n & 1) * kStage);
+            const uint32_t tO = tO0 + 64 * (n & 1);
+            QD_M(0);
+            if (lead) wait(&bar_load[n & 1], (n >> 1) & 1);
+            nb_sync(kBarH, 320);                          // h^T operand of chunk n is in place
+            QD_M(1);
+            if (lead) {
+                tc_fence_after();
+                // Delta-accumulator = h^T Wt (B: MN-major, lines = d_k)
+                umma_product<false, true>(tD, aH, 16384, st, 8192, C, D, false);
+                umma_commit(&bar_a);
+                QD_M(2);
+                // O-accumulator = h^T Qg^T (B: K-major); it reads the state tile, so the commit behind the
+                // H product below (which releases that tile) must cover it
+                umma_product<false, false>(tO, aH, 16384, st + 32768, 8192, C, D, false);
+            }
+            QD_M(3);
+            nb_sync(kBarD, 320);                          // Delta^T operands of chunk n are in place
+            QD_M(4);
+            if (lead) {
+                tc_fence_after();
+                // H-accumulator = scaled Delta^T K (B: MN-major, lines = tokens)
+                umma_product<false, true>(tH, aDs, 16384, st + 49152, 8192, D, C, false);
+                umma_commit(&bar_b);
+                QD_M(5);
+                // O-accumulator += Delta^T P^T (B: K-major [r][s])
+                umma_product<false, false>(tO, aD, 16384, st + 65536, 8192, C, C, true);
+                umma_commit(&bar_o);
+                umma_commit(&bar_e);
+                QD_M(6);
+            }
+        }
+        nb_sync(kBarH, 320);                              // final arrival of the compute warps
     } else {
-        // ---------------------------------- issue warp ----------------------------------
+        // ---------------------------------- TMA warp ----------------------------------
         const bool lead = (tid & 31) == 0;
         auto issue_load = [&](int n) {
             unsigned char* st = smem + (n & 1) * kStage;
@@ -504,26 +557,30 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         };
         if (lead) { issue_load(0); if (p.N > 1) issue_load(1); }
         for (int n = 0; n < p.N; ++n) {
-            const uint32_t st = smem_u32(smem + (n & 1) * kStage);
-            if (lead) wait(&bar_load[n & 1], (n >> 1) & 1);
-            nb_sync(kBarH);                               // h^T operand of chunk n is in place
             if (lead) {
-                tc_fence_after();
-                // Delta-accumulator = h^T Wt (B: MN-major, lines = d_k)
-                umma_product<false, true>(tD, smem_u32(sH), 16384, st, 8192, C, D, false);
-                umma_commit(&bar_a);
-                tma_store_wait_read_n<0>();               // Delta^T and output tiles of earlier chunks have been read
+                // every store issued so far (Delta^T of chunk n-1, output of chunk n-2) has read its tile:
+                // the Delta^T tiles may be rewritten (chunk n), the output staging tile too (chunk n-1)
+                tma_store_wait_read_n<0>();
                 mbar_arrive(&bar_a);
-                if (p.save) {
-                    // entry state of chunk n, bf16, exactly the operand tile: rows = d_v index, cols = d_k index
-                    const int yh = (int)(((size_t)bh * p.N + n) * D);
-                    tma_store_2d(&mapHs, sH, 0, yh);
-                    tma_store_2d(&mapHs, sH + 16384, 64, yh);
-                }
-                tma_store_commit();                       // group: entry state of chunk n
+                if (n > 0) mbar_arrive(&bar_o);
+            }
+            nb_sync(kBarH, 320);                          // h^T operand of chunk n is in place
+            if (lead && p.save) {
+                // entry state of chunk n, bf16, exactly the operand tile: rows = d_v index, cols = d_k index
+                const int yh = (int)(((size_t)bh * p.N + n) * D);
+                tma_store_2d(&mapHs, sH, 0, yh);
+                tma_store_2d(&mapHs, sH + 16384, 64, yh);
+            }
+            if (lead) tma_store_commit();                 // group: entry state of chunk n
+            nb_sync(kBarD, 320);                          // Delta^T of chunk n is in place
+            if (lead) {
+                if (p.save) tma_store_2d(&mapDt, sD, 0, (int)(((size_t)bh * p.N + n) * D));
+                tma_store_commit();                       // group: Delta^T of chunk n
+                tma_store_wait_read_n<1>();               // the entry-state tile has been read: it may be rewritten
+                mbar_arrive(&bar_b);
             }
             if (n > 0) {
-                nb_sync(kBarO);                           // output tile of chunk n-1 staged, O-accumulator free
+                nb_sync(kBarO, 288);                      // output tile of chunk n-1 staged
                 if (lead) {
                     const int yo = (int)((size_t)b * p.T + (size_t)(n - 1) * C);
                     tma_store_2d(&mapO, sO, hh * D, yo);
@@ -532,48 +589,25 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 }
             }
             if (lead) {
-                tc_fence_after();
-                // O-accumulator = h^T Qg^T (B: K-major); reads the state tile, so it must precede the release
-                // of that tile (the commit behind the H product below covers it)
-                umma_product<false, false>(tO, smem_u32(sH), 16384, st + 32768, 8192, C, D, false);
-            }
-            nb_sync(kBarD);                               // Delta^T operands of chunk n are in place
-            if (lead) {
-                tc_fence_after();
-                // H-accumulator = scaled Delta^T K (B: MN-major, lines = tokens): the critical product first
-                umma_product<false, true>(tH, smem_u32(sDs), 16384, st + 49152, 8192, D, C, false);
-                umma_commit(&bar_b);
-                // O-accumulator += Delta^T P^T (B: K-major [r][s])
-                umma_product<false, false>(tO, smem_u32(sD), 16384, st + 65536, 8192, C, C, true);
-                umma_commit(&bar_o);
-                umma_commit(&bar_e);
-                if (p.save) tma_store_2d(&mapDt, sD, 0, (int)(((size_t)bh * p.N + n) * D));
-                tma_store_commit();                       // group: Delta^T of chunk n (possibly empty)
-                tma_store_wait_read_n<1>();               // entry-state and output tiles may be rewritten
-                mbar_arrive(&bar_b);
-                mbar_arrive(&bar_o);
-                // every product of chunk n has finished: its stage can take chunk n+2
-                wait(&bar_e, n & 1);
+                wait(&bar_e, n & 1);                      // every product of chunk n has finished: refill its stage
                 if (n + 2 < p.N && !s_abort) issue_load(n + 2);
             }
         }
-        nb_sync(kBarH);                                   // final arrival of the compute warps (state of chunk N)
-        nb_sync(kBarO);                                   // output tile of the last chunk staged
+        nb_sync(kBarH, 320);                              // final arrival of the compute warps
+        if (lead) { tma_store_wait_read_n<0>(); mbar_arrive(&bar_o); }
+        nb_sync(kBarO, 288);                              // output tile of the last chunk staged
         if (lead) {
             const int yo = (int)((size_t)b * p.T + (size_t)(p.N - 1) * C);
             tma_store_2d(&mapO, sO, hh * D, yo);
             tma_store_2d(&mapO, sO + 8192, hh * D + 64, yo);
             tma_store_commit();
             tma_store_wait_all();
-            if (s_abort) {
-                // loads that were issued but never consumed may still be in flight: one more bounded chance
-                mbar_wait(&bar_load[0], 0); mbar_wait(&bar_load[1], 0);
-            }
+            if (s_abort) { mbar_wait(&bar_load[0], 0); mbar_wait(&bar_load[1], 0); }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (tid < 32) tmem_dealloc(tbase, 256);
+    if (tid < 32) tmem_dealloc(tbase, 512);
 }
 
 template <class K>
