@@ -1,6 +1,8 @@
 // C-ABI entry points: argument validation, workspace carving, kernel sequencing.
 #include "internal.h"
 
+#include <cstdio>
+#include <cstdlib>
 #include <vector>
 
 namespace qd {
@@ -80,7 +82,14 @@ struct StageTimer {
 
 template <class F> static cudaError_t timed(int stage, cudaStream_t s, F f) {
     StageTimer t(stage, s);
-    return f();
+    cudaError_t e = f();
+    // QDELTA_DEBUG=1 (debugging aid, breaks the "never synchronises" rule on purpose): wait for the
+    // stage and say which one failed
+    if (getenv("QDELTA_DEBUG")) {
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) fprintf(stderr, "[qdelta] stage %s: %s\n", kStageNames[stage], cudaGetErrorString(e));
+    }
+    return e;
 }
 
 }  // namespace qd

@@ -116,6 +116,13 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float* v) {
                  : "r"(taddr)
                  : "memory");
 }
+// store 8 consecutive 32-bit columns of this thread's lane
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 // address of (lane, column) relative to an allocation base
 __device__ __forceinline__ uint32_t tmem_addr(uint32_t base, uint32_t lane, uint32_t col) {
     return base + (lane << 16) + col;
@@ -176,6 +183,28 @@ __device__ __forceinline__ void umma_product(uint32_t d_tmem, uint32_t a_saddr, 
         const uint32_t ao = A_MN ? (uint32_t)k * 128u : (uint32_t)(k >> 6) * a_blk + (uint32_t)(k & 63) * 2u;
         const uint32_t bo = B_MN ? (uint32_t)k * 128u : (uint32_t)(k >> 6) * b_blk + (uint32_t)(k & 63) * 2u;
         umma_ss(d_tmem, a0 + (uint64_t)(ao >> 4), b0 + (uint64_t)(bo >> 4), idesc, accumulate || k > 0);
+    }
+}
+
+// D[tmem] (+)= A[tmem] * B[smem]: the A operand (M = 128 rows on the 128 lanes, bf16 pairs packed two per
+// 32-bit column: column c of lane m holds A[m][2c], A[m][2c+1]) is read from tensor memory.
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, bool accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"((uint32_t)accumulate)
+        : "memory");
+}
+template <bool B_MN>
+__device__ __forceinline__ void umma_product_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_saddr, uint32_t b_blk, int N,
+                                                int K, bool accumulate, bool a_neg = false) {
+    const uint32_t idesc = make_idesc(128, N, false, B_MN, a_neg);
+    const uint64_t b0 = B_MN ? desc_mnmajor(b_saddr, b_blk) : desc_kmajor(b_saddr);
+#pragma unroll
+    for (int k = 0; k < K; k += 16) {
+        const uint32_t bo = B_MN ? (uint32_t)k * 128u : (uint32_t)(k >> 6) * b_blk + (uint32_t)(k & 63) * 2u;
+        umma_ts(d_tmem, a_tmem + (uint32_t)(k >> 1), b0 + (uint64_t)(bo >> 4), idesc, accumulate || k > 0);
     }
 }
 

@@ -51,7 +51,7 @@ __global__ void __launch_bounds__(128) k_selftest(const __grid_constant__ CUtens
     __shared__ uint32_t tmem_slot;
     __shared__ int failed;
     const int tid = threadIdx.x, warp = tid >> 5;
-    const uint32_t ncols = a.N < 32 ? 32 : (uint32_t)a.N;
+    const uint32_t ncols = a.by_threads == 2 ? 256u : (a.N < 32 ? 32u : (uint32_t)a.N);
     if (tid == 0) {
         mbar_init(&bar_load, 1);
         mbar_init(&bar_mma, 1);
@@ -65,7 +65,26 @@ __global__ void __launch_bounds__(128) k_selftest(const __grid_constant__ CUtens
     const uint32_t tbase = tmem_slot;
     const uint32_t a_blk = (uint32_t)a.RA * 128u, b_blk = (uint32_t)a.RB * 128u;
 
-    if (a.by_threads) {
+    if (a.by_threads == 2) {
+        // A (row-major [128][K]) goes to tensor memory: thread = row, bf16 pairs packed per 32-bit column,
+        // columns [N, N + K/2); B to shared memory by threads
+        for (int c8 = 0; c8 < a.K / 16; ++c8) {
+            uint32_t r[8];
+            for (int j = 0; j < 8; ++j) {
+                const __nv_bfloat16 lo = a.A[(size_t)tid * a.K + c8 * 16 + 2 * j], hi = a.A[(size_t)tid * a.K + c8 * 16 + 2 * j + 1];
+                r[j] = (uint32_t)(*(const unsigned short*)&lo) | ((uint32_t)(*(const unsigned short*)&hi) << 16);
+            }
+            tmem_st8(tmem_addr(tbase, warp * 32, a.N + c8 * 8), r);
+        }
+        tmem_st_wait();
+        for (int e = tid; e < a.RB * a.CB; e += 128) {
+            const int r = e / a.CB, c = e % a.CB;
+            *(__nv_bfloat16*)(sB + (c >> 6) * b_blk + sw128_off(r, c & 63)) = a.B[e];
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+    } else if (a.by_threads) {
         for (int e = tid; e < a.RA * a.CA; e += 128) {
             const int r = e / a.CA, c = e % a.CA;
             *(__nv_bfloat16*)(sA + (c >> 6) * a_blk + sw128_off(r, c & 63)) = a.A[e];
@@ -89,7 +108,10 @@ __global__ void __launch_bounds__(128) k_selftest(const __grid_constant__ CUtens
         if (tid == 0) {
             tc_fence_after();
             const uint32_t sa = smem_u32(sA), sb = smem_u32(sB);
-            if (a.a_mn && a.b_mn) umma_product<true, true>(tbase, sa, a_blk, sb, b_blk, a.N, a.K, false);
+            if (a.by_threads == 2) {
+                if (a.b_mn) umma_product_ts<true>(tbase, tbase + a.N, sb, b_blk, a.N, a.K, false);
+                else umma_product_ts<false>(tbase, tbase + a.N, sb, b_blk, a.N, a.K, false);
+            } else if (a.a_mn && a.b_mn) umma_product<true, true>(tbase, sa, a_blk, sb, b_blk, a.N, a.K, false);
             else if (a.a_mn) umma_product<true, false>(tbase, sa, a_blk, sb, b_blk, a.N, a.K, false);
             else if (a.b_mn) umma_product<false, true>(tbase, sa, a_blk, sb, b_blk, a.N, a.K, false);
             else umma_product<false, false>(tbase, sa, a_blk, sb, b_blk, a.N, a.K, false);
@@ -137,4 +159,78 @@ extern "C" int qdelta_selftest_umma(const void* A, const void* B, float* D, int 
         return QD_ERR_CUDA;
     k_selftest<<<1, 128, smem, (cudaStream_t)stream>>>(mA, mB, a);
     return cudaGetLastError() == cudaSuccess ? QD_OK : QD_ERR_CUDA;
+}
+
+// ---- MMA issue-rate probe (timing only; operands are zeros) ------------------------------------------
+namespace qd {
+namespace {
+using namespace sm100;
+
+// `nthr` issuing threads (lane 0 of warps 0..nthr-1), each issuing `reps` products D[128 x N] += A B^T (K = 128,
+// 8 instructions, descriptors precomputed, fully unrolled) into its own accumulator.
+template <int N, bool TS>
+__global__ void __launch_bounds__(128) k_mma_rate(int nthr, int reps, long long* out) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ uint64_t bar;
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    for (int i = tid; i < (32768 + 65536) / 16; i += 128) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+    if (tid == 0) { mbar_init(&bar, (uint32_t)nthr); mbar_init_fence(); }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tb = tmem_slot;
+    if ((tid & 31) == 0 && warp < nthr) {
+        const uint32_t sa = smem_u32(smem), sb = smem_u32(smem + 32768);
+        constexpr uint32_t idesc = make_idesc(128, N, false, false);
+        const uint64_t a0 = desc_kmajor(sa), b0 = desc_kmajor(sb);
+        constexpr uint32_t b_blk = (uint32_t)N * 128u;
+        const uint32_t tA = tb + 448;
+        const uint32_t d = tb + (uint32_t)warp * (N > 64 ? 64u : (uint32_t)N);   // accumulators may overlap for N = 256: timing only
+        uint64_t ad[8], bd[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            ad[k] = a0 + (((uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u) >> 4);
+            bd[k] = b0 + (((uint32_t)(k >> 2) * b_blk + (uint32_t)(k & 3) * 32u) >> 4);
+        }
+        const long long t0 = clock64();
+#pragma unroll 1
+        for (int r = 0; r < reps; ++r) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                if (TS) umma_ts(d, tA + k * 8, bd[k], idesc, true);
+                else umma_ss(d, ad[k], bd[k], idesc, true);
+            }
+        }
+        const long long t1 = clock64();
+        umma_commit(&bar);
+        mbar_wait(&bar, 0);
+        const long long t2 = clock64();
+        if (warp == 0) { out[0] = t1 - t0; out[1] = t2 - t0; }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tb, 512);
+}
+
+}  // namespace
+}  // namespace qd
+
+// Timing probe, not part of the public header.  out[0] = cycles thread 0 needed to issue, out[1] = cycles until
+// every issuing thread's products have completed.
+extern "C" int qdelta_selftest_mma_rate(int N, int nthr, int ts, int reps, long long* out, qd_stream stream) {
+    using namespace qd;
+    if (!out || nthr < 1 || nthr > 4 || (N != 64 && N != 128 && N != 256)) return QD_ERR_INVALID_ARG;
+    const size_t smem = 32768 + 65536 + 1024;
+    auto launch = [&](auto kern) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return (int)QD_ERR_CUDA;
+        kern<<<1, 128, smem, (cudaStream_t)stream>>>(nthr, reps, out);
+        return cudaGetLastError() == cudaSuccess ? (int)QD_OK : (int)QD_ERR_CUDA;
+    };
+    if (N == 64) return ts ? launch(k_mma_rate<64, true>) : launch(k_mma_rate<64, false>);
+    if (N == 128) return ts ? launch(k_mma_rate<128, true>) : launch(k_mma_rate<128, false>);
+    return ts ? launch(k_mma_rate<256, true>) : launch(k_mma_rate<256, false>);
 }
