@@ -57,14 +57,19 @@ def path_flops_per_token_head(dk, dv, C):
 
 
 def stage_bytes_per_token_head(dk, dv, C):
-    """Compulsory HBM bytes of each kernel of the present decomposition, per token-head (bf16
-    intermediates, fp32 per-chunk states)."""
-    st = 4.0 * dk * dv / C            # one fp32 state per chunk, per token
+    """Compulsory HBM bytes of each kernel of the present decomposition, per token-head: bf16
+    intermediates stored in their consumer's operand orientation, one bf16 state per chunk."""
+    st = 2.0 * dk * dv / C            # one bf16 state per chunk, per token
+    qkv = 2 * (2 * dk + dv)
     return {
-        "prep": 2 * (2 * dk + dv) + 6 + 2 * (dk + dv) + 2 * C + 4,
-        "chain_fwd": 2 * (2 * dk + dv + dk) + 2 * C + 4 + 2 * dv + st + 2 * dv,
-        "chain_bwd": 2 * (2 * dk + dv) + 2 * dk + 2 * C + 2 * dv + 4 + st + 2 * dv + st,
-        "chunk_bwd": 2 * (2 * dk + 2 * dv) + 6 + 4 + 2 * C + 4 * dv + 2 * st + 2 * (2 * dk + dv) + 12,
+        # read q,k,v + 3 coefficients; write diag(gamma)Q, P, W~^T, U~^T, g and the inverse for backward
+        "prep": qkv + 6 + 2 * dk + 2 * C + 2 * dk + 2 * dv + 4 + 2 * C,
+        # read diag(gamma)Q, P, W~^T, U~^T, K, g; write o, entry states, Delta^T
+        "chain_fwd": 2 * dk + 2 * C + 2 * dk + 2 * dv + 2 * dk + 4 + 2 * dv + st + 2 * dv,
+        # read W~^T, dO, diag(gamma)Q, K, P, g; write dDelta^T and the exit-state gradients
+        "chain_bwd": 2 * dk + 2 * dv + 2 * dk + 2 * dk + 2 * C + 4 + 2 * dv + st,
+        # read q,k,v,dO, both per-chunk states, Delta^T, dDelta^T, inverse, P, coefficients, g; write 6 gradients
+        "chunk_bwd": qkv + 2 * dv + 2 * st + 4 * dv + 4 * C + 6 + 4 + qkv + 12,
     }
 
 
@@ -145,10 +150,9 @@ def run_ours(args, cfg):
     import torch
     from paper_2606_08804_b200 import binding as qd
     from paper_2606_08804_b200 import inputs as gen
+    from paper_2606_08804_b200 import sharding
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = sharding.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
@@ -164,7 +168,7 @@ def run_ours(args, cfg):
         torch.cuda.synchronize()
 
     # ---- inputs: pinned host copies and device copies ------------------------------------------
-    d = gen.make_chunk_inputs(cfg, seed=cfg.seed + rank)
+    d = gen.make_chunk_inputs(cfg, seed=sharding.rank_seed(cfg.seed, rank))
     bf, f32 = torch.bfloat16, torch.float32
     host, dev = {}, {}
     for n in ("q", "k", "v", "beta", "alpha", "lam", "dO"):
@@ -210,13 +214,10 @@ def run_ours(args, cfg):
     stages = qd.profile_read(reset=True)
     sampler.stop_flag.set()
     sampler.join()
-    if dist is not None:
-        tms = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-        ms = float(tms.item())
+    ms, tokens_total = sharding.aggregate(ms, B * T * args.steps, "cuda")   # slowest rank, all ranks' tokens
     ms_step = ms / args.steps
-    tokens_step = B * T * world
-    value = tokens_step / (ms_step * 1e-3)
+    tokens_step = tokens_total // args.steps
+    value = sharding.throughput(tokens_total, ms)
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ------------
     out_host = {"o": torch.empty_like(o, device="cpu").pin_memory(), "hT": torch.empty_like(hT, device="cpu").pin_memory()}
@@ -244,10 +245,7 @@ def run_ours(args, cfg):
     e1.record()
     barrier()
     ems = e0.elapsed_time(e1) if e2e_steps else float("nan")
-    if dist is not None:
-        tms = torch.tensor([ems], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tms, op=dist.ReduceOp.MAX)
-        ems = float(tms.item())
+    ems, _ = sharding.aggregate(ems, 0, "cuda")
     e2e_value = tokens_step / (ems / e2e_steps * 1e-3) if e2e_steps else None
 
     # ---- roofline of the dominant kernel and of the whole path -----------------------------------
