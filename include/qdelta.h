@@ -45,7 +45,8 @@ typedef enum {
     QD_ERR_UNSUPPORTED = 2,   /* (dk, dv, chunk, dtype) outside the supported set */
     QD_ERR_WORKSPACE = 3,     /* workspace null or smaller than qdelta_chunk_workspace_bytes */
     QD_ERR_CUDA = 4,          /* a CUDA runtime call (launch, attribute) failed */
-    QD_ERR_TIMEOUT = 5        /* device side: a bounded wait expired (see qdelta_workspace_status) */
+    QD_ERR_TIMEOUT = 5,       /* device side: a bounded wait expired (see qdelta_workspace_status) */
+    QD_ERR_STATIC_SCRATCH = 6 /* qdelta_chunk_fwd_static: the shape needs more than QDELTA_STATIC_SCRATCH_BYTES */
 } qd_status;
 
 typedef enum { QD_F32 = 0, QD_BF16 = 1 } qd_dtype;
@@ -133,6 +134,37 @@ int qdelta_profile_read(int stage, double *total_ms, long long *launches, int re
 
 /* Human-readable name of a qd_status. */
 const char *qdelta_status_string(int status);
+
+/* Size of the scratch array built into the library's device image for qdelta_chunk_fwd_static:
+ * 32 MiB, enough for B*T*H <= 32768 token-heads at d_k = d_v = 128 in bf16 (one 2048-token prompt
+ * with 16 heads). */
+#define QDELTA_STATIC_SCRATCH_BYTES ((size_t)32 << 20)
+
+/* Forward without a caller workspace and without any allocation.  The paper has no counterpart to
+ * this call: it is a deployment convenience of this library, not part of the method.
+ *
+ * Computes exactly what qdelta_chunk_fwd computes with flags = 0 (same arguments, same layouts,
+ * same kernels; o and hT as there), using a fixed scratch array of QDELTA_STATIC_SCRATCH_BYTES
+ * that is part of the library's device image instead of a workspace.  Meant for callers that cannot
+ * allocate device memory where the call is made (all HBM already handed to the caller's own pool,
+ * or an allocation's device-wide synchronisation is not acceptable there).
+ *
+ *  - Performs no cudaMalloc/cudaFree and calls no allocating library routine.  Keep the timing aid
+ *    (qdelta_profile_enable) off: it creates events.
+ *  - The first call on each device looks up the array's address (and the driver may load the
+ *    module then): make that first call, with that device current, before any stream capture.
+ *  - Every call on a device shares the one array.  Calls that overlap in time race on it; issue
+ *    them on one stream or otherwise serialise them.  The call itself clears the status word, the
+ *    only part of the array that must start at zero.
+ *  - Shapes whose forward workspace (qdelta_chunk_workspace_bytes(shape, 0)) exceeds
+ *    QDELTA_STATIC_SCRATCH_BYTES are rejected with QD_ERR_STATIC_SCRATCH before anything is enqueued.
+ *  - status_out: optional DEVICE pointer to one 32-bit word (4-byte aligned); after the kernels, the
+ *    device status word (0, or QD_ERR_TIMEOUT if a bounded wait ran out) is copied there on `stream`.
+ *  - All other pointers are device pointers with the meaning, layout and ownership documented at
+ *    qdelta_chunk_fwd; errors as there.  Not saved for backward: use qdelta_chunk_fwd for training. */
+int qdelta_chunk_fwd_static(const qd_shape *shape, const void *q, const void *k, const void *v,
+                            const void *beta, const void *alpha, const void *lambda, const float *h0,
+                            void *o, float *hT, unsigned *status_out, qd_stream stream);
 
 #ifdef __cplusplus
 }

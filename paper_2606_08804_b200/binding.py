@@ -18,7 +18,7 @@ QD_FWD_SAVE_FOR_BWD, QD_BWD_REUSE_FWD = 1, 2
 EXPORTS = ("qdelta_chunk_workspace_bytes", "qdelta_chunk_fwd", "qdelta_chunk_bwd",
            "qdelta_recurrent_step", "qdelta_workspace_status", "qdelta_status_string",
            "qdelta_profile_enable", "qdelta_profile_stage_count", "qdelta_profile_stage_name",
-           "qdelta_profile_read")
+           "qdelta_profile_read", "qdelta_chunk_fwd_static")
 
 
 class QdShape(ctypes.Structure):
@@ -49,6 +49,8 @@ def load():
     lib.qdelta_chunk_fwd.argtypes = [ctypes.POINTER(QdShape)] + [vp] * 9 + [vp, sz, u, vp]
     lib.qdelta_chunk_bwd.restype = i
     lib.qdelta_chunk_bwd.argtypes = [ctypes.POINTER(QdShape)] + [vp] * 16 + [vp, sz, u, vp]
+    lib.qdelta_chunk_fwd_static.restype = i
+    lib.qdelta_chunk_fwd_static.argtypes = [ctypes.POINTER(QdShape)] + [vp] * 9 + [vp, vp]
     lib.qdelta_recurrent_step.restype = i
     lib.qdelta_recurrent_step.argtypes = [i] * 5 + [vp] * 8 + [vp]
     lib.qdelta_workspace_status.restype = i
@@ -78,7 +80,7 @@ def profile_read(reset: bool = True) -> dict:
     for st in range(lib.qdelta_profile_stage_count()):
         ms, n = ctypes.c_double(0), ctypes.c_longlong(0)
         _check(lib.qdelta_profile_read(st, ctypes.byref(ms), ctypes.byref(n), 1 if reset else 0),
-               "qdelta_profile_read")
+               "qdelta_profile_read", "qdelta_chunk_fwd_static")
         out[lib.qdelta_profile_stage_name(st).decode()] = (ms.value, n.value)
     return out
 
@@ -160,6 +162,32 @@ def chunk_fwd(q, k, v, beta, alpha=None, lam=None, h0=None, chunk=64, save_for_b
         workspace.data_ptr(), workspace.numel(), QD_FWD_SAVE_FOR_BWD if save_for_bwd else 0, _stream())
     _check(rc, "qdelta_chunk_fwd")
     return o, hT, workspace
+
+
+def chunk_fwd_static(q, k, v, beta, alpha, lam, h0, o, hT=None, status=None, chunk=64):
+    """Forward on the library's built-in scratch array: no workspace, nothing allocated.
+
+    Every output is the caller's: `o` (required), `hT` (optional fp32 final state) and `status`
+    (optional int32/uint32 tensor of one element on the GPU that receives the device status word).
+    """
+    lib = load()
+    s = make_shape(q, v, chunk)
+    B, T, H, dk, dv, dt = s.B, s.T, s.H, s.dk, s.dv, q.dtype
+    if o is None:
+        raise QdeltaError("chunk_fwd_static: the output tensor must be supplied (this call allocates nothing)")
+    sp = None
+    if status is not None:
+        if status.numel() != 1 or status.element_size() != 4 or not status.is_cuda:
+            raise QdeltaError("chunk_fwd_static: status must be one 32-bit word on the GPU")
+        sp = status.data_ptr()
+    rc = lib.qdelta_chunk_fwd_static(
+        ctypes.byref(s), _ptr(q, dt, (B, T, H, dk), "q"), _ptr(k, dt, (B, T, H, dk), "k"),
+        _ptr(v, dt, (B, T, H, dv), "v"), _ptr(beta, dt, (B, T, H), "beta"),
+        _ptr(alpha, dt, (B, T, H), "alpha"), _ptr(lam, dt, (B, T, H), "lam"),
+        _ptr(h0, torch.float32, (B, H, dk, dv), "h0"), _ptr(o, dt, (B, T, H, dv), "o"),
+        _ptr(hT, torch.float32, (B, H, dk, dv), "hT"), sp, _stream())
+    _check(rc, "qdelta_chunk_fwd_static")
+    return o, hT
 
 
 def chunk_bwd(q, k, v, beta, alpha, lam, h0, dO, dhT=None, chunk=64, workspace=None,

@@ -269,6 +269,7 @@ const char* qdelta_status_string(int status) {
         case QD_ERR_WORKSPACE: return "QD_ERR_WORKSPACE";
         case QD_ERR_CUDA: return "QD_ERR_CUDA";
         case QD_ERR_TIMEOUT: return "QD_ERR_TIMEOUT";
+        case QD_ERR_STATIC_SCRATCH: return "QD_ERR_STATIC_SCRATCH (shape needs more than the built-in scratch array)";
         default: return "QD_ERR_UNKNOWN";
     }
 }

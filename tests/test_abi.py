@@ -42,6 +42,18 @@ def test_status_strings(lib):
     assert binding.status_string(99) == "QD_ERR_UNKNOWN"
 
 
+def test_static_forward_rejects_shapes_beyond_its_scratch(lib):
+    from paper_2606_08804_b200.binding import QdShape, status_string
+    fake = 0x1000          # never dereferenced: the size check comes first
+    big = QdShape(8, 2048, 16, 128, 128, 64, 1)
+    rc = lib.qdelta_chunk_fwd_static(ctypes.byref(big), fake, fake, fake, fake, None, None, None, fake, None, None, None)
+    assert rc == 6 and "STATIC_SCRATCH" in status_string(rc)
+    bad = QdShape(8, 2000, 16, 128, 128, 64, 1)
+    assert lib.qdelta_chunk_fwd_static(ctypes.byref(bad), fake, fake, fake, fake, None, None, None, fake, None, None, None) == 1
+    ok = QdShape(1, 2048, 16, 128, 128, 64, 1)
+    assert lib.qdelta_chunk_fwd_static(ctypes.byref(ok), fake, fake, fake, fake, None, None, None, fake, None, fake + 2, None) == 1
+
+
 def test_workspace_size_and_shape_validation(lib):
     from paper_2606_08804_b200.binding import QdShape, chunk_workspace_bytes, QdeltaError
     s = QdShape(8, 2048, 16, 128, 128, 64, 1)
