@@ -80,7 +80,7 @@ def profile_read(reset: bool = True) -> dict:
     for st in range(lib.qdelta_profile_stage_count()):
         ms, n = ctypes.c_double(0), ctypes.c_longlong(0)
         _check(lib.qdelta_profile_read(st, ctypes.byref(ms), ctypes.byref(n), 1 if reset else 0),
-               "qdelta_profile_read", "qdelta_chunk_fwd_static")
+               "qdelta_profile_read")
         out[lib.qdelta_profile_stage_name(st).decode()] = (ms.value, n.value)
     return out
 
