@@ -45,6 +45,7 @@ struct PrepParams {
     bf16 *Qg, *P, *Wt, *Ut;
     bf16* Mt;                  // optional: ((I+A)^-1)^T per chunk, [column i][row r]; kept for the backward
     unsigned* status;
+    long long* timeline;       // diagnostic builds only (QD_CTA_TIMELINE): 16 stamp slots per CTA
 };
 
 // 96 KB: Q (later X, in place) | K (later A in fp32, then the T tiles) | V.  Two CTAs fit on one SM.
@@ -62,6 +63,14 @@ __device__ __forceinline__ int at_off(int i, int r) { return i * C + ((((r >> 2)
 #define QD_PCLK(i) do { if (blockIdx.x == QD_CLK_CTA && threadIdx.x == 0) ((long long*)((char*)p.status + 64))[i] = clock64(); } while (0)
 #else
 #define QD_PCLK(i) do { } while (0)
+#endif
+// Optional per-CTA timeline (build with -DQD_CTA_TIMELINE; the workspace must be backward-sized): thread 0 of
+// every CTA writes the global nanosecond timer at four points into the (then unused) entry-state section.
+#ifdef QD_CTA_TIMELINE
+__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define QD_TL(i) do { if (threadIdx.x == 0) p.timeline[(size_t)blockIdx.x * 16 + (i)] = gtime(); } while (0)
+#else
+#define QD_TL(i) do { } while (0)
 #endif
 
 __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
@@ -84,6 +93,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     const size_t tok = (size_t)b * p.T + (size_t)pr * 128 + tid;      // row in the [B*T] view
     const size_t wtok = (size_t)bh * p.T + (size_t)pr * 128 + tid;    // row in the [BH*T] view
 
+    QD_TL(10);
     if (tid == 0) {
         mbar_init(&bar_load, 1);
         mbar_init(&bar_mma, 1);
@@ -96,6 +106,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     const uint32_t tbase = tmem_slot;
 
     QD_PCLK(0);
+    QD_TL(0);
     if (tid == 0) {
         mbar_expect_tx(&bar_load, 3 * 32768);
         const int y = (int)((size_t)b * p.T + (size_t)pr * 128);
@@ -132,6 +143,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         return;
     }
     QD_PCLK(1);
+    QD_TL(1);
     if (tid == 0) {
         tc_fence_after();
         // G2 = Q K^T -> columns [128,256)
@@ -159,6 +171,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         return;
     }
     QD_PCLK(2);
+    QD_TL(2);
     // X = K + lambda Q, in place over Q (row `tid`, K-major swizzled layout)
 #pragma unroll
     for (int blk = 0; blk < 2; ++blk)
@@ -176,6 +189,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     QD_PCLK(3);
+    QD_TL(3);
     if (tid == 0) {
         tc_fence_after();
         // G1 = X K^T -> columns [0,128)
@@ -190,6 +204,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     }
     tc_fence_after();
     QD_PCLK(4);
+    QD_TL(4);
     // A = strictLower(beta_r Gamma_ri (x_r . k_i)) -> shared fp32;  P = Gamma_ri (q_r . k_i), i <= r -> workspace
     {
         float* Ac = sA + c * C * C;
@@ -218,6 +233,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     QD_PCLK(5);
+    QD_TL(5);
     // M_c = (I + A_c)^-1: thread (c, j) solves column j by forward substitution, column in registers.
     // Rows above j come out as exact zeros, row j as one.
     float m[C];
@@ -252,6 +268,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     }
     __syncthreads();
     QD_PCLK(6);
+    QD_TL(6);
     // T_c = M_c diag(beta), T_c diag(gamma): thread (c, i) owns column i and writes line i (MN-major tile)
     {
         unsigned char* t0 = sT + c * 8192;
@@ -272,6 +289,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     QD_PCLK(7);
+    QD_TL(7);
     if (tid == 0) {
         tc_fence_after();
         for (int cc = 0; cc < 2; ++cc) {
@@ -291,6 +309,7 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     }
     tc_fence_after();
     QD_PCLK(8);
+    QD_TL(8);
     // rows `tid` (a d_v resp. d_k index) of Ut and Wt, both chunks
 #pragma unroll
     for (int which = 0; which < 2; ++which) {
@@ -307,9 +326,11 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         }
     }
     QD_PCLK(9);
+    QD_TL(9);
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tbase, 256);
+    QD_TL(11);
 }
 
 // =================================================================================================
@@ -659,6 +680,9 @@ cudaError_t tc_prep(const ChunkArgs& a) {
     p.Wt = (bf16*)(a.ws + a.TL.Wt); p.Ut = (bf16*)(a.ws + a.TL.Ut);
     p.Mt = a.save ? (bf16*)(a.ws + a.TL.Mt) : nullptr;
     p.status = (unsigned*)(a.ws + a.TL.status);
+#ifdef QD_CTA_TIMELINE
+    p.timeline = (long long*)(a.ws + a.TL.hsT);
+#endif
     cudaError_t e = set_smem(k_tc_prep, kPrepSmem);
     if (e != cudaSuccess) return e;
     const int grid = s.B * s.H * (p.N / 2);
