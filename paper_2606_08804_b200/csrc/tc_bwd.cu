@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
 
 // =================================================================================================
 struct ChunkBwdParams {
-    int T, H, N;
+    int T, H, N, total;        // total = B*H*N chunks
     const bf16 *beta, *alpha, *lam;
     const float* g;
     float *dbeta, *dalpha, *dlam;
@@ -289,7 +289,8 @@ struct ChunkBwdParams {
 
 // shared-memory map of k_tc_chunk_bwd (bytes from the 1024-aligned base)
 constexpr int oQ = 0, oK = 16384, oV = 32768, odO = 49152, oX = 65536, oMt = 81920, oP = 90112, oDt = 98304,
-              odDt = 114688, oH = 131072, odH = 163840, kBwdLoadBytes = 180224;   // all TMA-loaded tiles (X is built)
+              odDt = 114688, oH = 131072, odH = 163840;                            // TMA-loaded tiles (X is built)
+constexpr int kBwdEarlyBytes = 3 * 16384 + 2 * 8192, kBwdLateBytes = 16384 + 2 * 16384 + 2 * 32768;
 // tiles built later reuse regions whose contents are dead by then
 constexpr int odPG = oV, odTb = oV + 8192, odW = odO, oN = oH, odXK = oH + 8192, oPP = oH + 16384,
               oAA = odH + 1024, oStDv = odDt, oStDk = oDt, oStDq = odDt;
@@ -299,10 +300,10 @@ constexpr int kNWG = 4;                       // warpgroups; each owns 64/kNWG c
 constexpr int kCW = C / kNWG, kG8 = kCW / 8;    // columns per warpgroup, groups of 8 columns
 constexpr int kBwdThreads = 128 * kNWG;
 
-// Optional phase timestamps (build with -DQD_PHASE_CLOCKS -DQD_CLK_CTA=<block>): thread 0 of that CTA
+// Optional phase timestamps (build with -DQD_PHASE_CLOCKS -DQD_CLK_CTA=<chunk>): thread 0 of the CTA that owns that chunk
 // writes clock64() values into bytes 64.. of the workspace status section.
 #ifdef QD_PHASE_CLOCKS
-#define QD_CLK(i) do { if (blockIdx.x == QD_CLK_CTA && threadIdx.x == 0) ((long long*)((char*)p.status + 64))[i] = clock64(); } while (0)
+#define QD_CLK(i) do { if (ch_id == QD_CLK_CTA && threadIdx.x == 0) ((long long*)((char*)p.status + 64))[i] = clock64(); } while (0)
 #else
 #define QD_CLK(i) do { } while (0)
 #endif
@@ -351,7 +352,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                                                               ChunkBwdParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ uint64_t bar_load, bar_mma;
+    __shared__ uint64_t bar_load, bar_late, bar_mma;
     __shared__ uint32_t tmem_slot;
     __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C], segc[C];
     __shared__ float sred[3][4][C];   // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
@@ -360,12 +361,10 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
 
     const int tid = threadIdx.x, wg = tid >> 7, l = tid & 127, lane = tid & 31, wq = (tid >> 5) & 3;
     const int c0 = wg * kCW;                                      // my columns of a 64-column accumulator
-    const int ch_id = blockIdx.x, n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
-    const size_t row0 = (size_t)b * p.T + (size_t)n * C;          // token row in the [B*T] view
-    const size_t wrow0 = (size_t)bh * p.T + (size_t)n * C;        // token row in the [BH*T] view
 
     if (tid == 0) {
         mbar_init(&bar_load, 1);
+        mbar_init(&bar_late, 1);
         mbar_init(&bar_mma, 1);
         mbar_init_fence();
     }
@@ -379,40 +378,75 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     const uint32_t lane_base = (uint32_t)wq * 32;
     auto my = [&](uint32_t t) { return tmem_addr(t, lane_base, (uint32_t)c0); };
 
-    QD_CLK(0);
-    if (tid == 0) {
-        mbar_expect_tx(&bar_load, kBwdLoadBytes);
-        const int yi = (int)row0, yt = (int)wrow0;
-        const int yc = (int)(((size_t)bh * p.N + n) * D), ym = (int)(((size_t)bh * p.N + n) * C);
+    // The tiles of a chunk arrive in two groups.  "early": K, V, dO, M^T, P -- their regions are dead once the
+    // last products of the previous chunk have finished; "late": Q, Delta^T, dDelta^T, h^T, dh^T -- regions
+    // that the previous chunk uses up to its end (staging tiles of the stores, scratch of the reductions).
+    auto issue_early = [&](int ch) {
+        const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
+        const int yi = (int)((size_t)b_ * p.T + (size_t)n_ * C), yt = (int)((size_t)bh_ * p.T + (size_t)n_ * C);
+        const int ym = (int)(((size_t)bh_ * p.N + n_) * C);
+        mbar_expect_tx(&bar_load, kBwdEarlyBytes);
         for (int blk = 0; blk < 2; ++blk) {
-            tma_load_2d(sm + oQ + blk * 8192, &mapQ, hh * D + blk * 64, yi, &bar_load);
-            tma_load_2d(sm + oK + blk * 8192, &mapK, hh * D + blk * 64, yi, &bar_load);
-            tma_load_2d(sm + oV + blk * 8192, &mapV, hh * D + blk * 64, yi, &bar_load);
-            tma_load_2d(sm + odO + blk * 8192, &mapdO, hh * D + blk * 64, yi, &bar_load);
-            tma_load_2d(sm + oH + blk * 16384, &mapHs, blk * 64, yc, &bar_load);
-            tma_load_2d(sm + odH + blk * 16384, &mapdHs, blk * 64, yc, &bar_load);
+            tma_load_2d(sm + oK + blk * 8192, &mapK, hh_ * D + blk * 64, yi, &bar_load);
+            tma_load_2d(sm + oV + blk * 8192, &mapV, hh_ * D + blk * 64, yi, &bar_load);
+            tma_load_2d(sm + odO + blk * 8192, &mapdO, hh_ * D + blk * 64, yi, &bar_load);
         }
         tma_load_2d(sm + oMt, &mapMt, 0, ym, &bar_load);
         tma_load_2d(sm + oP, &mapP, 0, yt, &bar_load);
-        tma_load_2d(sm + oDt, &mapDt, 0, yc, &bar_load);
-        tma_load_2d(sm + odDt, &mapdDt, 0, yc, &bar_load);
+    };
+    auto issue_late = [&](int ch) {
+        const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
+        const int yi = (int)((size_t)b_ * p.T + (size_t)n_ * C);
+        const int yc = (int)(((size_t)bh_ * p.N + n_) * D);
+        mbar_expect_tx(&bar_late, kBwdLateBytes);
+        for (int blk = 0; blk < 2; ++blk) {
+            tma_load_2d(sm + oQ + blk * 8192, &mapQ, hh_ * D + blk * 64, yi, &bar_late);
+            tma_load_2d(sm + oH + blk * 16384, &mapHs, blk * 64, yc, &bar_late);
+            tma_load_2d(sm + odH + blk * 16384, &mapdHs, blk * 64, yc, &bar_late);
+        }
+        tma_load_2d(sm + oDt, &mapDt, 0, yc, &bar_late);
+        tma_load_2d(sm + odDt, &mapdDt, 0, yc, &bar_late);
+    };
+    // coefficients of token tid (< C) of a chunk, fetched one chunk ahead into registers
+    float cf_beta = 0.f, cf_lam = 0.f, cf_alpha = 1.f, cf_g = 0.f;
+    auto fetch_coef = [&](int ch) {
+        if (tid < C) {
+            const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
+            const size_t cr = ((size_t)b_ * p.T + (size_t)n_ * C + tid) * p.H + hh_;
+            cf_beta = __bfloat162float(p.beta[cr]);
+            cf_lam = p.lam ? __bfloat162float(p.lam[cr]) : 0.f;
+            cf_alpha = p.alpha ? __bfloat162float(p.alpha[cr]) : 1.f;
+            cf_g = p.g[(size_t)bh_ * p.T + (size_t)n_ * C + tid];
+        }
+    };
+    if ((int)blockIdx.x < p.total) {
+        if (tid == 0) { issue_early(blockIdx.x); issue_late(blockIdx.x); }
+        fetch_coef(blockIdx.x);
     }
+    uint32_t mma_ph = 0;                                          // parity of the next completion of bar_mma
+
+    for (int ch_id = blockIdx.x, it = 0; ch_id < p.total; ch_id += gridDim.x, ++it) {
+    const int n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
+    const size_t row0 = (size_t)b * p.T + (size_t)n * C;          // token row in the [B*T] view
+    const int next_id = ch_id + gridDim.x;
+
+    QD_CLK(0);
     if (tid < C) {
-        const size_t cr = (row0 + tid) * p.H + hh;
-        sbeta[tid] = __bfloat162float(p.beta[cr]);
-        slam[tid] = p.lam ? __bfloat162float(p.lam[cr]) : 0.f;
-        salpha[tid] = p.alpha ? __bfloat162float(p.alpha[cr]) : 1.f;
-        const float gv = p.g[wrow0 + tid];
-        sg[tid] = gv;
-        sgam[tid] = __expf(gv);
+        sbeta[tid] = cf_beta;
+        slam[tid] = cf_lam;
+        salpha[tid] = cf_alpha;
+        sg[tid] = cf_g;
+        sgam[tid] = __expf(cf_g);
     }
     __syncthreads();
     if (tid < C) segc[tid] = __expf(sg[C - 1] - sg[tid]);
 
-    bool fail = !mbar_wait(&bar_load, 0);
+    bool fail = !mbar_wait(&bar_load, it & 1);
+    fail = fail || !mbar_wait(&bar_late, it & 1);
     if (__syncthreads_or(fail)) {
         if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        mbar_wait(&bar_load, 0);
+        mbar_wait(&bar_load, it & 1);
+        mbar_wait(&bar_late, it & 1);
         __syncthreads();
         if (tid < 32) tmem_dealloc(tb, 512);
         return;
@@ -468,7 +502,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         umma_product<false, false>(T7, adH, 16384, aK, 8192, C, D, false);          // dh^T K^T         [j][s]
         umma_commit(&bar_mma);
     }
-    fail = !mbar_wait(&bar_mma, 0);
+    fail = !mbar_wait(&bar_mma, mma_ph);
+    mma_ph ^= 1;
     if (__syncthreads_or(fail)) {
         if (tid == 0) *p.status = QD_ERR_TIMEOUT;
         if (tid < 32) tmem_dealloc(tb, 512);
@@ -538,7 +573,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         umma_product<false, false>(T6, adW, 16384, aMt, 8192, C, C, false);         // dW<-^T M         [i][s]
         umma_commit(&bar_mma);
     }
-    fail = !mbar_wait(&bar_mma, 1);
+    fail = !mbar_wait(&bar_mma, mma_ph);
+    mma_ph ^= 1;
     if (__syncthreads_or(fail)) {
         if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
         if (tid < 32) tmem_dealloc(tb, 512);
@@ -581,7 +617,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         umma_product<true, true>(T1, adTb, 8192, aMt, 8192, C, C, false);           // [r][u]
         umma_commit(&bar_mma);
     }
-    fail = !mbar_wait(&bar_mma, 0);
+    fail = !mbar_wait(&bar_mma, mma_ph);
+    mma_ph ^= 1;
     if (__syncthreads_or(fail)) {
         if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
         if (tid < 32) tmem_dealloc(tb, 512);
@@ -607,7 +644,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         umma_product<false, true>(T2, aMt, 8192, aN, 8192, C, C, false, true);      // [r][s]
         umma_commit(&bar_mma);
     }
-    fail = !mbar_wait(&bar_mma, 1);
+    fail = !mbar_wait(&bar_mma, mma_ph);
+    mma_ph ^= 1;
     if (__syncthreads_or(fail)) {
         if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
         if (tid < 32) tmem_dealloc(tb, 512);
@@ -659,7 +697,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         umma_commit(&bar_mma);
         tma_store_wait_read();                                      // the dv staging tile may be reused now
     }
-    fail = !mbar_wait(&bar_mma, 0);
+    fail = !mbar_wait(&bar_mma, mma_ph);
+    mma_ph ^= 1;
     if (__syncthreads_or(fail)) {
         if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
         if (tid < 32) tmem_dealloc(tb, 512);
@@ -667,6 +706,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     }
     tc_fence_after();
     QD_CLK(11);
+    if (next_id < p.total) {
+        // K, V, dO, M^T, P of this chunk are dead: fetch the next chunk's, and its coefficients
+        if (tid == 0) issue_early(next_id);
+        fetch_coef(next_id);
+    }
     {
         const int i = l;                                            // d_k index; my 32 tokens c0..c0+31 in groups of 8
         unsigned char* stk = sm + oStDk + (i >> 6) * 8192;
@@ -709,6 +753,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 1);
     if (lane == 0) swp[tid >> 5] = dhh_part;
     fence_proxy_async();
+    tc_fence_before();
     __syncthreads();
     if (tid == 0) {
         tma_store_2d(&mapdK, sm + oStDk, hh * D, (int)row0);
@@ -774,8 +819,15 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         }
     }
     QD_CLK(13);
-    if (tid == 0) tma_store_wait_all();
+    __syncthreads();                     // every read of this chunk's tiles and scratch is done
+    if (tid == 0) {
+        tma_store_wait_read();           // the staging tiles have been read by the stores
+        fence_proxy_async();
+        if (next_id < p.total) issue_late(next_id);
+    }
     QD_CLK(14);
+    }  // chunk loop
+    if (tid == 0) tma_store_wait_all();
     tc_fence_before();
     __syncthreads();
     if (tid < 32) tmem_dealloc(tb, 512);
@@ -832,14 +884,19 @@ cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
         !make_tmap_bf16_2d(&mdHs, a.ws + a.TL.dhsT, D, BH * N * D, D * 2, 128))
         return cudaErrorInvalidValue;
     ChunkBwdParams p{};
-    p.T = s.T; p.H = s.H; p.N = (int)N;
+    p.T = s.T; p.H = s.H; p.N = (int)N; p.total = (int)(BH * N);
     p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
     p.g = (const float*)(a.ws + a.TL.g);
     p.dbeta = a.dbeta; p.dalpha = a.dalpha; p.dlam = a.dlam;
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_chunk_bwd, kBwdSmem);
     if (e != cudaSuccess) return e;
-    k_tc_chunk_bwd<<<(unsigned)(BH * N), kBwdThreads, kBwdSmem, a.stream>>>(mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs,
+    // persistent: one CTA per SM walks the chunks with stride gridDim.x
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const unsigned grid = (unsigned)std::min<uint64_t>(BH * N, (uint64_t)sms);
+    k_tc_chunk_bwd<<<grid, kBwdThreads, kBwdSmem, a.stream>>>(mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs,
                                                                                mdQ, mdK, mdV, p);
     return cudaGetLastError();
 }

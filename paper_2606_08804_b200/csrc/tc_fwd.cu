@@ -23,7 +23,6 @@ typedef __nv_bfloat16 bf16;
 
 constexpr int C = kChunk;      // 64
 constexpr int D = 128;         // d_k = d_v
-constexpr int LDA = C + 1;
 
 __device__ __forceinline__ void load8(const unsigned char* p, float* f) {
     const uint4 u = *reinterpret_cast<const uint4*>(p);
@@ -42,30 +41,19 @@ struct PrepParams {
     int T, H, N;
     const bf16 *beta, *alpha, *lam;
     float* g;
-    bf16 *Qg, *P, *Wt, *Ut;
+    bf16 *Qg, *P;
     bf16* Mt;                  // optional: ((I+A)^-1)^T per chunk, [column i][row r]; kept for the backward
     unsigned* status;
     long long* timeline;       // diagnostic builds only (QD_CTA_TIMELINE): 16 stamp slots per CTA
 };
 
-// 96 KB: Q (later X, in place) | K (later A in fp32, then the T tiles) | V.  Two CTAs fit on one SM.
+// 96 KB: Q (later X, in place) | K (later A in fp32, then the T tiles) | V; at the end the first and the
+// last 32 KB stage U~^T and W~^T for their TMA stores.  Two CTAs fit on one SM.
 constexpr int kPrepSmem = 3 * 32768 + 1024;
+constexpr int kPrepThreads = 256;
 
-// A (fp32, 64 x 64 per chunk) is kept unpadded; 16-byte groups of a row are XOR-swizzled with the
-// row index so that row-wise 16-byte stores by 32 different rows do not collide on banks.
-// A (fp32, 64 x 64 per chunk) is kept transposed and unpadded: element (column i, row r) of A^T at
-// i*64 + r, with the 16-byte group index of r XOR-ed with (i & 15) so that reading one column as
-// float4 and writing one row element-wise are both free of bank conflicts.
-__device__ __forceinline__ int at_off(int i, int r) { return i * C + ((((r >> 2) ^ i) & 15) << 2) + (r & 3); }
-
-// Optional phase timestamps (build with -DQD_PHASE_CLOCKS): CTA 0, thread 0 -> bytes 64.. of the status section.
-#ifdef QD_PHASE_CLOCKS
-#define QD_PCLK(i) do { if (blockIdx.x == QD_CLK_CTA && threadIdx.x == 0) ((long long*)((char*)p.status + 64))[i] = clock64(); } while (0)
-#else
-#define QD_PCLK(i) do { } while (0)
-#endif
 // Optional per-CTA timeline (build with -DQD_CTA_TIMELINE; the workspace must be backward-sized): thread 0 of
-// every CTA writes the global nanosecond timer at four points into the (then unused) entry-state section.
+// every CTA writes the global nanosecond timer at each phase boundary into the (then unused) entry-state section.
 #ifdef QD_CTA_TIMELINE
 __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 #define QD_TL(i) do { if (threadIdx.x == 0) p.timeline[(size_t)blockIdx.x * 16 + (i)] = gtime(); } while (0)
@@ -73,25 +61,32 @@ __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u6
 #define QD_TL(i) do { } while (0)
 #endif
 
-__global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
-                                                    const __grid_constant__ CUtensorMap mapK,
-                                                    const __grid_constant__ CUtensorMap mapV, PrepParams p) {
+// One CTA prepares a pair of chunks (128 tokens) of one head.  Thread roles change by phase:
+//   scan / coefficients   thread t < 128 owns token t
+//   row-wise elementwise  16 threads per 256-byte row (coalesced), 16 rows per pass
+//   Gram epilogue         thread (row = t & 127, half = t >> 7) owns 32 columns of its TMEM lane
+//   triangular inverse    thread (column = t >> 1, parity = t & 1) owns the 8-row blocks of that parity
+//   final epilogue        thread (d = t & 127, which = t >> 7) owns one row of U~^T resp. W~^T
+__global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
+                                                             const __grid_constant__ CUtensorMap mapK,
+                                                             const __grid_constant__ CUtensorMap mapV,
+                                                             const __grid_constant__ CUtensorMap mapUt,
+                                                             const __grid_constant__ CUtensorMap mapWt, PrepParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char *sQ = smem, *sK = smem + 32768, *sV = smem + 65536;
     unsigned char* sX = sQ;                                     // X overwrites Q once Q K^T has been formed
-    float* sA = reinterpret_cast<float*>(sK);                   // [2][64][64], aliases K once both Grams are read
+    float* sA = reinterpret_cast<float*>(sK);                   // A^T [2][column i][row r], aliases K once both Grams are read
     unsigned char* sT = sK;                                     // [2] T_c, [2] T_c diag(gamma): 8 KB each, alias A
     __shared__ uint64_t bar_load, bar_mma;
     __shared__ uint32_t tmem_slot;
-    __shared__ float sg[128], swsum[4];
+    __shared__ float sg[128], sbeta[128], slam[128], swsum[4];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int c = tid >> 6, r = tid & 63;
     const int pairs = p.N / 2, bh = blockIdx.x / pairs, pr = blockIdx.x % pairs;
     const int b = bh / p.H, hh = bh % p.H;
-    const size_t tok = (size_t)b * p.T + (size_t)pr * 128 + tid;      // row in the [B*T] view
-    const size_t wtok = (size_t)bh * p.T + (size_t)pr * 128 + tid;    // row in the [BH*T] view
+    const size_t tok0 = (size_t)b * p.T + (size_t)pr * 128;          // first row in the [B*T] view
+    const size_t wtok0 = (size_t)bh * p.T + (size_t)pr * 128;        // first row in the [BH*T] view
 
     QD_TL(10);
     if (tid == 0) {
@@ -105,34 +100,34 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
     tc_fence_after();
     const uint32_t tbase = tmem_slot;
 
-    QD_PCLK(0);
     QD_TL(0);
     if (tid == 0) {
         mbar_expect_tx(&bar_load, 3 * 32768);
-        const int y = (int)((size_t)b * p.T + (size_t)pr * 128);
+        const int y = (int)tok0;
         for (int blk = 0; blk < 2; ++blk) {
             tma_load_2d(sQ + blk * 16384, &mapQ, hh * D + blk * 64, y, &bar_load);
             tma_load_2d(sK + blk * 16384, &mapK, hh * D + blk * 64, y, &bar_load);
             tma_load_2d(sV + blk * 16384, &mapV, hh * D + blk * 64, y, &bar_load);
         }
     }
-    // coefficients of my token; in-chunk cumulative log-decay by a two-warp scan
-    const size_t crow = tok * p.H + hh;
-    const float beta = __bfloat162float(p.beta[crow]);
-    const float lam = p.lam ? __bfloat162float(p.lam[crow]) : 0.f;
-    const float alpha = p.alpha ? __bfloat162float(p.alpha[crow]) : 1.f;
-    float g = logf(alpha);
+    // coefficients of token tid; in-chunk cumulative log-decay by a two-warp scan per chunk
+    if (tid < 128) {
+        const size_t crow = (tok0 + tid) * p.H + hh;
+        sbeta[tid] = __bfloat162float(p.beta[crow]);
+        slam[tid] = p.lam ? __bfloat162float(p.lam[crow]) : 0.f;
+        const float alpha = p.alpha ? __bfloat162float(p.alpha[crow]) : 1.f;
+        float g = logf(alpha);
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const float t = __shfl_up_sync(0xffffffffu, g, o);
-        if (lane >= o) g += t;
+        for (int o = 1; o < 32; o <<= 1) {
+            const float t = __shfl_up_sync(0xffffffffu, g, o);
+            if (lane >= o) g += t;
+        }
+        if (lane == 31) swsum[warp] = g;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (warp & 1) g += swsum[warp - 1];
+        sg[tid] = g;
+        p.g[wtok0 + tid] = g;
     }
-    if (lane == 31) swsum[warp] = g;
-    __syncthreads();
-    if (warp & 1) g += swsum[warp - 1];
-    sg[tid] = g;
-    p.g[wtok] = g;
-    const float gam = __expf(g);
 
     bool fail = !mbar_wait(&bar_load, 0);
     if (__syncthreads_or(fail)) {
@@ -142,7 +137,6 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         if (warp == 0) tmem_dealloc(tbase, 256);
         return;
     }
-    QD_PCLK(1);
     QD_TL(1);
     if (tid == 0) {
         tc_fence_after();
@@ -150,19 +144,22 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         umma_product<false, false>(tbase + 128, smem_u32(sQ), 16384, smem_u32(sK), 16384, 128, 128, false);
         umma_commit(&bar_mma);
     }
-    // meanwhile: Qg = gamma Q to the workspace (row `tid`)
+    // row-wise work: 16 lanes cover one 256-byte row (chunk `ch` of 16 bytes each), 16 rows per pass
+    const int ch = tid & 15, rsub = tid >> 4;
+    const uint32_t coff = (ch >> 3) * 16384;
+    // meanwhile: Qg = gamma Q to the workspace, a warp writes two full rows per store
     {
-        bf16* qg = p.Qg + wtok * D;
+        bf16* qg = p.Qg + wtok0 * D + ch * 8;
+#pragma unroll 4
+        for (int it = 0; it < 8; ++it) {
+            const int row = it * 16 + rsub;
+            const float gr = __expf(sg[row]);
+            float qv[8];
+            load8(sQ + coff + sw128_chunk(row, ch & 7), qv);
 #pragma unroll
-        for (int blk = 0; blk < 2; ++blk)
-#pragma unroll
-            for (int ch = 0; ch < 8; ++ch) {
-                float qv[8];
-                load8(sQ + blk * 16384 + sw128_chunk(tid, ch), qv);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) qv[e] *= gam;
-                *reinterpret_cast<uint4*>(qg + blk * 64 + ch * 8) = pack8(qv);
-            }
+            for (int e = 0; e < 8; ++e) qv[e] *= gr;
+            *reinterpret_cast<uint4*>(qg + (size_t)row * D) = pack8(qv);
+        }
     }
     fail = !mbar_wait(&bar_mma, 0);
     if (__syncthreads_or(fail)) {
@@ -170,25 +167,23 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         if (warp == 0) tmem_dealloc(tbase, 256);
         return;
     }
-    QD_PCLK(2);
     QD_TL(2);
-    // X = K + lambda Q, in place over Q (row `tid`, K-major swizzled layout)
+    // X = K + lambda Q, in place over Q (K-major swizzled layout)
+#pragma unroll 4
+    for (int it = 0; it < 8; ++it) {
+        const int row = it * 16 + rsub;
+        const uint32_t off = coff + sw128_chunk(row, ch & 7);
+        const float lm = slam[row];
+        float qv[8], kv[8];
+        load8(sQ + off, qv);
+        load8(sK + off, kv);
 #pragma unroll
-    for (int blk = 0; blk < 2; ++blk)
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-            const uint32_t off = blk * 16384 + sw128_chunk(tid, ch);
-            float qv[8], kv[8];
-            load8(sQ + off, qv);
-            load8(sK + off, kv);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) kv[e] = fmaf(lam, qv[e], kv[e]);
-            sts128(sX + off, pack8(kv));
-        }
+        for (int e = 0; e < 8; ++e) kv[e] = fmaf(lm, qv[e], kv[e]);
+        sts128(sX + off, pack8(kv));
+    }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    QD_PCLK(3);
     QD_TL(3);
     if (tid == 0) {
         tc_fence_after();
@@ -203,92 +198,82 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         return;
     }
     tc_fence_after();
-    QD_PCLK(4);
     QD_TL(4);
-    // A = strictLower(beta_r Gamma_ri (x_r . k_i)) -> shared fp32;  P = Gamma_ri (q_r . k_i), i <= r -> workspace
+    // A = strictLower(beta_r Gamma_ri (x_r . k_i)) -> shared fp32, transposed;  P = Gamma_ri (q_r . k_i), i <= r -> workspace
     {
-        float* Ac = sA + c * C * C;
-        bf16* prow = p.P + wtok * C;
+        const int row = tid & 127, half = tid >> 7, c = row >> 6, r = row & 63;
+        const float g = sg[row], beta = sbeta[row];
         const float* gc = sg + c * C;
+        float* Ac = sA + c * C * C;
+        float v1[32], v2[32];
+        tmem_ld32(tmem_addr(tbase, (warp & 3) * 32, c * C + half * 32), v1);
+        tmem_ld32(tmem_addr(tbase, (warp & 3) * 32, 128 + c * C + half * 32), v2);
+        tmem_ld_wait();
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            float v1[32], v2[32];
-            tmem_ld32(tmem_addr(tbase, warp * 32, c * C + half * 32), v1);
-            tmem_ld32(tmem_addr(tbase, warp * 32, 128 + c * C + half * 32), v2);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const int col = half * 32 + i;
-                const float dec = (col <= r) ? __expf(g - gc[col]) : 0.f;
-                v1[i] = (col < r) ? beta * dec * v1[i] : 0.f;
-                v2[i] = dec * v2[i];
-            }
-            // A^T: entry (column i, row r) so that a column of A is contiguous over r
-#pragma unroll
-            for (int i = 0; i < 32; ++i) Ac[at_off(half * 32 + i, r)] = v1[i];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(prow + half * 32 + i * 8) = pack8(v2 + i * 8);
+        for (int i = 0; i < 32; ++i) {
+            const int col = half * 32 + i;
+            const float dec = (col <= r) ? __expf(g - gc[col]) : 0.f;
+            v1[i] = (col < r) ? beta * dec * v1[i] : 0.f;
+            v2[i] = dec * v2[i];
         }
+        // A^T: entry (column i, row r) at i*64 + r, so that 8 consecutive rows of one column are contiguous
+#pragma unroll
+        for (int i = 0; i < 32; ++i) Ac[(half * 32 + i) * C + r] = v1[i];
+        bf16* prow = p.P + (wtok0 + row) * C + half * 32;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(prow + i * 8) = pack8(v2 + i * 8);
     }
     tc_fence_before();
     __syncthreads();
-    QD_PCLK(5);
     QD_TL(5);
-    // M_c = (I + A_c)^-1: thread (c, j) solves column j by forward substitution, column in registers.
-    // Rows above j come out as exact zeros, row j as one.
-    float m[C];
+    // M_c = (I + A_c)^-1 by right-looking substitution, one column per thread pair, the column in registers:
+    // the thread of parity `par` owns the 8-row blocks 2s + par (s = 0..3).  Once m[i] is final its owner
+    // hands it to the partner lane and every later row gets its update m[r] -= A[r][i] m[i]; rows <= i of a
+    // block see A = 0 exactly.  Rows above the column index come out as exact zeros, the diagonal as one.
+    const int colid = tid >> 1, par = tid & 1, ic = colid >> 6, ij = colid & 63;
+    float m[4][8];
     {
-        // right-looking substitution: once m[i] is final, every later row gets its update
-        // m[r] -= A[r][i] m[i]; the updates of one step are independent of each other, and the
-        // loads of A do not depend on the recurrence.
-        const float* Ac = sA + c * C * C;
-        const int j = r;
-#ifdef QD_REP
-#pragma unroll 1
-        for (int rep = 0; rep < QD_REP; ++rep) {
-#endif
+        const float* Ac = sA + ic * C * C + par * 8;
 #pragma unroll
-        for (int rr = 0; rr < C; ++rr) m[rr] = (rr == j) ? 1.f : 0.f;
+        for (int s = 0; s < 4; ++s)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) m[s][e] = ((2 * s + par) * 8 + e == ij) ? 1.f : 0.f;
 #pragma unroll
         for (int i = 0; i < C - 1; ++i) {
-            const float mi = m[i];
+            const float mi = __shfl_sync(0xffffffffu, m[i >> 4][i & 7], (lane & ~1) | ((i >> 3) & 1));
 #pragma unroll
-            for (int q4 = (i + 1) / 4; q4 < C / 4; ++q4) {
-                const float4 av = *reinterpret_cast<const float4*>(Ac + i * C + (((q4 ^ i) & 15) << 2));
-                // rows 4*q4 .. 4*q4+3; entries with row <= i are zero (A is strictly lower)
-                m[q4 * 4] = fmaf(-av.x, mi, m[q4 * 4]);
-                m[q4 * 4 + 1] = fmaf(-av.y, mi, m[q4 * 4 + 1]);
-                m[q4 * 4 + 2] = fmaf(-av.z, mi, m[q4 * 4 + 2]);
-                m[q4 * 4 + 3] = fmaf(-av.w, mi, m[q4 * 4 + 3]);
+            for (int s = (i + 1) >> 4; s < 4; ++s) {
+                const float4 a0 = *reinterpret_cast<const float4*>(Ac + i * C + s * 16);
+                const float4 a1 = *reinterpret_cast<const float4*>(Ac + i * C + s * 16 + 4);
+                m[s][0] = fmaf(-a0.x, mi, m[s][0]); m[s][1] = fmaf(-a0.y, mi, m[s][1]);
+                m[s][2] = fmaf(-a0.z, mi, m[s][2]); m[s][3] = fmaf(-a0.w, mi, m[s][3]);
+                m[s][4] = fmaf(-a1.x, mi, m[s][4]); m[s][5] = fmaf(-a1.y, mi, m[s][5]);
+                m[s][6] = fmaf(-a1.z, mi, m[s][6]); m[s][7] = fmaf(-a1.w, mi, m[s][7]);
             }
         }
-#ifdef QD_REP
-        }
-#endif
     }
     __syncthreads();
-    QD_PCLK(6);
     QD_TL(6);
-    // T_c = M_c diag(beta), T_c diag(gamma): thread (c, i) owns column i and writes line i (MN-major tile)
+    // T_c = M_c diag(beta), T_c diag(gamma): line j of the MN-major tiles holds column j over the rows
     {
-        unsigned char* t0 = sT + c * 8192;
-        unsigned char* t1 = sT + 16384 + c * 8192;
-        bf16* mt = p.Mt ? p.Mt + (((size_t)bh * p.N + 2 * pr + c) * C + r) * C : nullptr;
-        const float bg = beta * gam;
+        unsigned char* t0 = sT + ic * 8192;
+        unsigned char* t1 = sT + 16384 + ic * 8192;
+        bf16* mt = p.Mt ? p.Mt + (((size_t)bh * p.N + 2 * pr + ic) * C + ij) * C : nullptr;
+        const float beta = sbeta[colid], bg = beta * __expf(sg[colid]);
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
+        for (int s = 0; s < 4; ++s) {
+            const int kb = 2 * s + par;
             float a[8], bq[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) { a[e] = m[ch * 8 + e] * beta; bq[e] = m[ch * 8 + e] * bg; }
-            sts128(t0 + sw128_chunk(r, ch), pack8(a));
-            sts128(t1 + sw128_chunk(r, ch), pack8(bq));
-            if (mt) *reinterpret_cast<uint4*>(mt + ch * 8) = pack8(m + ch * 8);
+            for (int e = 0; e < 8; ++e) { a[e] = m[s][e] * beta; bq[e] = m[s][e] * bg; }
+            sts128(t0 + sw128_chunk(ij, kb), pack8(a));
+            sts128(t1 + sw128_chunk(ij, kb), pack8(bq));
+            if (mt) *reinterpret_cast<uint4*>(mt + kb * 8) = pack8(m[s]);
         }
     }
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    QD_PCLK(7);
     QD_TL(7);
     if (tid == 0) {
         tc_fence_after();
@@ -308,28 +293,39 @@ __global__ void __launch_bounds__(128, 2) k_tc_prep(const __grid_constant__ CUte
         return;
     }
     tc_fence_after();
-    QD_PCLK(8);
     QD_TL(8);
-    // rows `tid` (a d_v resp. d_k index) of Ut and Wt, both chunks
-#pragma unroll
-    for (int which = 0; which < 2; ++which) {
-        bf16* dst = which ? p.Wt : p.Ut;
+    // row d = tid & 127 of U~^T (threads < 128) resp. W~^T (the others), both chunks: staged as swizzled
+    // [128][64] tiles over the dead Q/X and V regions, then written by TMA
+    {
+        const int d = tid & 127, which = tid >> 7;
+        unsigned char* stage = which ? sV : sQ;
 #pragma unroll
         for (int q4 = 0; q4 < 4; ++q4) {
             float v[32];
-            tmem_ld32(tmem_addr(tbase, warp * 32, which * 128 + q4 * 32), v);
+            tmem_ld32(tmem_addr(tbase, (warp & 3) * 32, which * 128 + q4 * 32), v);
             tmem_ld_wait();
-            const int cc = q4 >> 1;
-            bf16* row = dst + (((size_t)bh * p.N + 2 * pr + cc) * D + tid) * C + (q4 & 1) * 32;
+            unsigned char* tile = stage + (q4 >> 1) * 16384;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) *reinterpret_cast<uint4*>(row + i * 8) = pack8(v + i * 8);
+            for (int i = 0; i < 4; ++i) sts128(tile + sw128_chunk(d, (q4 & 1) * 4 + i), pack8(v + i * 8));
         }
     }
-    QD_PCLK(9);
-    QD_TL(9);
+    fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tbase, 256);
+    QD_TL(9);
+    if (tid == 0) {
+        const int y = (int)(((size_t)bh * p.N + 2 * pr) * D);
+        tma_store_2d(&mapUt, sQ, 0, y);
+        tma_store_2d(&mapUt, sQ + 16384, 0, y + D);
+        tma_store_2d(&mapWt, sV, 0, y);
+        tma_store_2d(&mapWt, sV + 16384, 0, y + D);
+        tma_store_commit();
+        tma_store_wait_read();             // the staging tiles must outlive the reads; the writes complete with the grid
+    }
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tbase, 256);
+    }
     QD_TL(11);
 }
 
@@ -667,17 +663,19 @@ TcLayout tc_layout(const qd_shape& s) {
 
 cudaError_t tc_prep(const ChunkArgs& a) {
     const qd_shape& s = a.s;
-    CUtensorMap mQ, mK, mV;
+    CUtensorMap mQ, mK, mV, mUt, mWt;
     const uint64_t rows = (uint64_t)s.B * s.T, cols = (uint64_t)s.H * D;
+    const uint64_t trows = (uint64_t)s.B * s.H * (s.T / kChunk) * D;          // rows of the [chunk][d][64] tiles
     if (!make_tmap_bf16_2d(&mQ, a.q, cols, rows, cols * 2, 128) || !make_tmap_bf16_2d(&mK, a.k, cols, rows, cols * 2, 128) ||
-        !make_tmap_bf16_2d(&mV, a.v, cols, rows, cols * 2, 128))
+        !make_tmap_bf16_2d(&mV, a.v, cols, rows, cols * 2, 128) ||
+        !make_tmap_bf16_2d(&mUt, a.ws + a.TL.Ut, 64, trows, 128, 128) ||
+        !make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, trows, 128, 128))
         return cudaErrorInvalidValue;
     PrepParams p{};
     p.T = s.T; p.H = s.H; p.N = s.T / kChunk;
     p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
     p.g = (float*)(a.ws + a.TL.g);
     p.Qg = (bf16*)(a.ws + a.TL.Qg); p.P = (bf16*)(a.ws + a.TL.P);
-    p.Wt = (bf16*)(a.ws + a.TL.Wt); p.Ut = (bf16*)(a.ws + a.TL.Ut);
     p.Mt = a.save ? (bf16*)(a.ws + a.TL.Mt) : nullptr;
     p.status = (unsigned*)(a.ws + a.TL.status);
 #ifdef QD_CTA_TIMELINE
@@ -686,7 +684,7 @@ cudaError_t tc_prep(const ChunkArgs& a) {
     cudaError_t e = set_smem(k_tc_prep, kPrepSmem);
     if (e != cudaSuccess) return e;
     const int grid = s.B * s.H * (p.N / 2);
-    k_tc_prep<<<grid, 128, kPrepSmem, a.stream>>>(mQ, mK, mV, p);
+    k_tc_prep<<<grid, kPrepThreads, kPrepSmem, a.stream>>>(mQ, mK, mV, mUt, mWt, p);
     return cudaGetLastError();
 }
 
