@@ -292,13 +292,17 @@ constexpr int oQ = 0, oK = 16384, oV = 32768, odO = 49152, oX = 65536, oMt = 819
               odDt = 114688, oH = 131072, odH = 163840;                            // TMA-loaded tiles (X is built)
 constexpr int kBwdEarlyBytes = 3 * 16384 + 2 * 8192, kBwdLateBytes = 16384 + 2 * 16384 + 2 * 32768;
 // tiles built later reuse regions whose contents are dead by then
-constexpr int odPG = oV, odTb = oV + 8192, odW = odO, oN = oH, odXK = oH + 8192, oPP = oH + 16384,
+constexpr int odPG = oV, odTb = oV + 8192, odW = 196608, oN = oH, odXK = oH + 8192, oPP = oH + 16384,
               oAA = odH + 1024, oStDv = odDt, oStDk = oDt, oStDq = odDt;
-constexpr int kBwdSmem = 196608 + 1024;
+constexpr int kBwdSmem = 196608 + 16384 + 1024;      // + the dW<-^T tile, written while dO is still an operand
 constexpr int LDAA = C + 1;
 constexpr int kNWG = 4;                       // warpgroups; each owns 64/kNWG columns of every 64-column accumulator
 constexpr int kCW = C / kNWG, kG8 = kCW / 8;    // columns per warpgroup, groups of 8 columns
-constexpr int kBwdThreads = 128 * kNWG;
+constexpr int kBwdCompute = 128 * kNWG;                 // epilogue threads
+constexpr int kBwdThreads = kBwdCompute + 32;            // + one warp that issues every TMA copy and every MMA
+// named barriers of k_tc_chunk_bwd: 1 = the epilogue threads among themselves; the others are raised by the
+// epilogue threads (bar.arrive) when an operand tile is complete and awaited by the issuing warp (bar.sync)
+constexpr int kNbC = 1, kNbX = 2, kNbDW = 3, kNbDTb = 4, kNbN = 5, kNbDXK = 6, kNbOut = 7, kNbDV = 8;
 
 // Optional phase timestamps (build with -DQD_PHASE_CLOCKS -DQD_CLK_CTA=<chunk>): thread 0 of the CTA that owns that chunk
 // writes clock64() values into bytes 64.. of the workspace status section.
@@ -352,12 +356,13 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                                                               ChunkBwdParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ uint64_t bar_load, bar_late, bar_mma;
+    __shared__ uint64_t bar_load, bar_late, bm_a, bm_b, bm_2, bm_3, bm_4, bm_5;
     __shared__ uint32_t tmem_slot;
+    __shared__ volatile int s_abort, s_latch;
     __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C], segc[C];
     __shared__ float sred[3][4][C];   // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
     __shared__ float srow[4][kNWG][C];   // per-row partial sums over each warpgroup's columns: rPP, d beta, t2, rAA
-    __shared__ float sdg[C], skd[C], swp[kBwdThreads / 32], scol[2][kBwdThreads / 64][C];
+    __shared__ float sdg[C], skd[C], swp[kBwdCompute / 32], scol[2][kBwdCompute / 64][C];
 
     const int tid = threadIdx.x, wg = tid >> 7, l = tid & 127, lane = tid & 31, wq = (tid >> 5) & 3;
     const int c0 = wg * kCW;                                      // my columns of a 64-column accumulator
@@ -365,8 +370,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     if (tid == 0) {
         mbar_init(&bar_load, 1);
         mbar_init(&bar_late, 1);
-        mbar_init(&bar_mma, 1);
+        mbar_init(&bm_a, 1); mbar_init(&bm_b, 1); mbar_init(&bm_2, 1); mbar_init(&bm_3, 1); mbar_init(&bm_4, 1);
+        mbar_init(&bm_5, 2);              // the products' completion and "the dv staging tile has been read"
         mbar_init_fence();
+        s_abort = 0;
+        s_latch = 0;
     }
     if (tid < 32) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
     tc_fence_before();
@@ -419,16 +427,117 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             cf_g = p.g[(size_t)bh_ * p.T + (size_t)n_ * C + tid];
         }
     };
-    if ((int)blockIdx.x < p.total) {
-        if (tid == 0) { issue_early(blockIdx.x); issue_late(blockIdx.x); }
-        fetch_coef(blockIdx.x);
-    }
-    uint32_t mma_ph = 0;                                          // parity of the next completion of bar_mma
+    // bounded wait; once any wait has expired every later wait returns at once and the kernel drains: all
+    // threads still pass every barrier, results are garbage, the status word says so
+    auto wait = [&](uint64_t* bar, uint32_t parity) {
+        if (s_abort) return;
+        if (!mbar_wait(bar, parity)) { s_abort = 1; *p.status = QD_ERR_TIMEOUT; }
+    };
+    const uint32_t aQ = smem_u32(sm + oQ), aK = smem_u32(sm + oK), aV = smem_u32(sm + oV), adO = smem_u32(sm + odO),
+                   aX = smem_u32(sm + oX), aMt = smem_u32(sm + oMt), aDt = smem_u32(sm + oDt),
+                   adDt = smem_u32(sm + odDt), aH = smem_u32(sm + oH), adH = smem_u32(sm + odH);
+    const uint32_t adPG = smem_u32(sm + odPG), adTb = smem_u32(sm + odTb), adW = smem_u32(sm + odW),
+                   aN = smem_u32(sm + oN), adXK = smem_u32(sm + odXK);
+
+    if (tid >= kBwdCompute) {
+        // =============================== issuing warp: TMA copies and MMAs ===============================
+        const bool lead = lane == 0;
+        if (lead && (int)blockIdx.x < p.total) { issue_early(blockIdx.x); issue_late(blockIdx.x); }
+        for (int ch_id = blockIdx.x, it = 0; ch_id < p.total; ch_id += gridDim.x, ++it) {
+            const int n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
+            const int row0 = (int)((size_t)b * p.T + (size_t)n * C);
+            const int next_id = ch_id + gridDim.x;
+            const uint32_t ph = it & 1;
+            if (s_latch) break;
+            if (lead) {
+                wait(&bar_load, ph);
+                wait(&bar_late, ph);
+                tc_fence_after();
+                umma_product<true, true>(T3, aH, 16384, adDt, 8192, C, D, false, true);     // -h dDelta^T      [i][r] = dW<-^T
+                umma_commit(&bm_a);
+                umma_product<false, false>(T7, adH, 16384, aK, 8192, C, D, false);          // dh^T K^T         [j][s]
+                umma_product<false, false>(T6, adDt, 16384, aMt, 8192, C, C, false);        // dDelta^T M       [j][s]
+                umma_product<false, true>(T1, adO, 8192, aDt, 8192, C, D, false);           // dO Delta^T       [r][s]
+                umma_product<false, true>(T2, aV, 8192, adDt, 8192, C, D, false);           // V dDelta^T       [s][r]
+                umma_product<true, false>(T4, aH, 16384, adO, 8192, C, D, false);           // h dO^T           [i][r]
+                umma_commit(&bm_b);                 // from here on no product reads dO, V, dDelta^T or h any more
+                umma_product<true, true>(T5, adH, 16384, aDt, 8192, C, D, false);           // dh Delta^T       [i][s]
+            }
+            nb_sync(kNbX, kBwdThreads);                                  // X has been built
+            if (lead) {
+                tc_fence_after();
+                umma_product<false, false>(T0, aX, 8192, aK, 8192, C, D, false);            // X K^T            [r][i]
+            }
+            nb_sync(kNbDW, kBwdThreads);                                 // the dW<-^T tile is complete
+            if (lead) {
+                tc_fence_after();
+                umma_product<false, true>(T3, aX, 8192, adW, 8192, C, D, false);            // X dW<-^T         [s][r]
+                umma_commit(&bm_2);
+            }
+            nb_sync(kNbDV, kBwdThreads);                                 // the dv staging tile is complete, T6 has been read
+            if (lead) {
+                tma_store_2d(&mapdV, sm + oStDv, hh * D, row0);
+                tma_store_2d(&mapdV, sm + oStDv + 8192, hh * D + 64, row0);
+                tma_store_commit();
+                tc_fence_after();
+                umma_product<false, false>(T6, adW, 16384, aMt, 8192, C, C, false);         // dW<-^T M         [i][s]
+            }
+            nb_sync(kNbDTb, kBwdThreads);
+            if (lead) {
+                tc_fence_after();
+                umma_product<true, true>(T1, adTb, 8192, aMt, 8192, C, C, false);           // N~ = dT diag(beta) M^T   [r][u]
+                umma_commit(&bm_3);
+            }
+            nb_sync(kNbN, kBwdThreads);
+            if (lead) {
+                tc_fence_after();
+                umma_product<false, true>(T2, aMt, 8192, aN, 8192, C, C, false, true);      // dA = -M^T N~     [r][s]
+                umma_commit(&bm_4);
+            }
+            nb_sync(kNbDXK, kBwdThreads);
+            if (lead) {
+                tc_fence_after();
+                umma_product<true, false>(T7, aK, 8192, adXK, 8192, C, C, false);           // (dXK K)^T        [i][r]
+                umma_product<true, true>(T1, aX, 8192, adXK, 8192, C, C, false);            // (dXK^T X)^T      [i][s]
+                umma_product<true, true>(T1, aQ, 8192, adPG, 8192, C, C, true);             // + (dPG^T Q)^T
+                umma_product<true, false>(T2, aK, 8192, adPG, 8192, C, C, false);           // (dPG K)^T        [i][r]
+                umma_commit(&bm_5);
+                tma_store_wait_read();                                   // the dv staging tile may be reused now
+                mbar_arrive(&bm_5);
+                wait(&bm_5, ph);
+                // K, V, dO, M^T, P of this chunk are dead: fetch the next chunk's
+                if (next_id < p.total && !s_abort) issue_early(next_id);
+            }
+            nb_sync(kNbOut, kBwdThreads);                                // the dk and dq staging tiles are complete
+            if (lead) {
+                tma_store_2d(&mapdK, sm + oStDk, hh * D, row0);
+                tma_store_2d(&mapdK, sm + oStDk + 8192, hh * D + 64, row0);
+                tma_store_2d(&mapdQ, sm + oStDq, hh * D, row0);
+                tma_store_2d(&mapdQ, sm + oStDq + 8192, hh * D + 64, row0);
+                tma_store_commit();
+            }
+            // s_latch is read by everyone right after the barrier and not written again before the next one;
+            // an expiry that this read misses is seen one chunk later (waits return at once meanwhile)
+            if (lead) s_latch = s_abort;
+            __syncthreads();                                             // every read of this chunk's tiles and scratch is done
+            if (lead) {
+                tma_store_wait_read();                                   // the staging tiles have been read by the stores
+                fence_proxy_async();
+                if (next_id < p.total && !s_abort) issue_late(next_id);
+            }
+        }
+        if (lead) tma_store_wait_all();
+    } else {
+    // ======================================== epilogue threads ========================================
+    auto csync = [&]() { nb_sync(kNbC, kBwdCompute); };
+    if ((int)blockIdx.x < p.total) fetch_coef(blockIdx.x);
 
     for (int ch_id = blockIdx.x, it = 0; ch_id < p.total; ch_id += gridDim.x, ++it) {
     const int n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
     const size_t row0 = (size_t)b * p.T + (size_t)n * C;          // token row in the [B*T] view
     const int next_id = ch_id + gridDim.x;
+    const uint32_t ph = it & 1;
+    if (s_latch) break;
 
     QD_CLK(0);
     if (tid < C) {
@@ -438,23 +547,14 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         sg[tid] = cf_g;
         sgam[tid] = __expf(cf_g);
     }
-    __syncthreads();
+    csync();
     if (tid < C) segc[tid] = __expf(sg[C - 1] - sg[tid]);
-
-    bool fail = !mbar_wait(&bar_load, it & 1);
-    fail = fail || !mbar_wait(&bar_late, it & 1);
-    if (__syncthreads_or(fail)) {
-        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        mbar_wait(&bar_load, it & 1);
-        mbar_wait(&bar_late, it & 1);
-        __syncthreads();
-        if (tid < 32) tmem_dealloc(tb, 512);
-        return;
-    }
+    wait(&bar_load, ph);
+    wait(&bar_late, ph);
     QD_CLK(1);
-    // ---- phase 0: X = K + lambda Q; partial <dh,h>_F ------------------------------------------------
+    // ---- X = K + lambda Q (the products that do not read X are already running); partial <dh,h>_F -------
     {
-        constexpr int kPer = 16 / (kBwdThreads / 64);     // 16-byte chunks of a row per thread
+        constexpr int kPer = 16 / (kBwdCompute / 64);     // 16-byte chunks of a row per thread
         const int r = tid & 63, part = tid >> 6;
         const float lm = slam[r];
 #pragma unroll
@@ -469,6 +569,9 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             sts128(sm + oX + off, pack8(kv));
         }
     }
+    fence_proxy_async();
+    tc_fence_before();                                    // also orders the previous chunk's TMEM reads before the new products
+    nb_arrive(kNbX, kBwdThreads);
     float dhh_part = 0.f;
 #pragma unroll
     for (int cc = 0; cc < 16 / kNWG; ++cc) {
@@ -480,48 +583,33 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
 #pragma unroll
         for (int e = 0; e < 8; ++e) dhh_part = fmaf(a[e], c8[e], dhh_part);
     }
+    QD_CLK(2);
+    // ---- dW<-^T = -h dDelta^T: row i = l as an operand tile (region of its own: dO is still being read) -----
+    wait(&bm_a, ph);
+    tc_fence_after();
+#pragma unroll
+    for (int g8 = 0; g8 < kG8; ++g8) {
+        float dw[8];
+        ld8(my(T3) + g8 * 8, dw);
+        tmem_ld_wait();
+        sts128(sm + odW + sw128_chunk(l, wg * kG8 + g8), pack8(dw));
+    }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
-    QD_CLK(2);
-    // ---- phase 1 products ------------------------------------------------------------------------
-    const uint32_t aQ = smem_u32(sm + oQ), aK = smem_u32(sm + oK), aV = smem_u32(sm + oV), adO = smem_u32(sm + odO),
-                   aX = smem_u32(sm + oX), aMt = smem_u32(sm + oMt), aDt = smem_u32(sm + oDt),
-                   adDt = smem_u32(sm + odDt), aH = smem_u32(sm + oH), adH = smem_u32(sm + odH);
-    const uint32_t adPG = smem_u32(sm + odPG), adTb = smem_u32(sm + odTb), adW = smem_u32(sm + odW),
-                   aN = smem_u32(sm + oN), adXK = smem_u32(sm + odXK);
-    if (tid == 0) {
-        tc_fence_after();
-        umma_product<false, false>(T0, aX, 8192, aK, 8192, C, D, false);            // X K^T            [r][i]
-        umma_product<false, true>(T1, adO, 8192, aDt, 8192, C, D, false);           // dO Delta^T       [r][s]
-        umma_product<false, true>(T2, aV, 8192, adDt, 8192, C, D, false);           // V dDelta^T       [s][r]
-        umma_product<true, true>(T3, aH, 16384, adDt, 8192, C, D, false, true);     // -h dDelta^T      [i][r] = dW<-^T
-        umma_product<true, false>(T4, aH, 16384, adO, 8192, C, D, false);           // h dO^T           [i][r]
-        umma_product<true, true>(T5, adH, 16384, aDt, 8192, C, D, false);           // dh Delta^T       [i][s]
-        umma_product<false, false>(T6, adDt, 16384, aMt, 8192, C, C, false);        // dDelta^T M       [j][s]
-        umma_product<false, false>(T7, adH, 16384, aK, 8192, C, D, false);          // dh^T K^T         [j][s]
-        umma_commit(&bar_mma);
-    }
-    fail = !mbar_wait(&bar_mma, mma_ph);
-    mma_ph ^= 1;
-    if (__syncthreads_or(fail)) {
-        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        if (tid < 32) tmem_dealloc(tb, 512);
-        return;
-    }
+    nb_arrive(kNbDW, kBwdThreads);
+    wait(&bm_b, ph);
     tc_fence_after();
     QD_CLK(3);
     float* sPP = reinterpret_cast<float*>(sm + oPP);
     {
-        // my 32 columns in four groups of 8 (one 16-byte bf16 chunk each)
+        // my columns in groups of 8 (one 16-byte bf16 chunk each)
         float rPP = 0.f;
         unsigned char* stg = sm + oStDv + (l >> 6) * 8192;
-#pragma unroll 1
+#pragma unroll
         for (int g8 = 0; g8 < kG8; ++g8) {
             const int cb = c0 + g8 * 8, ck = wg * kG8 + g8;
-            float kd[8], dw[8], dvv[8];
+            float kd[8], dvv[8];
             ld8(my(T7) + g8 * 8, kd);
-            ld8(my(T3) + g8 * 8, dw);
             ld8(my(T6) + g8 * 8, dvv);
             tmem_ld_wait();
             // <(K-> dh)_s, Delta_s>: (K-> dh)^T[j][s] = gamma_C/gamma_s (dh^T K^T)[j][s] in fp32, times Delta^T[j][s];
@@ -532,8 +620,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             for (int e = 0; e < 8; ++e) kd[e] *= segc[cb + e] * dl[e];
             const float ksum = col_reduce8(kd, lane);
             if ((lane & 3) == 0) sred[0][wq][cb + col8_of_lane(lane)] = ksum;
-            // dW<-^T row i = l as an operand tile; dV^T row j = l scaled by beta_s into the staging tile
-            sts128(sm + odW + sw128_chunk(l, ck), pack8(dw));
+            // dV^T row j = l scaled by beta_s into the staging tile
 #pragma unroll
             for (int e = 0; e < 8; ++e)
                 sts16(stg + sw128_off(cb + e, l & 63), __float2bfloat16_rn(sbeta[cb + e] * dvv[e]));
@@ -561,25 +648,9 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    nb_arrive(kNbDV, kBwdThreads);
     QD_CLK(4);
-    // ---- phase 2 ---------------------------------------------------------------------------------
-    if (tid == 0) {
-        tma_store_2d(&mapdV, sm + oStDv, hh * D, (int)row0);
-        tma_store_2d(&mapdV, sm + oStDv + 8192, hh * D + 64, (int)row0);
-        tma_store_commit();
-        tc_fence_after();
-        umma_product<false, true>(T7, aX, 8192, adW, 8192, C, D, false);            // X dW<-^T         [s][r]
-        umma_product<false, false>(T6, adW, 16384, aMt, 8192, C, C, false);         // dW<-^T M         [i][s]
-        umma_commit(&bar_mma);
-    }
-    fail = !mbar_wait(&bar_mma, mma_ph);
-    mma_ph ^= 1;
-    if (__syncthreads_or(fail)) {
-        if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
-        if (tid < 32) tmem_dealloc(tb, 512);
-        return;
-    }
+    wait(&bm_2, ph);
     tc_fence_after();
     QD_CLK(5);
     if (l < C) {
@@ -587,12 +658,12 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         const int s = l;
         const float gs = sgam[s], bs = sbeta[s];
         float mb = 0.f, db = 0.f;
-#pragma unroll 1
+#pragma unroll
         for (int g8 = 0; g8 < kG8; ++g8) {
             const int ck = wg * kG8 + g8;
             float a[8], bq[8], m[8], tb8[8];
             ld8(my(T2) + g8 * 8, a);
-            ld8(my(T7) + g8 * 8, bq);
+            ld8(my(T3) + g8 * 8, bq);
             tmem_ld_wait();
             load8(sm + oMt + sw128_chunk(s, ck), m);
 #pragma unroll
@@ -609,24 +680,13 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    nb_arrive(kNbDTb, kBwdThreads);
     QD_CLK(6);
-    // ---- phase 3: N~ = dT diag(beta) M^T ----------------------------------------------------------
-    if (tid == 0) {
-        tc_fence_after();
-        umma_product<true, true>(T1, adTb, 8192, aMt, 8192, C, C, false);           // [r][u]
-        umma_commit(&bar_mma);
-    }
-    fail = !mbar_wait(&bar_mma, mma_ph);
-    mma_ph ^= 1;
-    if (__syncthreads_or(fail)) {
-        if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
-        if (tid < 32) tmem_dealloc(tb, 512);
-        return;
-    }
+    // ---- N~ = dT diag(beta) M^T, copied out as an operand tile --------------------------------------
+    wait(&bm_3, ph);
     tc_fence_after();
     if (l < C) {
-#pragma unroll 1
+#pragma unroll
         for (int g8 = 0; g8 < kG8; ++g8) {
             float v[8];
             ld8(my(T1) + g8 * 8, v);
@@ -636,21 +696,10 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    nb_arrive(kNbN, kBwdThreads);
     QD_CLK(8);
-    // ---- phase 4: dA = -M^T N~ ---------------------------------------------------------------------
-    if (tid == 0) {
-        tc_fence_after();
-        umma_product<false, true>(T2, aMt, 8192, aN, 8192, C, C, false, true);      // [r][s]
-        umma_commit(&bar_mma);
-    }
-    fail = !mbar_wait(&bar_mma, mma_ph);
-    mma_ph ^= 1;
-    if (__syncthreads_or(fail)) {
-        if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
-        if (tid < 32) tmem_dealloc(tb, 512);
-        return;
-    }
+    // ---- dA = -M^T N~ -----------------------------------------------------------------------------
+    wait(&bm_4, ph);
     tc_fence_after();
     QD_CLK(9);
     float* sAA = reinterpret_cast<float*>(sm + oAA);
@@ -658,7 +707,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         const int r = l;
         const float gr = sg[r], br = sbeta[r];
         float rAA = 0.f, db = 0.f;
-#pragma unroll 1
+#pragma unroll
         for (int g8 = 0; g8 < kG8; ++g8) {
             const int cb = c0 + g8 * 8;
             float da[8], xk[8];
@@ -685,38 +734,19 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     }
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
+    nb_arrive(kNbDXK, kBwdThreads);
     QD_CLK(10);
-    // ---- phase 5 ---------------------------------------------------------------------------------
-    if (tid == 0) {
-        tc_fence_after();
-        umma_product<true, false>(T7, aK, 8192, adXK, 8192, C, C, false);           // (dXK K)^T        [i][r]
-        umma_product<true, true>(T1, aX, 8192, adXK, 8192, C, C, false);            // (dXK^T X)^T      [i][s]
-        umma_product<true, true>(T1, aQ, 8192, adPG, 8192, C, C, true);             // + (dPG^T Q)^T
-        umma_product<true, false>(T2, aK, 8192, adPG, 8192, C, C, false);           // (dPG K)^T        [i][r]
-        umma_commit(&bar_mma);
-        tma_store_wait_read();                                      // the dv staging tile may be reused now
-    }
-    fail = !mbar_wait(&bar_mma, mma_ph);
-    mma_ph ^= 1;
-    if (__syncthreads_or(fail)) {
-        if (tid == 0) { *p.status = QD_ERR_TIMEOUT; tma_store_wait_all(); }
-        if (tid < 32) tmem_dealloc(tb, 512);
-        return;
-    }
+    // ---- the last products; meanwhile the coefficients of the next chunk ------------------------------
+    if (next_id < p.total) fetch_coef(next_id);
+    wait(&bm_5, ph);
     tc_fence_after();
     QD_CLK(11);
-    if (next_id < p.total) {
-        // K, V, dO, M^T, P of this chunk are dead: fetch the next chunk's, and its coefficients
-        if (tid == 0) issue_early(next_id);
-        fetch_coef(next_id);
-    }
     {
         const int i = l;                                            // d_k index; my 32 tokens c0..c0+31 in groups of 8
         unsigned char* stk = sm + oStDk + (i >> 6) * 8192;
         unsigned char* stq = sm + oStDq + (i >> 6) * 8192;
         const unsigned char* qcol = sm + oQ + (i >> 6) * 8192;
-#pragma unroll 1
+#pragma unroll
         for (int g8 = 0; g8 < kG8; ++g8) {
             const int cb = c0 + g8 * 8;
             float dx[8], v[8], w[8], u[8], z[8], y[8];
@@ -754,14 +784,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     if (lane == 0) swp[tid >> 5] = dhh_part;
     fence_proxy_async();
     tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
-        tma_store_2d(&mapdK, sm + oStDk, hh * D, (int)row0);
-        tma_store_2d(&mapdK, sm + oStDk + 8192, hh * D + 64, (int)row0);
-        tma_store_2d(&mapdQ, sm + oStDq, hh * D, (int)row0);
-        tma_store_2d(&mapdQ, sm + oStDq + 8192, hh * D + 64, (int)row0);
-        tma_store_commit();
-    }
+    nb_arrive(kNbOut, kBwdThreads);
+    csync();
     QD_CLK(12);
     // ---- decay gradient ----------------------------------------------------------------------------
     {
@@ -769,7 +793,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         const int r = tid & 63, part = tid >> 6;
         float cA = 0.f, cP = 0.f;
 #pragma unroll
-        constexpr int kRows = C / (kBwdThreads / 64);
+        constexpr int kRows = C / (kBwdCompute / 64);
 #pragma unroll
         for (int k = 0; k < kRows; ++k) {
             cA += sAA[(part * kRows + k) * LDAA + r];
@@ -778,14 +802,14 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         scol[0][part][r] = cA;
         scol[1][part][r] = cP;
     }
-    __syncthreads();
+    csync();
     if (tid < C) {
         const int r = tid;
         float kd = 0.f, dl = 0.f, t1 = 0.f, cAA = 0.f, cPP = 0.f;
 #pragma unroll
         for (int w4 = 0; w4 < 4; ++w4) { kd += sred[0][w4][r]; dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
 #pragma unroll
-        for (int w4 = 0; w4 < kBwdThreads / 64; ++w4) { cAA += scol[0][w4][r]; cPP += scol[1][w4][r]; }
+        for (int w4 = 0; w4 < kBwdCompute / 64; ++w4) { cAA += scol[0][w4][r]; cPP += scol[1][w4][r]; }
         float rPP = 0.f, t2 = 0.f, rAA = 0.f, dbt = 0.f;
 #pragma unroll
         for (int w4 = 0; w4 < kNWG; ++w4) { rPP += srow[0][w4][r]; dbt += srow[1][w4][r]; t2 += srow[2][w4][r]; rAA += srow[3][w4][r]; }
@@ -794,13 +818,13 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         p.dbeta[(row0 + r) * p.H + hh] = dbt;
         if (p.dlam) p.dlam[(row0 + r) * p.H + hh] = dl;
     }
-    __syncthreads();
+    csync();
     if (tid < 32) {
         // warp 0: lane owns tokens 2*lane, 2*lane+1; d log alpha_i = sum_{r >= i} dg_r (suffix sums)
         const float a = sdg[2 * lane];
         float b2 = sdg[2 * lane + 1];
         float kds = skd[2 * lane] + skd[2 * lane + 1];
-        float dhh = lane < kBwdThreads / 32 ? swp[lane] : 0.f;
+        float dhh = lane < kBwdCompute / 32 ? swp[lane] : 0.f;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             kds += __shfl_xor_sync(0xffffffffu, kds, o);
@@ -820,16 +844,12 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     }
     QD_CLK(13);
     __syncthreads();                     // every read of this chunk's tiles and scratch is done
-    if (tid == 0) {
-        tma_store_wait_read();           // the staging tiles have been read by the stores
-        fence_proxy_async();
-        if (next_id < p.total) issue_late(next_id);
-    }
     QD_CLK(14);
     }  // chunk loop
-    if (tid == 0) tma_store_wait_all();
+    }  // epilogue threads
     tc_fence_before();
     __syncthreads();
+    if (tid == kBwdCompute && s_abort) { mbar_wait(&bar_load, 0); mbar_wait(&bar_late, 0); }   // one more bounded chance for copies in flight
     if (tid < 32) tmem_dealloc(tb, 512);
 }
 
