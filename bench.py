@@ -73,6 +73,11 @@ def stage_bytes_per_token_head(dk, dv, C):
     }
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
+# profiles/tc_kernels_dram_traffic_cfg2.md (full-size cfg2); other workloads: not captured
+NCU_TRAFFIC_BYTES = {"cfg2": {"prep": 418.2e6, "chain_fwd": 535.7e6, "chain_bwd": 471.8e6, "chunk_bwd": 928.9e6}}
+
+
 class ClockSampler(threading.Thread):
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -212,6 +217,13 @@ def run_ours(args, cfg):
     qd.profile_enable(False)
     ms = e0.elapsed_time(e1)
     stages = qd.profile_read(reset=True)
+    # the timed region lasts milliseconds, nvidia-smi answers in ~0.1 s: keep the same step loop running
+    # (untimed) for a second or so, so that the clock samples are taken under this load
+    t_probe = time.perf_counter()
+    while time.perf_counter() - t_probe < 1.5:
+        for _ in range(20):
+            step()
+        torch.cuda.synchronize()
     sampler.stop_flag.set()
     sampler.join()
     ms, tokens_total = sharding.aggregate(ms, B * T * args.steps, "cuda")   # slowest rank, all ranks' tokens
@@ -257,7 +269,7 @@ def run_ours(args, cfg):
     dom_ms = chunk_stages[dom][0] / chunk_stages[dom][1]
     ach = sb[dom] * th / (dom_ms * 1e-3) / 1e9
     roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / pk["hbm_gbs"], "traffic": None, "peak_kind": "of " + pk_kind,
+                "frac": ach / pk["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(cfg.name, {}).get(dom), "peak_kind": "of " + pk_kind,
                 "ms_per_launch": dom_ms, "algorithmic_bytes_per_launch": sb[dom] * th}
     fb, bb = path_bytes_per_token_head(dk, dv)
     ff, fbw = path_flops_per_token_head(dk, dv, cfg.chunk)
@@ -268,6 +280,8 @@ def run_ours(args, cfg):
     path = {"bytes_per_step": (fb + bb) * th + state_io, "flops_per_step": (ff + fbw) * th,
             "roofline_ms": max(t_bytes, t_flops) * 1e3, "frac": max(t_bytes, t_flops) * 1e3 / per_rank_ms,
             "peak_kind": "of " + pk_kind,
+            "roofline_ms_nominal": max(((fb + bb) * th + state_io) / 8.0e12, (ff + fbw) * th / 2.25e15) * 1e3,
+            "frac_nominal": max(((fb + bb) * th + state_io) / 8.0e12, (ff + fbw) * th / 2.25e15) * 1e3 / per_rank_ms,
             "stage_ms_per_launch": {n: v[0] / v[1] for n, v in chunk_stages.items()}}
     launches = int(sum(v[1] for v in stages.values()))
 
@@ -278,6 +292,7 @@ def run_ours(args, cfg):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(cfg), "l2": "inputs larger than L2 (no flush)",
+                       "clock_sampling": "nvidia-smi during the timed steps and 1.5 s more of the same step loop",
                        "tokens_per_step": tokens_step, "parallelism": "batch sharded over %d rank(s), no collective" % world},
             "clocks": sampler.summary(),
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -286,11 +301,12 @@ def run_ours(args, cfg):
     if rank == 0:
         if world == 1 and not args.no_extras:
             cores = os.cpu_count() or 1
-            nseq = max(1, min(B * H, 4 * cores))
-            v, dt, thr = oracle_sample(cfg, nseq)
+            nseq = max(1, min(B * H, 8 * cores))
+            reps = 4
+            v, dt, thr = oracle_sample(cfg, nseq, steps=reps)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": thr, "kind": "oracle",
-                                    "sample": "first %d of %d (batch, head) sequences, fwd + reverse pass, fp64, %.1f s"
-                                              % (nseq, B * H, dt)}
+                                    "sample": "first %d of %d (batch, head) sequences, fwd + reverse pass, fp64, %d passes of %.1f s"
+                                              % (nseq, B * H, reps, dt)}
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()
