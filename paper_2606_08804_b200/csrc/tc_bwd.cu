@@ -74,7 +74,7 @@ constexpr int kChainThreads = 320;                 // 8 compute warps, 1 MMA-iss
 constexpr int kMmaWarp = 8;
 
 // named barriers: compute threads arrive, the MMA and TMA warps wait
-constexpr int kBarH = 1, kBarD = 2;
+constexpr int kBarH = 1, kBarD = 2, kBarHt = 4, kBarDt = 5;   // ..t: the same event, awaited by the TMA warp
 __device__ __forceinline__ void nb_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 __device__ __forceinline__ void nb_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 
@@ -99,6 +99,9 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
     __shared__ uint64_t bar_load[2], bar_a, bar_b, bar_e;
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int s_abort;
+    // per iteration parity: gamma_C / gamma_t for the 64 tokens, then gamma_C; written by the TMA warp one chunk
+    // ahead and published with its arrival on bar_a
+    __shared__ __align__(16) float sG[2][68];
 
     const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, l = tid & 127, wq = warp & 3;
     const int bh = blockIdx.x, b = bh / p.H, hh = bh % p.H;
@@ -138,25 +141,21 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) sts128(sdH + wg * 16384 + sw128_chunk(l, ch), pack8(dh + ch * 8));
         fence_proxy_async();
-        nb_arrive(kBarH, 320);
+        nb_arrive(kBarH, 288); nb_arrive(kBarHt, 288);
 
         for (int it = 0; it < p.N; ++it) {
-            const int n = p.N - 1 - it;
-            const float gC = gseq[(size_t)n * C + C - 1];
+            wait(&bar_a, it & 1);
+            tc_fence_after();
             float sc[32];
             {
-                const float4* gp = reinterpret_cast<const float4*>(gseq + (size_t)n * C + wg * 32);
+                const float4* gp = reinterpret_cast<const float4*>(&sG[it & 1][wg * 32]);
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const float4 t = gp[q];
                     sc[q * 4] = t.x; sc[q * 4 + 1] = t.y; sc[q * 4 + 2] = t.z; sc[q * 4 + 3] = t.w;
                 }
             }
-#pragma unroll
-            for (int i = 0; i < 32; ++i) sc[i] = __expf(gC - sc[i]);
-            const float gamC = __expf(gC);
-            wait(&bar_a, it & 1);
-            tc_fence_after();
+            const float gamC = sG[it & 1][64];
             // dDelta^T = A1 + gamma_C/gamma_s A2, my 32 tokens
             {
                 float a1[32], a2[32];
@@ -170,7 +169,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarD, 320);
+            nb_arrive(kBarD, 288); nb_arrive(kBarDt, 288);
             wait(&bar_b, it & 1);
             tc_fence_after();
 #pragma unroll
@@ -186,7 +185,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarH, 320);
+            nb_arrive(kBarH, 288); nb_arrive(kBarHt, 288);
         }
         if (p.dh0 && !s_abort) {
             float* dst = p.dh0 + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
@@ -200,7 +199,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
         for (int it = 0; it < p.N; ++it) {
             const uint32_t st = smem_u32(smem + (it & 1) * kStage);
             if (lead) wait(&bar_load[it & 1], (it >> 1) & 1);
-            nb_sync(kBarH, 320);                          // dh^T operand (exit state of this chunk) is in place
+            nb_sync(kBarH, 288);                          // dh^T operand (exit state of this chunk) is in place
             if (lead) {
                 tc_fence_after();
                 const uint32_t sdO = st + 16384;
@@ -211,7 +210,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
                 // H-accumulator = dO^T Qg (B MN-major: lines = token r, two blocks of d_k)
                 umma_product<true, true>(tH, sdO, 8192, st + 32768, 8192, D, C, false);
             }
-            nb_sync(kBarD, 320);                          // dDelta^T operand is in place
+            nb_sync(kBarD, 288);                          // dDelta^T operand is in place
             if (lead) {
                 tc_fence_after();
                 // H-accumulator -= dDelta^T W<-   (A negated; B K-major: lines = d_k index, contraction over tokens)
@@ -220,7 +219,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
                 umma_commit(&bar_e);
             }
         }
-        nb_sync(kBarH, 320);                              // final arrival of the compute warps
+        nb_sync(kBarH, 288);                              // final arrival of the compute warps
     } else {
         // ---------------------------------- TMA warp ----------------------------------
         const bool lead = (tid & 31) == 0;
@@ -243,13 +242,24 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
             tma_load_2d(st + 65536, &mapP, 0, yt, bar);
         };
         if (lead) { issue_load(0); if (p.N > 1) issue_load(1); }
+        const int ln = tid & 31;
+        const float* gl = gseq + (size_t)(p.N - 1) * C;               // cumulative log-decays of the last chunk
+        float g0 = gl[ln], g1 = gl[32 + ln], gc = gl[C - 1];
         for (int it = 0; it < p.N; ++it) {
             const int n = p.N - 1 - it;
+            sG[it & 1][ln] = __expf(gc - g0);
+            sG[it & 1][32 + ln] = __expf(gc - g1);
+            if (ln == 0) sG[it & 1][64] = __expf(gc);
+            __syncwarp();
+            if (n > 0) {                                      // in flight while this chunk is processed
+                const float* gn = gseq + (size_t)(n - 1) * C;
+                g0 = gn[ln]; g1 = gn[32 + ln]; gc = gn[C - 1];
+            }
             if (lead) {
                 tma_store_wait_read_n<0>();               // dDelta^T tile of the previous chunk has been read
                 mbar_arrive(&bar_a);
             }
-            nb_sync(kBarH, 320);                          // dh^T operand (exit state of chunk n) is in place
+            nb_sync(kBarHt, 288);                          // dh^T operand (exit state of chunk n) is in place
             if (lead) {
                 // gradient w.r.t. the exit state of chunk n, bf16, as the operand tile (rows = d_v, cols = d_k)
                 const int yh = (int)(((size_t)bh * p.N + n) * D);
@@ -257,7 +267,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
                 tma_store_2d(&mapdHs, sdH + 16384, 64, yh);
                 tma_store_commit();
             }
-            nb_sync(kBarD, 320);                          // dDelta^T of chunk n is in place
+            nb_sync(kBarDt, 288);                          // dDelta^T of chunk n is in place
             if (lead) {
                 tma_store_2d(&mapdDt, sdD, 0, (int)(((size_t)bh * p.N + n) * D));
                 tma_store_commit();
@@ -267,7 +277,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
                 if (it + 2 < p.N && !s_abort) issue_load(it + 2);
             }
         }
-        nb_sync(kBarH, 320);                              // final arrival of the compute warps
+        nb_sync(kBarHt, 288);                              // final arrival of the compute warps
         if (lead) {
             tma_store_wait_all();
             if (s_abort) { mbar_wait(&bar_load[0], 0); mbar_wait(&bar_load[1], 0); }

@@ -345,7 +345,7 @@ constexpr int kChainThreads = 320;                 // 8 compute warps, 1 MMA-iss
 constexpr int kMmaWarp = 8, kTmaWarp = 9;
 
 // named barriers: compute threads arrive, the MMA and/or TMA warp wait
-constexpr int kBarH = 1, kBarD = 2, kBarO = 3;
+constexpr int kBarH = 1, kBarD = 2, kBarO = 3, kBarHt = 4, kBarDt = 5;   // ..t: the same event, awaited by the TMA warp
 __device__ __forceinline__ void nb_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 __device__ __forceinline__ void nb_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
 
@@ -373,6 +373,9 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
     __shared__ uint64_t bar_load[2], bar_a, bar_b, bar_o, bar_e;
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int s_abort;
+    // per chunk parity: gamma_C / gamma_t for the 64 tokens, then gamma_C; written by the TMA warp one chunk
+    // ahead and published with its arrival on bar_a, so no epilogue thread waits for a global load
+    __shared__ __align__(16) float sG[2][68];
 
     const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, l = tid & 127, wq = warp & 3;
     const int bh = blockIdx.x, b = bh / p.H, hh = bh % p.H;
@@ -417,7 +420,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         for (int e = 0; e < 8; ++e)
             xoff[e] = (uint32_t)e * 128u + (((((uint32_t)l & 63u) >> 3) ^ (uint32_t)e) << 4) + ((uint32_t)l & 7u) * 2u;
         fence_proxy_async();
-        nb_arrive(kBarH, 320);
+        nb_arrive(kBarH, 288); nb_arrive(kBarHt, 288);
 
         auto o_stage = [&](int m) {
             // output of chunk m: O^T row j = l, my 32 tokens -> staging tile (token-major); stored by the TMA warp
@@ -442,25 +445,22 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         for (int n = 0; n < p.N; ++n) {
             QD_C(0);
             const unsigned char* st = smem + (n & 1) * kStage;
-            const float gC = gseq[(size_t)n * C + C - 1];
+            QD_C(1);
+            wait(&bar_load[n & 1], (n >> 1) & 1);
+            wait(&bar_a, n & 1);
+            QD_C(2);
+            tc_fence_after();
             // decay ratios of my 32 tokens
             float sc[32];
             {
-                const float4* gp = reinterpret_cast<const float4*>(gseq + (size_t)n * C + wg * 32);
+                const float4* gp = reinterpret_cast<const float4*>(&sG[n & 1][wg * 32]);
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     const float4 t = gp[q];
                     sc[q * 4] = t.x; sc[q * 4 + 1] = t.y; sc[q * 4 + 2] = t.z; sc[q * 4 + 3] = t.w;
                 }
             }
-#pragma unroll
-            for (int i = 0; i < 32; ++i) sc[i] = __expf(gC - sc[i]);
-            const float gamC = __expf(gC);
-            QD_C(1);
-            wait(&bar_load[n & 1], (n >> 1) & 1);
-            wait(&bar_a, n & 1);
-            QD_C(2);
-            tc_fence_after();
+            const float gamC = sG[n & 1][64];
             // Delta^T = Ut - acc, my 32 tokens; two bf16 copies (plain, and scaled by gamma_C/gamma_r) as A operands
             {
                 const unsigned char* ut = st + 16384;
@@ -483,7 +483,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarD, 320);
+            nb_arrive(kBarD, 288); nb_arrive(kBarDt, 288);
             QD_C(3);
             // in the shadow of the H product: output epilogue of the previous chunk
             if (n > 0) { wait(&bar_o, (n - 1) & 1); tc_fence_after(); o_stage(n - 1); }
@@ -505,7 +505,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarH, 320);
+            nb_arrive(kBarH, 288); nb_arrive(kBarHt, 288);
             QD_C(6);
         }
         wait(&bar_o, (p.N - 1) & 1);
@@ -525,7 +525,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             const uint32_t tO = tO0 + 64 * (n & 1);
             QD_M(0);
             if (lead) wait(&bar_load[n & 1], (n >> 1) & 1);
-            nb_sync(kBarH, 320);                          // h^T operand of chunk n is in place
+            nb_sync(kBarH, 288);                          // h^T operand of chunk n is in place
             QD_M(1);
             if (lead) {
                 tc_fence_after();
@@ -538,7 +538,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 umma_product<false, false>(tO, aH, 16384, st + 32768, 8192, C, D, false);
             }
             QD_M(3);
-            nb_sync(kBarD, 320);                          // Delta^T operands of chunk n are in place
+            nb_sync(kBarD, 288);                          // Delta^T operands of chunk n are in place
             QD_M(4);
             if (lead) {
                 tc_fence_after();
@@ -553,7 +553,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 QD_M(6);
             }
         }
-        nb_sync(kBarH, 320);                              // final arrival of the compute warps
+        nb_sync(kBarH, 288);                              // final arrival of the compute warps
     } else {
         // ---------------------------------- TMA warp ----------------------------------
         const bool lead = (tid & 31) == 0;
@@ -573,7 +573,17 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             tma_load_2d(st + 65536, &mapP, 0, yt, bar);
         };
         if (lead) { issue_load(0); if (p.N > 1) issue_load(1); }
+        const int ln = tid & 31;
+        float g0 = gseq[ln], g1 = gseq[32 + ln], gc = gseq[C - 1];     // cumulative log-decays of chunk 0
         for (int n = 0; n < p.N; ++n) {
+            sG[n & 1][ln] = __expf(gc - g0);
+            sG[n & 1][32 + ln] = __expf(gc - g1);
+            if (ln == 0) sG[n & 1][64] = __expf(gc);
+            __syncwarp();
+            if (n + 1 < p.N) {                                  // in flight while this chunk is processed
+                const float* gn = gseq + (size_t)(n + 1) * C;
+                g0 = gn[ln]; g1 = gn[32 + ln]; gc = gn[C - 1];
+            }
             if (lead) {
                 // every store issued so far (Delta^T of chunk n-1, output of chunk n-2) has read its tile:
                 // the Delta^T tiles may be rewritten (chunk n), the output staging tile too (chunk n-1)
@@ -581,7 +591,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 mbar_arrive(&bar_a);
                 if (n > 0) mbar_arrive(&bar_o);
             }
-            nb_sync(kBarH, 320);                          // h^T operand of chunk n is in place
+            nb_sync(kBarHt, 288);                          // h^T operand of chunk n is in place
             if (lead && p.save) {
                 // entry state of chunk n, bf16, exactly the operand tile: rows = d_v index, cols = d_k index
                 const int yh = (int)(((size_t)bh * p.N + n) * D);
@@ -589,7 +599,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 tma_store_2d(&mapHs, sH + 16384, 64, yh);
             }
             if (lead) tma_store_commit();                 // group: entry state of chunk n
-            nb_sync(kBarD, 320);                          // Delta^T of chunk n is in place
+            nb_sync(kBarDt, 288);                          // Delta^T of chunk n is in place
             if (lead) {
                 if (p.save) tma_store_2d(&mapDt, sD, 0, (int)(((size_t)bh * p.N + n) * D));
                 tma_store_commit();                       // group: Delta^T of chunk n
@@ -610,7 +620,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 if (n + 2 < p.N && !s_abort) issue_load(n + 2);
             }
         }
-        nb_sync(kBarH, 320);                              // final arrival of the compute warps
+        nb_sync(kBarHt, 288);                              // final arrival of the compute warps
         if (lead) { tma_store_wait_read_n<0>(); mbar_arrive(&bar_o); }
         nb_sync(kBarO, 288);                              // output tile of the last chunk staged
         if (lead) {
