@@ -295,6 +295,7 @@ struct ChunkBwdParams {
     const float* g;
     float *dbeta, *dalpha, *dlam;
     unsigned* status;
+    long long* timeline;       // diagnostic builds only (QD_CTA_TIMELINE): start time of every chunk
 };
 
 // shared-memory map of k_tc_chunk_bwd (bytes from the 1024-aligned base)
@@ -550,6 +551,9 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     if (s_latch) break;
 
     QD_CLK(0);
+#ifdef QD_CTA_TIMELINE
+    if (tid == 0) { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); p.timeline[ch_id] = t; }
+#endif
     if (tid < C) {
         sbeta[tid] = cf_beta;
         slam[tid] = cf_lam;
@@ -919,6 +923,9 @@ cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
     p.g = (const float*)(a.ws + a.TL.g);
     p.dbeta = a.dbeta; p.dalpha = a.dalpha; p.dlam = a.dlam;
     p.status = (unsigned*)(a.ws + a.TL.status);
+#ifdef QD_CTA_TIMELINE
+    p.timeline = (long long*)(a.ws + a.TL.Ut);      // U~^T is not read by the backward kernels
+#endif
     cudaError_t e = set_smem(k_tc_chunk_bwd, kBwdSmem);
     if (e != cudaSuccess) return e;
     // persistent: one CTA per SM walks the chunks with stride gridDim.x
