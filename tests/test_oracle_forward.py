@@ -1,4 +1,5 @@
 """Pins of the forward recurrence oracle (CPU only)."""
+import os
 import numpy as np
 import pytest
 
@@ -204,3 +205,22 @@ def test_heads_and_batches_are_independent():
             o1, h1 = orc.forward(**sl)
             np.testing.assert_allclose(o1[0, :, 0], o[b, :, hh], atol=1e-15)
             np.testing.assert_allclose(h1[0, 0], hT[b, hh], atol=1e-15)
+
+
+def test_golden_fixture_reproduced():
+    """The stored results of a tiny seeded problem (tests/golden/qdelta_tiny.txt, written by make_golden.py
+    from the oracle alone) are reproduced: guards against unintended changes of the oracle's arithmetic."""
+    import importlib.util
+    here = os.path.dirname(os.path.abspath(__file__))
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "golden", "make_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    got = mod.compute()
+    lines = [l for l in open(os.path.join(here, "golden", "qdelta_tiny.txt")) if not l.startswith("#")]
+    assert len(lines) == 2 * len(got)
+    for head, vals in zip(lines[0::2], lines[1::2]):
+        f = head.split()
+        name, shape = f[0], tuple(int(x) for x in f[1:])
+        want = np.array([float(x) for x in vals.split()]).reshape(shape)
+        assert np.asarray(got[name]).shape == shape
+        np.testing.assert_allclose(np.asarray(got[name], np.float64), want, rtol=1e-13, atol=1e-15)
