@@ -76,7 +76,10 @@ constexpr int kMmaWarp = 8;
 // named barriers: compute threads arrive, the MMA and TMA warps wait
 constexpr int kBarH = 1, kBarD = 2, kBarHt = 4, kBarDt = 5;   // ..t: the same event, awaited by the TMA warp
 __device__ __forceinline__ void nb_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
-__device__ __forceinline__ void nb_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+__device__ __forceinline__ void nb_sync(int id, int count) {
+    __syncwarp();                                   // the lanes of a warp reach the barrier together
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
 
 // Reverse state chain.  Per chunk the dependency is
 //   dh ready -> A2 = dh^T K^T -> dDelta^T -> H-accumulator -= dDelta^T W<- -> dh update;
@@ -540,7 +543,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         if (lead) tma_store_wait_all();
     } else {
     // ======================================== epilogue threads ========================================
-    auto csync = [&]() { nb_sync(kNbC, kBwdCompute); };
+    auto csync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(kNbC), "r"(kBwdCompute) : "memory"); };   // warps arrive converged
     if ((int)blockIdx.x < p.total) fetch_coef(blockIdx.x);
 
     for (int ch_id = blockIdx.x, it = 0; ch_id < p.total; ch_id += gridDim.x, ++it) {

@@ -347,7 +347,10 @@ constexpr int kMmaWarp = 8, kTmaWarp = 9;
 // named barriers: compute threads arrive, the MMA and/or TMA warp wait
 constexpr int kBarH = 1, kBarD = 2, kBarO = 3, kBarHt = 4, kBarDt = 5;   // ..t: the same event, awaited by the TMA warp
 __device__ __forceinline__ void nb_arrive(int id, int count) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory"); }
-__device__ __forceinline__ void nb_sync(int id, int count) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory"); }
+__device__ __forceinline__ void nb_sync(int id, int count) {
+    __syncwarp();                                   // the lanes of a warp reach the barrier together
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
 
 // Forward state chain.  The only true dependency per chunk is
 //   h ready -> Delta-accumulator = h^T Wt -> Delta^T -> H-accumulator = (scaled Delta^T) K -> h update;
