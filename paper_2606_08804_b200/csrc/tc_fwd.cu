@@ -65,7 +65,7 @@ __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u6
 //   scan / coefficients   thread t < 128 owns token t
 //   row-wise elementwise  16 threads per 256-byte row (coalesced), 16 rows per pass
 //   Gram epilogue         thread (row = t & 127, half = t >> 7) owns 32 columns of its TMEM lane
-//   triangular inverse    thread (column = t >> 1, parity = t & 1) owns the 8-row blocks of that parity
+//   triangular inverse    lane pair (t >> 1, t < 128) owns columns j0 < 32 and j0 + 32 of one chunk, parity t & 1 the 8-row blocks
 //   final epilogue        thread (d = t & 127, which = t >> 7) owns one row of U~^T resp. W~^T
 __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
                                                              const __grid_constant__ CUtensorMap mapK,
@@ -226,49 +226,72 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     tc_fence_before();
     __syncthreads();
     QD_TL(5);
-    // M_c = (I + A_c)^-1 by right-looking substitution, one column per thread pair, the column in registers:
-    // the thread of parity `par` owns the 8-row blocks 2s + par (s = 0..3).  Once m[i] is final its owner
-    // hands it to the partner lane and every later row gets its update m[r] -= A[r][i] m[i]; rows <= i of a
-    // block see A = 0 exactly.  Rows above the column index come out as exact zeros, the diagonal as one.
-    const int colid = tid >> 1, par = tid & 1, ic = colid >> 6, ij = colid & 63;
-    float m[4][8];
-    {
+    // M_c = (I + A_c)^-1 by right-looking substitution, columns in registers.  A lane pair of the first four warps
+    // owns two columns of one chunk, j0 < 32 and j1 = j0 + 32 (the same loads of A serve both); the lane of parity
+    // `par` owns the 8-row blocks 2s + par.  Once m[i] is final its owner hands it to the partner lane and every
+    // later row gets its update m[r] -= A[r][i] m[i]; rows <= i of a block see A = 0 exactly.  Column j1 is zero
+    // above row 32, so it joins at step 32 and keeps only its blocks 4..7.  The loads of A are warp-wide
+    // broadcasts, and shared-memory wavefronts are what bounds this phase: hence two columns per load.
+    const int q = tid >> 1, par = tid & 1, ic = (q >> 5) & 1, j0 = q & 31, j1 = j0 + 32;
+    float m0[4][8], m1[2][8];
+    if (tid < 128) {
         const float* Ac = sA + ic * C * C + par * 8;
 #pragma unroll
         for (int s = 0; s < 4; ++s)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) m[s][e] = ((2 * s + par) * 8 + e == ij) ? 1.f : 0.f;
+            for (int e = 0; e < 8; ++e) m0[s][e] = ((2 * s + par) * 8 + e == j0) ? 1.f : 0.f;
+#pragma unroll
+        for (int s = 0; s < 2; ++s)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) m1[s][e] = ((2 * s + 4 + par) * 8 + e == j1) ? 1.f : 0.f;
 #pragma unroll
         for (int i = 0; i < C - 1; ++i) {
-            const float mi = __shfl_sync(0xffffffffu, m[i >> 4][i & 7], (lane & ~1) | ((i >> 3) & 1));
+            const int src = (lane & ~1) | ((i >> 3) & 1);
+            const float mi0 = __shfl_sync(0xffffffffu, m0[i >> 4][i & 7], src);
+            float mi1 = 0.f;
+            if (i >= 32) mi1 = __shfl_sync(0xffffffffu, m1[(i >> 4) - 2][i & 7], src);
 #pragma unroll
             for (int s = (i + 1) >> 4; s < 4; ++s) {
                 const float4 a0 = *reinterpret_cast<const float4*>(Ac + i * C + s * 16);
                 const float4 a1 = *reinterpret_cast<const float4*>(Ac + i * C + s * 16 + 4);
-                m[s][0] = fmaf(-a0.x, mi, m[s][0]); m[s][1] = fmaf(-a0.y, mi, m[s][1]);
-                m[s][2] = fmaf(-a0.z, mi, m[s][2]); m[s][3] = fmaf(-a0.w, mi, m[s][3]);
-                m[s][4] = fmaf(-a1.x, mi, m[s][4]); m[s][5] = fmaf(-a1.y, mi, m[s][5]);
-                m[s][6] = fmaf(-a1.z, mi, m[s][6]); m[s][7] = fmaf(-a1.w, mi, m[s][7]);
+                m0[s][0] = fmaf(-a0.x, mi0, m0[s][0]); m0[s][1] = fmaf(-a0.y, mi0, m0[s][1]);
+                m0[s][2] = fmaf(-a0.z, mi0, m0[s][2]); m0[s][3] = fmaf(-a0.w, mi0, m0[s][3]);
+                m0[s][4] = fmaf(-a1.x, mi0, m0[s][4]); m0[s][5] = fmaf(-a1.y, mi0, m0[s][5]);
+                m0[s][6] = fmaf(-a1.z, mi0, m0[s][6]); m0[s][7] = fmaf(-a1.w, mi0, m0[s][7]);
+                if (i >= 32) {
+                    float* mm = m1[s >= 2 ? s - 2 : 0];
+                    mm[0] = fmaf(-a0.x, mi1, mm[0]); mm[1] = fmaf(-a0.y, mi1, mm[1]);
+                    mm[2] = fmaf(-a0.z, mi1, mm[2]); mm[3] = fmaf(-a0.w, mi1, mm[3]);
+                    mm[4] = fmaf(-a1.x, mi1, mm[4]); mm[5] = fmaf(-a1.y, mi1, mm[5]);
+                    mm[6] = fmaf(-a1.z, mi1, mm[6]); mm[7] = fmaf(-a1.w, mi1, mm[7]);
+                }
             }
         }
     }
     __syncthreads();
     QD_TL(6);
     // T_c = M_c diag(beta), T_c diag(gamma): line j of the MN-major tiles holds column j over the rows
-    {
+    if (tid < 128) {
         unsigned char* t0 = sT + ic * 8192;
         unsigned char* t1 = sT + 16384 + ic * 8192;
-        bf16* mt = p.Mt ? p.Mt + (((size_t)bh * p.N + 2 * pr + ic) * C + ij) * C : nullptr;
-        const float beta = sbeta[colid], bg = beta * __expf(sg[colid]);
+        bf16* mt = p.Mt ? p.Mt + ((size_t)bh * p.N + 2 * pr + ic) * C * C : nullptr;
 #pragma unroll
-        for (int s = 0; s < 4; ++s) {
-            const int kb = 2 * s + par;
-            float a[8], bq[8];
+        for (int col = 0; col < 2; ++col) {
+            const int j = col ? j1 : j0;
+            const float beta = sbeta[ic * C + j], bg = beta * __expf(sg[ic * C + j]);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) { a[e] = m[s][e] * beta; bq[e] = m[s][e] * bg; }
-            sts128(t0 + sw128_chunk(ij, kb), pack8(a));
-            sts128(t1 + sw128_chunk(ij, kb), pack8(bq));
-            if (mt) *reinterpret_cast<uint4*>(mt + kb * 8) = pack8(m[s]);
+            for (int s = 0; s < 4; ++s) {
+                const int kb = 2 * s + par;
+                float mv[8], a[8], bq[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    mv[e] = col ? (s >= 2 ? m1[s >= 2 ? s - 2 : 0][e] : 0.f) : m0[s][e];
+                    a[e] = mv[e] * beta; bq[e] = mv[e] * bg;
+                }
+                sts128(t0 + sw128_chunk(j, kb), pack8(a));
+                sts128(t1 + sw128_chunk(j, kb), pack8(bq));
+                if (mt) *reinterpret_cast<uint4*>(mt + (size_t)j * C + kb * 8) = pack8(mv);
+            }
         }
     }
     fence_proxy_async();
