@@ -70,8 +70,10 @@ struct ChainBwdParams {
 
 constexpr int kStage = 73728;                           // Wt 16K | dO 16K | Qg 16K | K 16K | P 8K
 constexpr int kChainSmem = 2 * kStage + 32768 + 16384 + 1024;
-constexpr int kChainThreads = 320;                 // 8 compute warps, 1 MMA-issue warp, 1 TMA warp
-constexpr int kMmaWarp = 8;
+constexpr int kChainCompute = 512;                 // 16 epilogue warps: 4 warpgroups split the accumulator columns
+constexpr int kChainThreads = kChainCompute + 64;  // + 1 MMA-issue warp, 1 TMA warp
+constexpr int kMmaWarp = kChainCompute / 32;
+constexpr int kNb = kChainCompute + 32;            // participants of a named barrier: the epilogue threads and one waiting warp
 
 // named barriers: compute threads arrive, the MMA and TMA warps wait
 constexpr int kBarH = 1, kBarD = 2, kBarHt = 4, kBarDt = 5;   // ..t: the same event, awaited by the TMA warp
@@ -130,70 +132,71 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
     };
     const float* gseq = p.g + (size_t)bh * p.T;
 
-    if (warp < 8) {
+    if (warp < kMmaWarp) {
         // ---------------------------------- compute warps ----------------------------------
-        float dh[64];     // dh^T[j = l][64 wg .. 64 wg + 63]
+        float dh[32];     // dh^T[j = l][32 wg .. 32 wg + 31]
         if (p.dhT) {
-            const float* src = p.dhT + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
+            const float* src = p.dhT + (size_t)bh * D * D + (size_t)(32 * wg) * D + l;
 #pragma unroll
-            for (int i = 0; i < 64; ++i) dh[i] = src[(size_t)i * D];
+            for (int i = 0; i < 32; ++i) dh[i] = src[(size_t)i * D];
         } else {
 #pragma unroll
-            for (int i = 0; i < 64; ++i) dh[i] = 0.f;
+            for (int i = 0; i < 32; ++i) dh[i] = 0.f;
         }
+        // my 32 columns of the operand tile: 64-column block wg >> 1, 16-byte chunks 4 (wg & 1) ..
+        unsigned char* myH = sdH + (wg >> 1) * 16384;
+        const int hc0 = (wg & 1) * 4;
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) sts128(sdH + wg * 16384 + sw128_chunk(l, ch), pack8(dh + ch * 8));
+        for (int ch = 0; ch < 4; ++ch) sts128(myH + sw128_chunk(l, hc0 + ch), pack8(dh + ch * 8));
         fence_proxy_async();
-        nb_arrive(kBarH, 288); nb_arrive(kBarHt, 288);
+        nb_arrive(kBarH, kNb); nb_arrive(kBarHt, kNb);
 
         for (int it = 0; it < p.N; ++it) {
             wait(&bar_a, it & 1);
             tc_fence_after();
-            float sc[32];
+            float sc[16];
             {
-                const float4* gp = reinterpret_cast<const float4*>(&sG[it & 1][wg * 32]);
+                const float4* gp = reinterpret_cast<const float4*>(&sG[it & 1][wg * 16]);
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
+                for (int q = 0; q < 4; ++q) {
                     const float4 t = gp[q];
                     sc[q * 4] = t.x; sc[q * 4 + 1] = t.y; sc[q * 4 + 2] = t.z; sc[q * 4 + 3] = t.w;
                 }
             }
             const float gamC = sG[it & 1][64];
-            // dDelta^T = A1 + gamma_C/gamma_s A2, my 32 tokens
+            // dDelta^T = A1 + gamma_C/gamma_s A2, my 16 tokens
             {
-                float a1[32], a2[32];
-                tmem_ld32(tmem_addr(tA1, lane_base, wg * 32), a1);
-                tmem_ld32(tmem_addr(tA2, lane_base, wg * 32), a2);
+                float a1[16], a2[16];
+                tmem_ld16(tmem_addr(tA1, lane_base, wg * 16), a1);
+                tmem_ld16(tmem_addr(tA2, lane_base, wg * 16), a2);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) a1[i] = fmaf(sc[i], a2[i], a1[i]);
+                for (int i = 0; i < 16; ++i) a1[i] = fmaf(sc[i], a2[i], a1[i]);
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc) sts128(sdD + sw128_chunk(l, wg * 4 + cc), pack8(a1 + cc * 8));
+                for (int cc = 0; cc < 2; ++cc) sts128(sdD + sw128_chunk(l, wg * 2 + cc), pack8(a1 + cc * 8));
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarD, 288); nb_arrive(kBarDt, 288);
+            nb_arrive(kBarD, kNb); nb_arrive(kBarDt, kNb);
             wait(&bar_b, it & 1);
             tc_fence_after();
-#pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2) {
+            {
                 float v[32];
-                tmem_ld32(tmem_addr(tH, lane_base, wg * 64 + q2 * 32), v);
+                tmem_ld32(tmem_addr(tH, lane_base, wg * 32), v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) dh[q2 * 32 + i] = fmaf(gamC, dh[q2 * 32 + i], v[i]);
+                for (int i = 0; i < 32; ++i) dh[i] = fmaf(gamC, dh[i], v[i]);
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
-                    sts128(sdH + wg * 16384 + sw128_chunk(l, q2 * 4 + cc), pack8(dh + q2 * 32 + cc * 8));
+                for (int cc = 0; cc < 4; ++cc) sts128(myH + sw128_chunk(l, hc0 + cc), pack8(dh + cc * 8));
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarH, 288); nb_arrive(kBarHt, 288);
+            nb_arrive(kBarH, kNb); nb_arrive(kBarHt, kNb);
         }
         if (p.dh0 && !s_abort) {
-            float* dst = p.dh0 + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
+            float* dst = p.dh0 + (size_t)bh * D * D + (size_t)(32 * wg) * D + l;
 #pragma unroll
-            for (int i = 0; i < 64; ++i) dst[(size_t)i * D] = dh[i];
+            for (int i = 0; i < 32; ++i) dst[(size_t)i * D] = dh[i];
         }
     } else if (warp == kMmaWarp) {
         // ---------------------------------- MMA-issue warp ----------------------------------
@@ -202,7 +205,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
         for (int it = 0; it < p.N; ++it) {
             const uint32_t st = smem_u32(smem + (it & 1) * kStage);
             if (lead) wait(&bar_load[it & 1], (it >> 1) & 1);
-            nb_sync(kBarH, 288);                          // dh^T operand (exit state of this chunk) is in place
+            nb_sync(kBarH, kNb);                          // dh^T operand (exit state of this chunk) is in place
             if (lead) {
                 tc_fence_after();
                 const uint32_t sdO = st + 16384;
@@ -213,7 +216,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
                 // H-accumulator = dO^T Qg (B MN-major: lines = token r, two blocks of d_k)
                 umma_product<true, true>(tH, sdO, 8192, st + 32768, 8192, D, C, false);
             }
-            nb_sync(kBarD, 288);                          // dDelta^T operand is in place
+            nb_sync(kBarD, kNb);                          // dDelta^T operand is in place
             if (lead) {
                 tc_fence_after();
                 // H-accumulator -= dDelta^T W<-   (A negated; B K-major: lines = d_k index, contraction over tokens)
@@ -222,7 +225,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
                 umma_commit(&bar_e);
             }
         }
-        nb_sync(kBarH, 288);                              // final arrival of the compute warps
+        nb_sync(kBarH, kNb);                              // final arrival of the compute warps
     } else {
         // ---------------------------------- TMA warp ----------------------------------
         const bool lead = (tid & 31) == 0;
@@ -262,7 +265,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
                 tma_store_wait_read_n<0>();               // dDelta^T tile of the previous chunk has been read
                 mbar_arrive(&bar_a);
             }
-            nb_sync(kBarHt, 288);                          // dh^T operand (exit state of chunk n) is in place
+            nb_sync(kBarHt, kNb);                          // dh^T operand (exit state of chunk n) is in place
             if (lead) {
                 // gradient w.r.t. the exit state of chunk n, bf16, as the operand tile (rows = d_v, cols = d_k)
                 const int yh = (int)(((size_t)bh * p.N + n) * D);
@@ -270,7 +273,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
                 tma_store_2d(&mapdHs, sdH + 16384, 64, yh);
                 tma_store_commit();
             }
-            nb_sync(kBarDt, 288);                          // dDelta^T of chunk n is in place
+            nb_sync(kBarDt, kNb);                          // dDelta^T of chunk n is in place
             if (lead) {
                 tma_store_2d(&mapdDt, sdD, 0, (int)(((size_t)bh * p.N + n) * D));
                 tma_store_commit();
@@ -280,7 +283,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
                 if (it + 2 < p.N && !s_abort) issue_load(it + 2);
             }
         }
-        nb_sync(kBarHt, 288);                              // final arrival of the compute warps
+        nb_sync(kBarHt, kNb);                              // final arrival of the compute warps
         if (lead) {
             tma_store_wait_all();
             if (s_abort) { mbar_wait(&bar_load[0], 0); mbar_wait(&bar_load[1], 0); }

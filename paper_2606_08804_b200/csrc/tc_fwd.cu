@@ -364,8 +364,10 @@ struct ChainParams {
 
 constexpr int kStage = 73728;                                   // Wt 16K | Ut 16K | Qg 16K | K 16K | P 8K
 constexpr int kChainSmem = 2 * kStage + 65536 + 16384 + 1024;   // + h^T 32K, Delta^T 16K, scaled Delta^T 16K, O 16K
-constexpr int kChainThreads = 320;                 // 8 compute warps, 1 MMA-issue warp, 1 TMA warp
-constexpr int kMmaWarp = 8, kTmaWarp = 9;
+constexpr int kChainCompute = 512;                 // 16 epilogue warps: 4 warpgroups split the accumulator columns
+constexpr int kChainThreads = kChainCompute + 64;  // + 1 MMA-issue warp, 1 TMA warp
+constexpr int kMmaWarp = kChainCompute / 32;
+constexpr int kNb = kChainCompute + 32;            // participants of a named barrier: the epilogue threads and one waiting warp
 
 // named barriers: compute threads arrive, the MMA and/or TMA warp wait
 constexpr int kBarH = 1, kBarD = 2, kBarO = 3, kBarHt = 4, kBarDt = 5;   // ..t: the same event, awaited by the TMA warp
@@ -427,38 +429,41 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
     };
     const float* gseq = p.g + (size_t)bh * p.T;
 
-    if (warp < 8) {
+    if (warp < kMmaWarp) {
         // ---------------------------------- compute warps ----------------------------------
-        float h[64];      // h^T[j = l][64 wg .. 64 wg + 63], fp32
+        float h[32];      // h^T[j = l][32 wg .. 32 wg + 31], fp32
         if (p.h0) {
-            const float* src = p.h0 + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
+            const float* src = p.h0 + (size_t)bh * D * D + (size_t)(32 * wg) * D + l;
 #pragma unroll
-            for (int i = 0; i < 64; ++i) h[i] = src[(size_t)i * D];
+            for (int i = 0; i < 32; ++i) h[i] = src[(size_t)i * D];
         } else {
 #pragma unroll
-            for (int i = 0; i < 64; ++i) h[i] = 0.f;
+            for (int i = 0; i < 32; ++i) h[i] = 0.f;
         }
+        // my 32 columns of the operand tile: 64-column block wg >> 1, 16-byte chunks 4 (wg & 1) ..
+        unsigned char* myH = sH + (wg >> 1) * 16384;
+        const int hc0 = (wg & 1) * 4;
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) sts128(sH + wg * 16384 + sw128_chunk(l, ch), pack8(h + ch * 8));
+        for (int ch = 0; ch < 4; ++ch) sts128(myH + sw128_chunk(l, hc0 + ch), pack8(h + ch * 8));
         // byte offsets of my (fixed) column inside a staging line, for the 8 possible (token & 7)
         uint32_t xoff[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e)
             xoff[e] = (uint32_t)e * 128u + (((((uint32_t)l & 63u) >> 3) ^ (uint32_t)e) << 4) + ((uint32_t)l & 7u) * 2u;
         fence_proxy_async();
-        nb_arrive(kBarH, 288); nb_arrive(kBarHt, 288);
+        nb_arrive(kBarH, kNb); nb_arrive(kBarHt, kNb);
 
         auto o_stage = [&](int m) {
-            // output of chunk m: O^T row j = l, my 32 tokens -> staging tile (token-major); stored by the TMA warp
-            unsigned char* stg = sO + (l >> 6) * 8192 + (wg * 32) * 128;
-            float v[32];
-            tmem_ld32(tmem_addr(tO0 + 64 * (m & 1), lane_base, wg * 32), v);
+            // output of chunk m: O^T row j = l, my 16 tokens -> staging tile (token-major); stored by the TMA warp
+            unsigned char* stg = sO + (l >> 6) * 8192 + (wg * 16) * 128;
+            float v[16];
+            tmem_ld16(tmem_addr(tO0 + 64 * (m & 1), lane_base, wg * 16), v);
             tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) sts16(stg + (i >> 3) * 1024 + xoff[i & 7], __float2bfloat16_rn(v[i]));
+            for (int i = 0; i < 16; ++i) sts16(stg + (i >> 3) * 1024 + xoff[i & 7], __float2bfloat16_rn(v[i]));
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarO, 288);
+            nb_arrive(kBarO, kNb);
         };
 
 #ifdef QD_PHASE_CLOCKS
@@ -476,27 +481,27 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             wait(&bar_a, n & 1);
             QD_C(2);
             tc_fence_after();
-            // decay ratios of my 32 tokens
-            float sc[32];
+            // decay ratios of my 16 tokens
+            float sc[16];
             {
-                const float4* gp = reinterpret_cast<const float4*>(&sG[n & 1][wg * 32]);
+                const float4* gp = reinterpret_cast<const float4*>(&sG[n & 1][wg * 16]);
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
+                for (int q = 0; q < 4; ++q) {
                     const float4 t = gp[q];
                     sc[q * 4] = t.x; sc[q * 4 + 1] = t.y; sc[q * 4 + 2] = t.z; sc[q * 4 + 3] = t.w;
                 }
             }
             const float gamC = sG[n & 1][64];
-            // Delta^T = Ut - acc, my 32 tokens; two bf16 copies (plain, and scaled by gamma_C/gamma_r) as A operands
+            // Delta^T = Ut - acc, my 16 tokens; two bf16 copies (plain, and scaled by gamma_C/gamma_r) as A operands
             {
                 const unsigned char* ut = st + 16384;
-                float v[32];
-                tmem_ld32(tmem_addr(tD, lane_base, wg * 32), v);
+                float v[16];
+                tmem_ld16(tmem_addr(tD, lane_base, wg * 16), v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc) {
+                for (int cc = 0; cc < 2; ++cc) {
                     float u[8], d1[8];
-                    const uint32_t off = sw128_chunk(l, wg * 4 + cc);
+                    const uint32_t off = sw128_chunk(l, wg * 2 + cc);
                     load8(ut + off, u);
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
@@ -509,38 +514,36 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarD, 288); nb_arrive(kBarDt, 288);
+            nb_arrive(kBarD, kNb); nb_arrive(kBarDt, kNb);
             QD_C(3);
             // in the shadow of the H product: output epilogue of the previous chunk
             if (n > 0) { wait(&bar_o, (n - 1) & 1); tc_fence_after(); o_stage(n - 1); }
             QD_C(4);
-            // h^T <- gamma_C h^T + acc (my 64 d_k columns), refresh the bf16 operand copy
+            // h^T <- gamma_C h^T + acc (my 32 d_k columns), refresh the bf16 operand copy
             wait(&bar_b, n & 1);
             QD_C(5);
             tc_fence_after();
-#pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2) {
+            {
                 float v[32];
-                tmem_ld32(tmem_addr(tH, lane_base, wg * 64 + q2 * 32), v);
+                tmem_ld32(tmem_addr(tH, lane_base, wg * 32), v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) h[q2 * 32 + i] = fmaf(gamC, h[q2 * 32 + i], v[i]);
+                for (int i = 0; i < 32; ++i) h[i] = fmaf(gamC, h[i], v[i]);
 #pragma unroll
-                for (int cc = 0; cc < 4; ++cc)
-                    sts128(sH + wg * 16384 + sw128_chunk(l, q2 * 4 + cc), pack8(h + q2 * 32 + cc * 8));
+                for (int cc = 0; cc < 4; ++cc) sts128(myH + sw128_chunk(l, hc0 + cc), pack8(h + cc * 8));
             }
             tc_fence_before();
             fence_proxy_async();
-            nb_arrive(kBarH, 288); nb_arrive(kBarHt, 288);
+            nb_arrive(kBarH, kNb); nb_arrive(kBarHt, kNb);
             QD_C(6);
         }
         wait(&bar_o, (p.N - 1) & 1);
         tc_fence_after();
         o_stage(p.N - 1);
         if (p.hT && !s_abort) {
-            float* dst = p.hT + (size_t)bh * D * D + (size_t)(64 * wg) * D + l;
+            float* dst = p.hT + (size_t)bh * D * D + (size_t)(32 * wg) * D + l;
 #pragma unroll
-            for (int i = 0; i < 64; ++i) dst[(size_t)i * D] = h[i];
+            for (int i = 0; i < 32; ++i) dst[(size_t)i * D] = h[i];
         }
     } else if (warp == kMmaWarp) {
         // ---------------------------------- MMA-issue warp ----------------------------------
@@ -551,7 +554,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             const uint32_t tO = tO0 + 64 * (n & 1);
             QD_M(0);
             if (lead) wait(&bar_load[n & 1], (n >> 1) & 1);
-            nb_sync(kBarH, 288);                          // h^T operand of chunk n is in place
+            nb_sync(kBarH, kNb);                          // h^T operand of chunk n is in place
             QD_M(1);
             if (lead) {
                 tc_fence_after();
@@ -564,7 +567,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 umma_product<false, false>(tO, aH, 16384, st + 32768, 8192, C, D, false);
             }
             QD_M(3);
-            nb_sync(kBarD, 288);                          // Delta^T operands of chunk n are in place
+            nb_sync(kBarD, kNb);                          // Delta^T operands of chunk n are in place
             QD_M(4);
             if (lead) {
                 tc_fence_after();
@@ -579,7 +582,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 QD_M(6);
             }
         }
-        nb_sync(kBarH, 288);                              // final arrival of the compute warps
+        nb_sync(kBarH, kNb);                              // final arrival of the compute warps
     } else {
         // ---------------------------------- TMA warp ----------------------------------
         const bool lead = (tid & 31) == 0;
@@ -617,7 +620,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 mbar_arrive(&bar_a);
                 if (n > 0) mbar_arrive(&bar_o);
             }
-            nb_sync(kBarHt, 288);                          // h^T operand of chunk n is in place
+            nb_sync(kBarHt, kNb);                          // h^T operand of chunk n is in place
             if (lead && p.save) {
                 // entry state of chunk n, bf16, exactly the operand tile: rows = d_v index, cols = d_k index
                 const int yh = (int)(((size_t)bh * p.N + n) * D);
@@ -625,7 +628,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 tma_store_2d(&mapHs, sH + 16384, 64, yh);
             }
             if (lead) tma_store_commit();                 // group: entry state of chunk n
-            nb_sync(kBarDt, 288);                          // Delta^T of chunk n is in place
+            nb_sync(kBarDt, kNb);                          // Delta^T of chunk n is in place
             if (lead) {
                 if (p.save) tma_store_2d(&mapDt, sD, 0, (int)(((size_t)bh * p.N + n) * D));
                 tma_store_commit();                       // group: Delta^T of chunk n
@@ -633,7 +636,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 mbar_arrive(&bar_b);
             }
             if (n > 0) {
-                nb_sync(kBarO, 288);                      // output tile of chunk n-1 staged
+                nb_sync(kBarO, kNb);                      // output tile of chunk n-1 staged
                 if (lead) {
                     const int yo = (int)((size_t)b * p.T + (size_t)(n - 1) * C);
                     tma_store_2d(&mapO, sO, hh * D, yo);
@@ -646,9 +649,9 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                 if (n + 2 < p.N && !s_abort) issue_load(n + 2);
             }
         }
-        nb_sync(kBarHt, 288);                              // final arrival of the compute warps
+        nb_sync(kBarHt, kNb);                              // final arrival of the compute warps
         if (lead) { tma_store_wait_read_n<0>(); mbar_arrive(&bar_o); }
-        nb_sync(kBarO, 288);                              // output tile of the last chunk staged
+        nb_sync(kBarO, kNb);                              // output tile of the last chunk staged
         if (lead) {
             const int yo = (int)((size_t)b * p.T + (size_t)(p.N - 1) * C);
             tma_store_2d(&mapO, sO, hh * D, yo);
