@@ -432,6 +432,20 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         tma_load_2d(sm + oDt, &mapDt, 0, yc, &bar_late);
         tma_load_2d(sm + odDt, &mapdDt, 0, yc, &bar_late);
     };
+    // the late group of a chunk into L2 only, issued a chunk time before its load: the load, which can only be
+    // issued at the very end of the previous chunk and is waited for at once, then finds the tiles in L2
+    auto prefetch_late = [&](int ch) {
+        const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
+        const int yi = (int)((size_t)b_ * p.T + (size_t)n_ * C);
+        const int yc = (int)(((size_t)bh_ * p.N + n_) * D);
+        for (int blk = 0; blk < 2; ++blk) {
+            tma_prefetch_2d(&mapQ, hh_ * D + blk * 64, yi);
+            tma_prefetch_2d(&mapHs, blk * 64, yc);
+            tma_prefetch_2d(&mapdHs, blk * 64, yc);
+        }
+        tma_prefetch_2d(&mapDt, 0, yc);
+        tma_prefetch_2d(&mapdDt, 0, yc);
+    };
     // coefficients of token tid (< C) of a chunk, fetched one chunk ahead into registers
     float cf_beta = 0.f, cf_lam = 0.f, cf_alpha = 1.f, cf_g = 0.f;
     auto fetch_coef = [&](int ch) {
@@ -479,6 +493,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 umma_product<true, false>(T4, aH, 16384, adO, 8192, C, D, false);           // h dO^T           [i][r]
                 umma_commit(&bm_b);                 // from here on no product reads dO, V, dDelta^T or h any more
                 umma_product<true, true>(T5, adH, 16384, aDt, 8192, C, D, false);           // dh Delta^T       [i][s]
+                if (next_id < p.total) prefetch_late(next_id);
             }
             nb_sync(kNbX, kBwdThreads);                                  // X has been built
             if (lead) {
