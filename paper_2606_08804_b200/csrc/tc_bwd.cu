@@ -307,7 +307,7 @@ struct ChunkBwdParams {
 // shared-memory map of k_tc_chunk_bwd (bytes from the 1024-aligned base)
 constexpr int oQ = 0, oK = 16384, oV = 32768, odO = 49152, oX = 65536, oMt = 81920, oP = 90112, oDt = 98304,
               odDt = 114688, oH = 131072, odH = 163840;                            // TMA-loaded tiles (X is built)
-constexpr int kBwdEarlyBytes = 3 * 16384 + 2 * 8192, kBwdLateBytes = 16384 + 2 * 16384 + 2 * 32768;
+constexpr int kBwdEarlyBytes = 3 * 16384 + 2 * 8192;
 // tiles built later reuse regions whose contents are dead by then
 constexpr int odPG = oV, odTb = oV + 8192, odW = 196608, oN = oH, odXK = oH + 8192, oPP = oH + 16384,
               oAA = odH + 1024, oStDv = odDt, oStDk = oDt, oStDq = odDt;
@@ -319,7 +319,7 @@ constexpr int kBwdCompute = 128 * kNWG;                 // epilogue threads
 constexpr int kBwdThreads = kBwdCompute + 32;            // + one warp that issues every TMA copy and every MMA
 // named barriers of k_tc_chunk_bwd: 1 = the epilogue threads among themselves; the others are raised by the
 // epilogue threads (bar.arrive) when an operand tile is complete and awaited by the issuing warp (bar.sync)
-constexpr int kNbC = 1, kNbX = 2, kNbDW = 3, kNbDTb = 4, kNbN = 5, kNbDXK = 6, kNbOut = 7, kNbDV = 8;
+constexpr int kNbC = 1, kNbX = 2, kNbDW = 3, kNbDTb = 4, kNbN = 5, kNbDXK = 6, kNbOut = 7, kNbDV = 8, kNbScr = 9;
 
 // Optional phase timestamps (build with -DQD_PHASE_CLOCKS -DQD_CLK_CTA=<chunk>): thread 0 of the CTA that owns that chunk
 // writes clock64() values into bytes 64.. of the workspace status section.
@@ -419,18 +419,27 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         tma_load_2d(sm + oMt, &mapMt, 0, ym, &bar_load);
         tma_load_2d(sm + oP, &mapP, 0, yt, &bar_load);
     };
-    auto issue_late = [&](int ch) {
+    // The late group goes in three batches as its regions fall free: part 0 = Q (after the last epilogue),
+    // part 1 = h^T, dh^T (after the column sums have read the scratch that aliases them), part 2 = Delta^T,
+    // dDelta^T (after the stores have read the staging tiles).  Only the last batch arrives on the barrier.
+    auto issue_late = [&](int ch, int part) {
         const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
         const int yi = (int)((size_t)b_ * p.T + (size_t)n_ * C);
         const int yc = (int)(((size_t)bh_ * p.N + n_) * D);
-        mbar_expect_tx(&bar_late, kBwdLateBytes);
-        for (int blk = 0; blk < 2; ++blk) {
-            tma_load_2d(sm + oQ + blk * 8192, &mapQ, hh_ * D + blk * 64, yi, &bar_late);
-            tma_load_2d(sm + oH + blk * 16384, &mapHs, blk * 64, yc, &bar_late);
-            tma_load_2d(sm + odH + blk * 16384, &mapdHs, blk * 64, yc, &bar_late);
+        if (part == 0) {
+            mbar_expect_tx_only(&bar_late, 16384);
+            for (int blk = 0; blk < 2; ++blk) tma_load_2d(sm + oQ + blk * 8192, &mapQ, hh_ * D + blk * 64, yi, &bar_late);
+        } else if (part == 1) {
+            mbar_expect_tx_only(&bar_late, 2 * 32768);
+            for (int blk = 0; blk < 2; ++blk) {
+                tma_load_2d(sm + oH + blk * 16384, &mapHs, blk * 64, yc, &bar_late);
+                tma_load_2d(sm + odH + blk * 16384, &mapdHs, blk * 64, yc, &bar_late);
+            }
+        } else {
+            mbar_expect_tx(&bar_late, 2 * 16384);
+            tma_load_2d(sm + oDt, &mapDt, 0, yc, &bar_late);
+            tma_load_2d(sm + odDt, &mapdDt, 0, yc, &bar_late);
         }
-        tma_load_2d(sm + oDt, &mapDt, 0, yc, &bar_late);
-        tma_load_2d(sm + odDt, &mapdDt, 0, yc, &bar_late);
     };
     // the late group of a chunk into L2 only, issued a chunk time before its load: the load, which can only be
     // issued at the very end of the previous chunk and is waited for at once, then finds the tiles in L2
@@ -473,7 +482,10 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     if (tid >= kBwdCompute) {
         // =============================== issuing warp: TMA copies and MMAs ===============================
         const bool lead = lane == 0;
-        if (lead && (int)blockIdx.x < p.total) { issue_early(blockIdx.x); issue_late(blockIdx.x); }
+        if (lead && (int)blockIdx.x < p.total) {
+            issue_early(blockIdx.x);
+            issue_late(blockIdx.x, 0); issue_late(blockIdx.x, 1); issue_late(blockIdx.x, 2);
+        }
         for (int ch_id = blockIdx.x, it = 0; ch_id < p.total; ch_id += gridDim.x, ++it) {
             const int n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
             const int row0 = (int)((size_t)b * p.T + (size_t)n * C);
@@ -547,6 +559,13 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 tma_store_2d(&mapdQ, sm + oStDq, hh * D, row0);
                 tma_store_2d(&mapdQ, sm + oStDq + 8192, hh * D + 64, row0);
                 tma_store_commit();
+                fence_proxy_async();                                     // the epilogue's reads of Q precede the copy into its region
+                if (next_id < p.total && !s_abort) issue_late(next_id, 0);
+            }
+            nb_sync(kNbScr, kBwdThreads);                                // the column sums have read the scratch over h^T, dh^T
+            if (lead) {
+                fence_proxy_async();
+                if (next_id < p.total && !s_abort) issue_late(next_id, 1);
             }
             // s_latch is read by everyone right after the barrier and not written again before the next one;
             // an expiry that this read misses is seen one chunk later (waits return at once meanwhile)
@@ -555,7 +574,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             if (lead) {
                 tma_store_wait_read();                                   // the staging tiles have been read by the stores
                 fence_proxy_async();
-                if (next_id < p.total && !s_abort) issue_late(next_id);
+                if (next_id < p.total && !s_abort) issue_late(next_id, 2);
             }
         }
         if (lead) tma_store_wait_all();
@@ -837,6 +856,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         scol[0][part][r] = cA;
         scol[1][part][r] = cP;
     }
+    nb_arrive(kNbScr, kBwdThreads);      // the scratch tiles over h^T and dh^T are dead from here on
     csync();
     if (tid < C) {
         const int r = tid;
