@@ -420,7 +420,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         tma_load_2d(sm + oP, &mapP, 0, yt, &bar_load);
     };
     // The late group goes in three batches as its regions fall free: part 0 = Q (after the last epilogue),
-    // part 1 = h^T, dh^T (after the column sums have read the scratch that aliases them), part 2 = Delta^T,
+    // part 1 = h^T, dh^T (after the last products and the column sums have read the scratch that aliases them), part 2 = Delta^T,
     // dDelta^T (after the stores have read the staging tiles).  Only the last batch arrives on the barrier.
     auto issue_late = [&](int ch, int part) {
         const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
@@ -552,6 +552,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 // K, V, dO, M^T, P of this chunk are dead: fetch the next chunk's
                 if (next_id < p.total && !s_abort) issue_early(next_id);
             }
+            nb_sync(kNbScr, kBwdThreads);                                // the column sums have read the scratch over h^T, dh^T
+            if (lead) {
+                fence_proxy_async();
+                if (next_id < p.total && !s_abort) issue_late(next_id, 1);
+            }
             nb_sync(kNbOut, kBwdThreads);                                // the dk and dq staging tiles are complete
             if (lead) {
                 tma_store_2d(&mapdK, sm + oStDk, hh * D, row0);
@@ -561,11 +566,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 tma_store_commit();
                 fence_proxy_async();                                     // the epilogue's reads of Q precede the copy into its region
                 if (next_id < p.total && !s_abort) issue_late(next_id, 0);
-            }
-            nb_sync(kNbScr, kBwdThreads);                                // the column sums have read the scratch over h^T, dh^T
-            if (lead) {
-                fence_proxy_async();
-                if (next_id < p.total && !s_abort) issue_late(next_id, 1);
             }
             // s_latch is read by everyone right after the barrier and not written again before the next one;
             // an expiry that this read misses is seen one chunk later (waits return at once meanwhile)
@@ -790,7 +790,23 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     tc_fence_before();
     nb_arrive(kNbDXK, kBwdThreads);
     QD_CLK(10);
-    // ---- the last products; meanwhile the coefficients of the next chunk ------------------------------
+    // ---- the last products; meanwhile the column sums of dA o A and dP o P (kBwdCompute/64 threads per column)
+    // and the coefficients of the next chunk -------------------------------------------------------------------
+    csync();
+    {
+        const float* sAAc = reinterpret_cast<const float*>(sm + oAA);
+        const int r = tid & 63, part = tid >> 6;
+        float cA = 0.f, cP = 0.f;
+        constexpr int kRows = C / (kBwdCompute / 64);
+#pragma unroll
+        for (int k = 0; k < kRows; ++k) {
+            cA += sAAc[(part * kRows + k) * LDAA + r];
+            cP += sPP[(part * kRows + k) * LDAA + r];
+        }
+        scol[0][part][r] = cA;
+        scol[1][part][r] = cP;
+    }
+    nb_arrive(kNbScr, kBwdThreads);      // the scratch tiles over h^T and dh^T are dead from here on
     if (next_id < p.total) fetch_coef(next_id);
     wait(&bm_5, ph);
     tc_fence_after();
@@ -842,22 +858,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     csync();
     QD_CLK(12);
     // ---- decay gradient ----------------------------------------------------------------------------
-    {
-        // column sums of dA o A and dP o P: kBwdThreads/64 threads per column
-        const int r = tid & 63, part = tid >> 6;
-        float cA = 0.f, cP = 0.f;
-#pragma unroll
-        constexpr int kRows = C / (kBwdCompute / 64);
-#pragma unroll
-        for (int k = 0; k < kRows; ++k) {
-            cA += sAA[(part * kRows + k) * LDAA + r];
-            cP += sPP[(part * kRows + k) * LDAA + r];
-        }
-        scol[0][part][r] = cA;
-        scol[1][part][r] = cP;
-    }
-    nb_arrive(kNbScr, kBwdThreads);      // the scratch tiles over h^T and dh^T are dead from here on
-    csync();
     if (tid < C) {
         const int r = tid;
         float kd = 0.f, dl = 0.f, t1 = 0.f, cAA = 0.f, cPP = 0.f;
