@@ -33,15 +33,9 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
     u.x = pack_bf16(f[0], f[1]); u.y = pack_bf16(f[2], f[3]); u.z = pack_bf16(f[4], f[5]); u.w = pack_bf16(f[6], f[7]);
     return u;
 }
-// 64 TMEM columns of this thread's lane
-__device__ __forceinline__ void ld64(uint32_t taddr, float* v) {
-    tmem_ld32(taddr, v);
-    tmem_ld32(taddr + 32, v + 32);
-    tmem_ld_wait();
-}
 
-// Column sums across the 32 lanes of a warp: every lane passes 64 values; on return v[0], v[1] hold
-// the warp-wide sums of columns col, col+1 with col = col_of_lane(lane).
+// One halving step of a column sum across the lanes of a warp: lanes whose `off` bit is set keep the upper half
+// of the N values, the others the lower half; each adds what its partner sends.
 template <int N>
 __device__ __forceinline__ void fold(float* v, int lane, int off) {
     const bool up = (lane & off) != 0;
@@ -51,12 +45,6 @@ __device__ __forceinline__ void fold(float* v, int lane, int off) {
         const float send = up ? v[k] : v[N / 2 + k];
         v[k] = keep + __shfl_xor_sync(0xffffffffu, send, off);
     }
-}
-__device__ __forceinline__ void col_reduce64(float* v, int lane) {
-    fold<64>(v, lane, 16); fold<32>(v, lane, 8); fold<16>(v, lane, 4); fold<8>(v, lane, 2); fold<4>(v, lane, 1);
-}
-__device__ __forceinline__ int col_of_lane(int lane) {
-    return ((lane & 16) ? 32 : 0) + ((lane & 8) ? 16 : 0) + ((lane & 4) ? 8 : 0) + ((lane & 2) ? 4 : 0) + ((lane & 1) ? 2 : 0);
 }
 
 // =================================================================================================
@@ -329,19 +317,6 @@ constexpr int kNbC = 1, kNbX = 2, kNbDW = 3, kNbDTb = 4, kNbN = 5, kNbDXK = 6, k
 #define QD_CLK(i) do { } while (0)
 #endif
 
-// 32 TMEM columns of this thread's lane
-__device__ __forceinline__ void ld32(uint32_t taddr, float* v) {
-    tmem_ld32(taddr, v);
-    tmem_ld_wait();
-}
-// Column sums across the 32 lanes of a warp for 32 columns: on return v[0] is the warp-wide sum of
-// column col32_of_lane(lane).
-__device__ __forceinline__ void col_reduce32(float* v, int lane) {
-    fold<32>(v, lane, 16); fold<16>(v, lane, 8); fold<8>(v, lane, 4); fold<4>(v, lane, 2); fold<2>(v, lane, 1);
-}
-__device__ __forceinline__ int col32_of_lane(int lane) {
-    return ((lane & 16) ? 16 : 0) + ((lane & 8) ? 8 : 0) + ((lane & 4) ? 4 : 0) + ((lane & 2) ? 2 : 0) + ((lane & 1) ? 1 : 0);
-}
 // Column sums across the 32 lanes of a warp for 8 columns: returns, in every lane, the warp-wide sum of
 // column col8_of_lane(lane) (four lanes hold each column).
 __device__ __forceinline__ float col_reduce8(float* v, int lane) {
