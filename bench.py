@@ -75,7 +75,7 @@ def stage_bytes_per_token_head(dk, dv, C):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
 # profiles/tc_kernels_dram_traffic_cfg2.md (full-size cfg2); other workloads: not captured
-NCU_TRAFFIC_BYTES = {"cfg2": {"prep": 418.2e6, "chain_fwd": 535.7e6, "chain_bwd": 471.8e6, "chunk_bwd": 928.9e6}}
+NCU_TRAFFIC_BYTES = {"cfg2": {"prep": 421.9e6, "chain_fwd": 532.8e6, "chain_bwd": 469.2e6, "chunk_bwd": 926.2e6}}
 
 
 class ClockSampler(threading.Thread):
