@@ -782,6 +782,29 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         scol[1][part][r] = cP;
     }
     nb_arrive(kNbScr, kBwdThreads);      // the scratch tiles over h^T and dh^T are dead from here on
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 16);
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 8);
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 4);
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 2);
+    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 1);
+    if (lane == 0) swp[tid >> 5] = dhh_part;
+    csync();
+    // everything of the decay gradient that does not wait for the last epilogue
+    float dg_pre = 0.f;
+    if (tid < C) {
+        const int r = tid;
+        float kd = 0.f, cAA = 0.f, cPP = 0.f;
+#pragma unroll
+        for (int w4 = 0; w4 < 4; ++w4) kd += sred[0][w4][r];
+#pragma unroll
+        for (int w4 = 0; w4 < kBwdCompute / 64; ++w4) { cAA += scol[0][w4][r]; cPP += scol[1][w4][r]; }
+        float rPP = 0.f, t2 = 0.f, rAA = 0.f, dbt = 0.f;
+#pragma unroll
+        for (int w4 = 0; w4 < kNWG; ++w4) { rPP += srow[0][w4][r]; dbt += srow[1][w4][r]; t2 += srow[2][w4][r]; rAA += srow[3][w4][r]; }
+        dg_pre = rPP - cPP + t2 + rAA - cAA - kd;
+        skd[r] = kd;                            // summed below into dg of the last token
+        p.dbeta[(row0 + r) * p.H + hh] = dbt;
+    }
     if (next_id < p.total) fetch_coef(next_id);
     wait(&bm_5, ph);
     tc_fence_after();
@@ -821,12 +844,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             }
         }
     }
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 16);
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 8);
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 4);
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 2);
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 1);
-    if (lane == 0) swp[tid >> 5] = dhh_part;
     fence_proxy_async();
     tc_fence_before();
     nb_arrive(kNbOut, kBwdThreads);
@@ -835,17 +852,10 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     // ---- decay gradient ----------------------------------------------------------------------------
     if (tid < C) {
         const int r = tid;
-        float kd = 0.f, dl = 0.f, t1 = 0.f, cAA = 0.f, cPP = 0.f;
+        float dl = 0.f, t1 = 0.f;
 #pragma unroll
-        for (int w4 = 0; w4 < 4; ++w4) { kd += sred[0][w4][r]; dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
-#pragma unroll
-        for (int w4 = 0; w4 < kBwdCompute / 64; ++w4) { cAA += scol[0][w4][r]; cPP += scol[1][w4][r]; }
-        float rPP = 0.f, t2 = 0.f, rAA = 0.f, dbt = 0.f;
-#pragma unroll
-        for (int w4 = 0; w4 < kNWG; ++w4) { rPP += srow[0][w4][r]; dbt += srow[1][w4][r]; t2 += srow[2][w4][r]; rAA += srow[3][w4][r]; }
-        sdg[r] = t1 + rPP - cPP + t2 + rAA - cAA - kd;
-        skd[r] = kd;                            // summed below into dg of the last token
-        p.dbeta[(row0 + r) * p.H + hh] = dbt;
+        for (int w4 = 0; w4 < 4; ++w4) { dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
+        sdg[r] = t1 + dg_pre;
         if (p.dlam) p.dlam[(row0 + r) * p.H + hh] = dl;
     }
     csync();
