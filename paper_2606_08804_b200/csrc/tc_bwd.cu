@@ -475,7 +475,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 umma_commit(&bm_a);
                 umma_product<false, false>(T7, adH, 16384, aK, 8192, C, D, false);          // dh^T K^T         [j][s]
                 umma_product<false, false>(T6, adDt, 16384, aMt, 8192, C, C, false);        // dDelta^T M       [j][s]
-                umma_product<false, true>(T1, adO, 8192, aDt, 8192, C, D, false);           // dO Delta^T       [r][s]
+                umma_product<false, true>(T1, adO - 8192, 8192, aDt, 8192, C, D, false);    // dO Delta^T [r][s], rows r on lanes 64 + r
                 umma_product<false, true>(T2, aV, 8192, adDt, 8192, C, D, false);           // V dDelta^T       [s][r]
                 umma_product<true, false>(T4, aH, 16384, adO, 8192, C, D, false);           // h dO^T           [i][r]
                 umma_commit(&bm_b);                 // from here on no product reads dO, V, dDelta^T or h any more
@@ -504,7 +504,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             nb_sync(kNbDTb, kBwdThreads);
             if (lead) {
                 tc_fence_after();
-                umma_product<true, true>(T1, adTb, 8192, aMt, 8192, C, C, false);           // N~ = dT diag(beta) M^T   [r][u]
+                umma_product<true, true>(T3, adTb, 8192, aMt, 8192, C, C, false);           // N~ = dT diag(beta) M^T   [r][u]
                 umma_commit(&bm_3);
             }
             nb_sync(kNbN, kBwdThreads);
@@ -632,7 +632,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     float* sPP = reinterpret_cast<float*>(sm + oPP);
     {
         // my columns in groups of 8 (one 16-byte bf16 chunk each)
-        float rPP = 0.f;
         unsigned char* stg = sm + oStDv + (l >> 6) * 8192;
 #pragma unroll
         for (int g8 = 0; g8 < kG8; ++g8) {
@@ -653,32 +652,42 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
 #pragma unroll
             for (int e = 0; e < 8; ++e)
                 sts16(stg + sw128_off(cb + e, l & 63), __float2bfloat16_rn(sbeta[cb + e] * dvv[e]));
-            if (l < C) {
-                // dP row r = l: causal mask, dP o P (row and column sums), dP o Gamma as an operand tile
-                const int r = l;
-                float v[8], pv[8], pg[8];
-                ld8(my(T1) + g8 * 8, v);
-                tmem_ld_wait();
-                load8(sm + oP + sw128_chunk(r, ck), pv);
-                const float gr = sg[r];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int s = cb + e;
-                    const float dp = (s <= r) ? v[e] : 0.f;
-                    const float pp = dp * pv[e];
-                    rPP += pp;
-                    sts32(&sPP[r * LDAA + s], pp);
-                    pg[e] = (s <= r) ? dp * __expf(gr - sg[s]) : 0.f;
-                }
-                sts128(sm + odPG + sw128_chunk(r, ck), pack8(pg));
-            }
         }
-        if (l < C) srow[0][wg][l] = rPP;
     }
     fence_proxy_async();
     tc_fence_before();
     nb_arrive(kNbDV, kBwdThreads);
     QD_CLK(4);
+    // From here to the column sums the two halves of every warpgroup go separate ways.  Lanes 64..127 (whose rows
+    // of the 64-row accumulators are padding) take dP, whose product was issued with its rows on their lanes; lanes
+    // 0..63 walk the dependent chain dT -> N~ -> dA -> dXK.  Both raise every barrier of the chain exactly once.
+    if (l >= C) {
+        nb_arrive(kNbDTb, kBwdThreads);
+        nb_arrive(kNbN, kBwdThreads);
+        // dP row r = l - 64: causal mask, dP o P (row and column sums), dP o Gamma as an operand tile
+        const int r = l - C;
+        const float gr = sg[r];
+        float rPP = 0.f;
+#pragma unroll
+        for (int g8 = 0; g8 < kG8; ++g8) {
+            const int cb = c0 + g8 * 8, ck = wg * kG8 + g8;
+            float v[8], pv[8], pg[8];
+            ld8(my(T1) + g8 * 8, v);
+            tmem_ld_wait();
+            load8(sm + oP + sw128_chunk(r, ck), pv);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int s = cb + e;
+                const float dp = (s <= r) ? v[e] : 0.f;
+                const float pp = dp * pv[e];
+                rPP += pp;
+                sts32(&sPP[r * LDAA + s], pp);
+                pg[e] = (s <= r) ? dp * __expf(gr - sg[s]) : 0.f;
+            }
+            sts128(sm + odPG + sw128_chunk(r, ck), pack8(pg));
+        }
+        srow[0][wg][r] = rPP;
+    } else {
     wait(&bm_2, ph);
     tc_fence_after();
     QD_CLK(5);
@@ -718,7 +727,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
 #pragma unroll
         for (int g8 = 0; g8 < kG8; ++g8) {
             float v[8];
-            ld8(my(T1) + g8 * 8, v);
+            ld8(my(T3) + g8 * 8, v);
             tmem_ld_wait();
             sts128(sm + oN + sw128_chunk(l, wg * kG8 + g8), pack8(v));
         }
@@ -761,6 +770,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         srow[1][wg][r] += db;
         srow[3][wg][r] = rAA;
     }
+    }  // lanes 0..63: the dependent chain
     fence_proxy_async();
     tc_fence_before();
     nb_arrive(kNbDXK, kBwdThreads);
