@@ -348,7 +348,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                                                               ChunkBwdParams p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* sm = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    __shared__ uint64_t bar_load, bar_late, bm_a, bm_b, bm_2, bm_3, bm_4, bm_5;
+    __shared__ uint64_t bar_load, bar_late, bm_a, bm_b, bm_c, bm_2, bm_3, bm_4, bm_5;
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int s_abort, s_latch;
     __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C], segc[C];
@@ -362,7 +362,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     if (tid == 0) {
         mbar_init(&bar_load, 1);
         mbar_init(&bar_late, 1);
-        mbar_init(&bm_a, 1); mbar_init(&bm_b, 1); mbar_init(&bm_2, 1); mbar_init(&bm_3, 1); mbar_init(&bm_4, 1);
+        mbar_init(&bm_a, 1); mbar_init(&bm_b, 1); mbar_init(&bm_c, 1); mbar_init(&bm_2, 1); mbar_init(&bm_3, 1); mbar_init(&bm_4, 1);
         mbar_init(&bm_5, 2);              // the products' completion and "the dv staging tile has been read"
         mbar_init_fence();
         s_abort = 0;
@@ -475,10 +475,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 umma_commit(&bm_a);
                 umma_product<false, false>(T7, adH, 16384, aK, 8192, C, D, false);          // dh^T K^T         [j][s]
                 umma_product<false, false>(T6, adDt, 16384, aMt, 8192, C, C, false);        // dDelta^T M       [j][s]
-                umma_product<false, true>(T1, adO - 8192, 8192, aDt, 8192, C, D, false);    // dO Delta^T [r][s], rows r on lanes 64 + r
                 umma_product<false, true>(T2, aV, 8192, adDt, 8192, C, D, false);           // V dDelta^T       [s][r]
+                umma_commit(&bm_b);                 // from here on no product reads V or dDelta^T any more
+                umma_product<false, true>(T1, adO - 8192, 8192, aDt, 8192, C, D, false);    // dO Delta^T [r][s], rows r on lanes 64 + r
                 umma_product<true, false>(T4, aH, 16384, adO, 8192, C, D, false);           // h dO^T           [i][r]
-                umma_commit(&bm_b);                 // from here on no product reads dO, V, dDelta^T or h any more
+                umma_commit(&bm_c);                 // from here on no product reads dO or h any more
                 umma_product<true, true>(T5, adH, 16384, aDt, 8192, C, D, false);           // dh Delta^T       [i][s]
                 if (next_id < p.total) prefetch_late(next_id);
             }
@@ -664,6 +665,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     if (l >= C) {
         nb_arrive(kNbDTb, kBwdThreads);
         nb_arrive(kNbN, kBwdThreads);
+        wait(&bm_c, ph);                  // dP's product; its scratch lies over h^T, which that group has read
+        tc_fence_after();
         // dP row r = l - 64: causal mask, dP o P (row and column sums), dP o Gamma as an operand tile
         const int r = l - C;
         const float gr = sg[r];
