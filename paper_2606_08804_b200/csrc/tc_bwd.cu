@@ -353,7 +353,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     __shared__ volatile int s_abort, s_latch;
     __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C], segc[C];
     __shared__ float sred[3][4][C];   // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
-    __shared__ float srow[4][kNWG][C];   // per-row partial sums over each warpgroup's columns: rPP, d beta, t2, rAA
+    __shared__ float srow[6][kNWG][C];   // per-row partial sums over each warpgroup's columns: rPP, d beta, t2, rAA; [4], [5]: d beta and
+                                         // rAA of the column groups that the upper lanes take
     __shared__ float sdg[C], skd[C], swp[kBwdCompute / 32], scol[2][kBwdCompute / 64][C];
 
     const int tid = threadIdx.x, wg = tid >> 7, l = tid & 127, lane = tid & 31, wq = (tid >> 5) & 3;
@@ -501,6 +502,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 tma_store_commit();
                 tc_fence_after();
                 umma_product<false, false>(T6, adW, 16384, aMt, 8192, C, C, false);         // dW<-^T M         [i][s]
+                umma_product<false, false>(T7, aX - 8192, 8192, aK, 8192, C, D, false);     // X K^T once more, rows r on lanes 64 + r
             }
             nb_sync(kNbDTb, kBwdThreads);
             if (lead) {
@@ -512,6 +514,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             if (lead) {
                 tc_fence_after();
                 umma_product<false, true>(T2, aMt, 8192, aN, 8192, C, C, false, true);      // dA = -M^T N~     [r][s]
+                umma_product<false, true>(T3, aMt - 8192, 8192, aN, 8192, C, C, false, true);   // once more, rows r on lanes 64 + r
                 umma_commit(&bm_4);
             }
             nb_sync(kNbDXK, kBwdThreads);
@@ -659,6 +662,31 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     tc_fence_before();
     nb_arrive(kNbDV, kBwdThreads);
     QD_CLK(4);
+    float* sAA = reinterpret_cast<float*>(sm + oAA);
+    // One group of 8 columns of the dA epilogue for row r; tA = dA, tX = X K^T, both with row r on this thread's lane.
+    auto dA_group = [&](uint32_t tA, uint32_t tX, int g8, int r, float& db, float& rAA) {
+        const float gr = sg[r], br = sbeta[r];
+        const int cb = c0 + g8 * 8;
+        float da[8], xk[8];
+        ld8(my(tA) + g8 * 8, da);
+        ld8(my(tX) + g8 * 8, xk);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int s = cb + e;
+            const bool on = s < r;
+            const float gm = on ? __expf(gr - sg[s]) : 0.f;
+            const float d = on ? da[e] : 0.f;
+            const float dgx = d * gm * xk[e];
+            db += dgx;
+            const float aa = br * dgx;
+            rAA += aa;
+            sts32(&sAA[r * LDAA + s], aa);
+            da[e] = d * br * gm;                               // dXK
+        }
+        sts128(sm + odXK + sw128_chunk(r, wg * kG8 + g8), pack8(da));
+    };
+    static_assert(kG8 == 2, "the dA epilogue gives one column group to each half of a warpgroup");
     // From here to the column sums the two halves of every warpgroup go separate ways.  Lanes 64..127 (whose rows
     // of the 64-row accumulators are padding) take dP, whose product was issued with its rows on their lanes; lanes
     // 0..63 walk the dependent chain dT -> N~ -> dA -> dXK.  Both raise every barrier of the chain exactly once.
@@ -690,6 +718,13 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             sts128(sm + odPG + sw128_chunk(r, ck), pack8(pg));
         }
         srow[0][wg][r] = rPP;
+        // second column group of the dA epilogue, from the copies of dA and X K^T whose rows lie on these lanes
+        wait(&bm_4, ph);
+        tc_fence_after();
+        float db = 0.f, rAA = 0.f;
+        dA_group(T3, T7, 1, r, db, rAA);
+        srow[4][wg][r] = db;
+        srow[5][wg][r] = rAA;
     } else {
     wait(&bm_2, ph);
     tc_fence_after();
@@ -743,33 +778,10 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     wait(&bm_4, ph);
     tc_fence_after();
     QD_CLK(9);
-    float* sAA = reinterpret_cast<float*>(sm + oAA);
-    if (l < C) {
+    {
         const int r = l;
-        const float gr = sg[r], br = sbeta[r];
         float rAA = 0.f, db = 0.f;
-#pragma unroll
-        for (int g8 = 0; g8 < kG8; ++g8) {
-            const int cb = c0 + g8 * 8;
-            float da[8], xk[8];
-            ld8(my(T2) + g8 * 8, da);
-            ld8(my(T0) + g8 * 8, xk);
-            tmem_ld_wait();
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int s = cb + e;
-                const bool on = s < r;
-                const float gm = on ? __expf(gr - sg[s]) : 0.f;
-                const float d = on ? da[e] : 0.f;
-                const float dgx = d * gm * xk[e];
-                db += dgx;
-                const float aa = br * dgx;
-                rAA += aa;
-                sts32(&sAA[r * LDAA + s], aa);
-                da[e] = d * br * gm;                               // dXK
-            }
-            sts128(sm + odXK + sw128_chunk(r, wg * kG8 + g8), pack8(da));
-        }
+        dA_group(T2, T0, 0, r, db, rAA);
         srow[1][wg][r] += db;
         srow[3][wg][r] = rAA;
     }
@@ -813,7 +825,9 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         for (int w4 = 0; w4 < kBwdCompute / 64; ++w4) { cAA += scol[0][w4][r]; cPP += scol[1][w4][r]; }
         float rPP = 0.f, t2 = 0.f, rAA = 0.f, dbt = 0.f;
 #pragma unroll
-        for (int w4 = 0; w4 < kNWG; ++w4) { rPP += srow[0][w4][r]; dbt += srow[1][w4][r]; t2 += srow[2][w4][r]; rAA += srow[3][w4][r]; }
+        for (int w4 = 0; w4 < kNWG; ++w4) {
+            rPP += srow[0][w4][r]; dbt += srow[1][w4][r] + srow[4][w4][r]; t2 += srow[2][w4][r]; rAA += srow[3][w4][r] + srow[5][w4][r];
+        }
         dg_pre = rPP - cPP + t2 + rAA - cAA - kd;
         skd[r] = kd;                            // summed below into dg of the last token
         p.dbeta[(row0 + r) * p.H + hh] = dbt;
