@@ -481,19 +481,17 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 umma_product<false, true>(T1, adO - 8192, 8192, aDt, 8192, C, D, false);    // dO Delta^T [r][s], rows r on lanes 64 + r
                 umma_product<true, false>(T4, aH, 16384, adO, 8192, C, D, false);           // h dO^T           [i][r]
                 umma_commit(&bm_c);                 // from here on no product reads dO or h any more
-                umma_product<true, true>(T5, adH, 16384, aDt, 8192, C, D, false);           // dh Delta^T       [i][s]
                 if (next_id < p.total) prefetch_late(next_id);
             }
             nb_sync(kNbX, kBwdThreads);                                  // X has been built
-            if (lead) {
-                tc_fence_after();
-                umma_product<false, false>(T0, aX, 8192, aK, 8192, C, D, false);            // X K^T            [r][i]
-            }
             nb_sync(kNbDW, kBwdThreads);                                 // the dW<-^T tile is complete
             if (lead) {
                 tc_fence_after();
+                // the product that the dependent chain waits for goes first, the two that are needed late after it
                 umma_product<false, true>(T3, aX, 8192, adW, 8192, C, D, false);            // X dW<-^T         [s][r]
                 umma_commit(&bm_2);
+                umma_product<true, true>(T5, adH, 16384, aDt, 8192, C, D, false);           // dh Delta^T       [i][s]
+                umma_product<false, false>(T0, aX, 8192, aK, 8192, C, D, false);            // X K^T            [r][i]
             }
             nb_sync(kNbDV, kBwdThreads);                                 // the dv staging tile is complete, T6 has been read
             if (lead) {
