@@ -352,6 +352,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int s_abort, s_latch;
     __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C], segc[C];
+    __shared__ float4 scf[C];         // per token: {gamma beta, gamma_C / gamma, gamma, lambda}, one load in the last epilogue
     __shared__ float sred[3][4][C];   // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
     __shared__ float srow[6][kNWG][C];   // per-row partial sums over each warpgroup's columns: rPP, d beta, t2, rAA; [4], [5]: d beta and
                                          // rAA of the column groups that the upper lanes take
@@ -579,7 +580,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         sgam[tid] = __expf(cf_g);
     }
     csync();
-    if (tid < C) segc[tid] = __expf(sg[C - 1] - sg[tid]);
+    if (tid < C) {
+        const float ec = __expf(sg[C - 1] - sg[tid]);
+        segc[tid] = ec;
+        scf[tid] = make_float4(sgam[tid] * sbeta[tid], ec, sgam[tid], slam[tid]);
+    }
     wait(&bar_load, ph);
     wait(&bar_late, ph);
     QD_CLK(1);
@@ -853,10 +858,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 const int t = cb + e;
-                const float dxe = fmaf(sgam[t] * sbeta[t], dx[e], v[e]);                   // dX^T[i][t]
-                sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(w[e] + segc[t] * u[e] + dxe));
-                const float q1 = sgam[t] * z[e];
-                sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(q1 + y[e] + slam[t] * dxe));
+                const float4 cf = scf[t];
+                const float dxe = fmaf(cf.x, dx[e], v[e]);                                  // dX^T[i][t]
+                sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(w[e] + cf.y * u[e] + dxe));
+                const float q1 = cf.z * z[e];
+                sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(q1 + y[e] + cf.w * dxe));
                 const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(t, i & 63)));
                 z[e] = q1 * qv;
                 dx[e] = dxe * qv;
