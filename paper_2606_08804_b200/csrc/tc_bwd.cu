@@ -295,7 +295,7 @@ struct ChunkBwdParams {
 // shared-memory map of k_tc_chunk_bwd (bytes from the 1024-aligned base)
 constexpr int oQ = 0, oK = 16384, oV = 32768, odO = 49152, oX = 65536, oMt = 81920, oP = 90112, oDt = 98304,
               odDt = 114688, oH = 131072, odH = 163840;                            // TMA-loaded tiles (X is built)
-constexpr int kBwdEarlyBytes = 3 * 16384 + 2 * 8192;
+constexpr int kBwdEarlyBytes = 2 * 16384 + 2 * 8192;
 // tiles built later reuse regions whose contents are dead by then
 constexpr int odPG = oV, odTb = oV + 8192, odW = 196608, oN = oH, odXK = oH + 8192, oPP = oH + 16384,
               oAA = odH + 1024, oStDv = odDt, oStDk = oDt, oStDq = odDt;
@@ -351,7 +351,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     __shared__ uint64_t bar_load, bar_late, bm_a, bm_b, bm_c, bm_2, bm_3, bm_4, bm_5;
     __shared__ uint32_t tmem_slot;
     __shared__ volatile int s_abort, s_latch;
-    __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C], segc[C];
+    __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C];
     __shared__ float4 scf[C];         // per token: {gamma beta, gamma_C / gamma, gamma, lambda}, one load in the last epilogue
     __shared__ float sred[3][4][C];   // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
     __shared__ float srow[6][kNWG][C];   // per-row partial sums over each warpgroup's columns: rPP, d beta, t2, rAA; [4], [5]: d beta and
@@ -380,7 +380,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     const uint32_t lane_base = (uint32_t)wq * 32;
     auto my = [&](uint32_t t) { return tmem_addr(t, lane_base, (uint32_t)c0); };
 
-    // The tiles of a chunk arrive in two groups.  "early": K, V, dO, M^T, P -- their regions are dead once the
+    // The tiles of a chunk arrive in two groups.  "early": V, dO, M^T, P -- their regions are dead once the
     // last products of the previous chunk have finished; "late": Q, Delta^T, dDelta^T, h^T, dh^T -- regions
     // that the previous chunk uses up to its end (staging tiles of the stores, scratch of the reductions).
     auto issue_early = [&](int ch) {
@@ -389,14 +389,13 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         const int ym = (int)(((size_t)bh_ * p.N + n_) * C);
         mbar_expect_tx(&bar_load, kBwdEarlyBytes);
         for (int blk = 0; blk < 2; ++blk) {
-            tma_load_2d(sm + oK + blk * 8192, &mapK, hh_ * D + blk * 64, yi, &bar_load);
             tma_load_2d(sm + oV + blk * 8192, &mapV, hh_ * D + blk * 64, yi, &bar_load);
             tma_load_2d(sm + odO + blk * 8192, &mapdO, hh_ * D + blk * 64, yi, &bar_load);
         }
         tma_load_2d(sm + oMt, &mapMt, 0, ym, &bar_load);
         tma_load_2d(sm + oP, &mapP, 0, yt, &bar_load);
     };
-    // The late group goes in three batches as its regions fall free: part 0 = Q (after the last epilogue),
+    // The late group goes in three batches as its regions fall free: part 0 = Q, K (after the last epilogue),
     // part 1 = h^T, dh^T (after the last products and the column sums have read the scratch that aliases them), part 2 = Delta^T,
     // dDelta^T (after the stores have read the staging tiles).  Only the last batch arrives on the barrier.
     auto issue_late = [&](int ch, int part) {
@@ -404,8 +403,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         const int yi = (int)((size_t)b_ * p.T + (size_t)n_ * C);
         const int yc = (int)(((size_t)bh_ * p.N + n_) * D);
         if (part == 0) {
-            mbar_expect_tx_only(&bar_late, 16384);
-            for (int blk = 0; blk < 2; ++blk) tma_load_2d(sm + oQ + blk * 8192, &mapQ, hh_ * D + blk * 64, yi, &bar_late);
+            mbar_expect_tx_only(&bar_late, 2 * 16384);
+            for (int blk = 0; blk < 2; ++blk) {
+                tma_load_2d(sm + oQ + blk * 8192, &mapQ, hh_ * D + blk * 64, yi, &bar_late);
+                tma_load_2d(sm + oK + blk * 8192, &mapK, hh_ * D + blk * 64, yi, &bar_late);
+            }
         } else if (part == 1) {
             mbar_expect_tx_only(&bar_late, 2 * 32768);
             for (int blk = 0; blk < 2; ++blk) {
@@ -426,6 +428,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         const int yc = (int)(((size_t)bh_ * p.N + n_) * D);
         for (int blk = 0; blk < 2; ++blk) {
             tma_prefetch_2d(&mapQ, hh_ * D + blk * 64, yi);
+            tma_prefetch_2d(&mapK, hh_ * D + blk * 64, yi);
             tma_prefetch_2d(&mapHs, blk * 64, yc);
             tma_prefetch_2d(&mapdHs, blk * 64, yc);
         }
@@ -475,7 +478,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 tc_fence_after();
                 umma_product<true, true>(T3, aH, 16384, adDt, 8192, C, D, false, true);     // -h dDelta^T      [i][r] = dW<-^T
                 umma_commit(&bm_a);
-                umma_product<false, false>(T7, adH, 16384, aK, 8192, C, D, false);          // dh^T K^T         [j][s]
                 umma_product<false, false>(T6, adDt, 16384, aMt, 8192, C, C, false);        // dDelta^T M       [j][s]
                 umma_product<false, true>(T2, aV, 8192, adDt, 8192, C, D, false);           // V dDelta^T       [s][r]
                 umma_commit(&bm_b);                 // from here on no product reads V or dDelta^T any more
@@ -493,6 +495,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 umma_commit(&bm_2);
                 umma_product<true, true>(T5, adH, 16384, aDt, 8192, C, D, false);           // dh Delta^T       [i][s]
                 umma_product<false, false>(T0, aX, 8192, aK, 8192, C, D, false);            // X K^T            [r][i]
+                umma_product<false, false>(T7, aX - 8192, 8192, aK, 8192, C, D, false);     // once more, rows r on lanes 64 + r
             }
             nb_sync(kNbDV, kBwdThreads);                                 // the dv staging tile is complete, T6 has been read
             if (lead) {
@@ -501,7 +504,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 tma_store_commit();
                 tc_fence_after();
                 umma_product<false, false>(T6, adW, 16384, aMt, 8192, C, C, false);         // dW<-^T M         [i][s]
-                umma_product<false, false>(T7, aX - 8192, 8192, aK, 8192, C, D, false);     // X K^T once more, rows r on lanes 64 + r
             }
             nb_sync(kNbDTb, kBwdThreads);
             if (lead) {
@@ -527,7 +529,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 tma_store_wait_read();                                   // the dv staging tile may be reused now
                 mbar_arrive(&bm_5);
                 wait(&bm_5, ph);
-                // K, V, dO, M^T, P of this chunk are dead: fetch the next chunk's
+                // V, dO, M^T, P of this chunk are dead: fetch the next chunk's
                 if (next_id < p.total && !s_abort) issue_early(next_id);
             }
             nb_sync(kNbScr, kBwdThreads);                                // the column sums have read the scratch over h^T, dh^T
@@ -582,7 +584,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     csync();
     if (tid < C) {
         const float ec = __expf(sg[C - 1] - sg[tid]);
-        segc[tid] = ec;
         scf[tid] = make_float4(sgam[tid] * sbeta[tid], ec, sgam[tid], slam[tid]);
     }
     wait(&bar_load, ph);
@@ -642,19 +643,10 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         unsigned char* stg = sm + oStDv + (l >> 6) * 8192;
 #pragma unroll
         for (int g8 = 0; g8 < kG8; ++g8) {
-            const int cb = c0 + g8 * 8, ck = wg * kG8 + g8;
-            float kd[8], dvv[8];
-            ld8(my(T7) + g8 * 8, kd);
+            const int cb = c0 + g8 * 8;
+            float dvv[8];
             ld8(my(T6) + g8 * 8, dvv);
             tmem_ld_wait();
-            // <(K-> dh)_s, Delta_s>: (K-> dh)^T[j][s] = gamma_C/gamma_s (dh^T K^T)[j][s] in fp32, times Delta^T[j][s];
-            // the sum over j runs across lanes
-            float dl[8];
-            load8(sm + oDt + sw128_chunk(l, ck), dl);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) kd[e] *= segc[cb + e] * dl[e];
-            const float ksum = col_reduce8(kd, lane);
-            if ((lane & 3) == 0) sred[0][wq][cb + col8_of_lane(lane)] = ksum;
             // dV^T row j = l scaled by beta_s into the staging tile
 #pragma unroll
             for (int e = 0; e < 8; ++e)
@@ -715,7 +707,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 const float dp = (s <= r) ? v[e] : 0.f;
                 const float pp = dp * pv[e];
                 rPP += pp;
-                sts32(&sPP[r * LDAA + s], pp);
+                sts32(&sPP[r * C + ((s + r) & (C - 1))], pp);   // rotated rows: 64 x 64 floats fit the h^T half exactly
                 pg[e] = (s <= r) ? dp * __expf(gr - sg[s]) : 0.f;
             }
             sts128(sm + odPG + sw128_chunk(r, ck), pack8(pg));
@@ -804,7 +796,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
 #pragma unroll
         for (int k = 0; k < kRows; ++k) {
             cA += sAAc[(part * kRows + k) * LDAA + r];
-            cP += sPP[(part * kRows + k) * LDAA + r];
+            cP += sPP[(part * kRows + k) * C + ((r + part * kRows + k) & (C - 1))];
         }
         scol[0][part][r] = cA;
         scol[1][part][r] = cP;
@@ -821,9 +813,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     float dg_pre = 0.f;
     if (tid < C) {
         const int r = tid;
-        float kd = 0.f, cAA = 0.f, cPP = 0.f;
-#pragma unroll
-        for (int w4 = 0; w4 < 4; ++w4) kd += sred[0][w4][r];
+        float cAA = 0.f, cPP = 0.f;
 #pragma unroll
         for (int w4 = 0; w4 < kBwdCompute / 64; ++w4) { cAA += scol[0][w4][r]; cPP += scol[1][w4][r]; }
         float rPP = 0.f, t2 = 0.f, rAA = 0.f, dbt = 0.f;
@@ -831,8 +821,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         for (int w4 = 0; w4 < kNWG; ++w4) {
             rPP += srow[0][w4][r]; dbt += srow[1][w4][r] + srow[4][w4][r]; t2 += srow[2][w4][r]; rAA += srow[3][w4][r] + srow[5][w4][r];
         }
-        dg_pre = rPP - cPP + t2 + rAA - cAA - kd;
-        skd[r] = kd;                            // summed below into dg of the last token
+        dg_pre = rPP - cPP + t2 + rAA - cAA;
         p.dbeta[(row0 + r) * p.H + hh] = dbt;
     }
     if (next_id < p.total) fetch_coef(next_id);
@@ -844,6 +833,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         unsigned char* stk = sm + oStDk + (i >> 6) * 8192;
         unsigned char* stq = sm + oStDq + (i >> 6) * 8192;
         const unsigned char* qcol = sm + oQ + (i >> 6) * 8192;
+        const unsigned char* kcol = sm + oK + (i >> 6) * 8192;
 #pragma unroll
         for (int g8 = 0; g8 < kG8; ++g8) {
             const int cb = c0 + g8 * 8;
@@ -860,16 +850,20 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 const int t = cb + e;
                 const float4 cf = scf[t];
                 const float dxe = fmaf(cf.x, dx[e], v[e]);                                  // dX^T[i][t]
-                sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(w[e] + cf.y * u[e] + dxe));
+                const float kh = cf.y * u[e];                                               // (K-> ^T applied to dh Delta^T)[i][t]
+                sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(w[e] + kh + dxe));
+                // <(K-> dh)_t, Delta_t> = gamma_C/gamma_t sum_i K[t][i] (dh Delta^T)[i][t], all of it in fp32
+                u[e] = kh * __bfloat162float(*reinterpret_cast<const bf16*>(kcol + sw128_off(t, i & 63)));
                 const float q1 = cf.z * z[e];
                 sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(q1 + y[e] + cf.w * dxe));
                 const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(t, i & 63)));
                 z[e] = q1 * qv;
                 dx[e] = dxe * qv;
             }
-            const float dls = col_reduce8(dx, lane), t1s = col_reduce8(z, lane);
+            const float dls = col_reduce8(dx, lane), t1s = col_reduce8(z, lane), kds = col_reduce8(u, lane);
             if ((lane & 3) == 0) {
                 const int col = cb + col8_of_lane(lane);
+                sred[0][wq][col] = kds;
                 sred[1][wq][col] = dls;
                 sred[2][wq][col] = t1s;
             }
@@ -883,10 +877,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     // ---- decay gradient ----------------------------------------------------------------------------
     if (tid < C) {
         const int r = tid;
-        float dl = 0.f, t1 = 0.f;
+        float kd = 0.f, dl = 0.f, t1 = 0.f;
 #pragma unroll
-        for (int w4 = 0; w4 < 4; ++w4) { dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
-        sdg[r] = t1 + dg_pre;
+        for (int w4 = 0; w4 < 4; ++w4) { kd += sred[0][w4][r]; dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
+        sdg[r] = t1 + dg_pre - kd;
+        skd[r] = kd;                            // summed below into dg of the last token
         if (p.dlam) p.dlam[(row0 + r) * p.H + hh] = dl;
     }
     csync();
