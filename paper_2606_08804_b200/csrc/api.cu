@@ -100,14 +100,13 @@ extern "C" {
 
 size_t qdelta_chunk_workspace_bytes(const qd_shape* shape, int for_backward) {
     if (check_shape(shape) != QD_OK) return 0;
-    WsLayout L = ws_layout(*shape);
-    size_t n = for_backward ? L.bwd_end : L.fwd_end;
+    // the tensor-core path and the fp32 path lay the workspace out differently; a shape takes exactly one of them
     if (tc_supported(*shape)) {
         TcLayout TL = tc_layout(*shape);
-        const size_t m = for_backward ? TL.bwd_end : TL.fwd_end;
-        if (m > n) n = m;
+        return for_backward ? TL.bwd_end : TL.fwd_end;
     }
-    return n;
+    WsLayout L = ws_layout(*shape);
+    return for_backward ? L.bwd_end : L.fwd_end;
 }
 
 int qdelta_chunk_fwd(const qd_shape* shape, const void* q, const void* k, const void* v, const void* beta,
@@ -127,14 +126,13 @@ int qdelta_chunk_fwd(const qd_shape* shape, const void* q, const void* k, const 
     a.s = *shape;
     a.L = ws_layout(*shape);
     a.save = (flags & QD_FWD_SAVE_FOR_BWD) != 0;
-    if (!workspace || workspace_bytes < (a.save ? a.L.bwd_end : a.L.fwd_end)) return QD_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < qdelta_chunk_workspace_bytes(shape, a.save ? 1 : 0)) return QD_ERR_WORKSPACE;
     a.q = q; a.k = k; a.v = v; a.beta = beta; a.alpha = alpha; a.lam = lambda; a.h0 = h0; a.o = o; a.hT = hT;
     a.ws = (char*)workspace;
     a.stream = (cudaStream_t)stream;
-    if (cudaMemsetAsync(a.ws + a.L.status, 0, 256, a.stream) != cudaSuccess) return QD_ERR_CUDA;
+    if (cudaMemsetAsync(a.ws + a.L.status, 0, 256, a.stream) != cudaSuccess) return QD_ERR_CUDA;   // offset 0 in both layouts
     if (tc_supported(*shape)) {
         a.TL = tc_layout(*shape);
-        if (workspace_bytes < (a.save ? a.TL.bwd_end : a.TL.fwd_end)) return QD_ERR_WORKSPACE;
         if (timed(ST_PREP, a.stream, [&] { return tc_prep(a); }) != cudaSuccess) return QD_ERR_CUDA;
         if (timed(ST_CHAIN_FWD, a.stream, [&] { return tc_chain_fwd(a); }) != cudaSuccess) return QD_ERR_CUDA;
         return QD_OK;
@@ -166,7 +164,7 @@ int qdelta_chunk_bwd(const qd_shape* shape, const void* q, const void* k, const 
     a.s = *shape;
     a.L = ws_layout(*shape);
     a.save = true;
-    if (!workspace || workspace_bytes < a.L.bwd_end) return QD_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes < qdelta_chunk_workspace_bytes(shape, 1)) return QD_ERR_WORKSPACE;
     a.q = q; a.k = k; a.v = v; a.beta = beta; a.alpha = alpha; a.lam = lambda; a.h0 = h0;
     a.dO = dO; a.dhT = dhT; a.dq = dq; a.dk = dk; a.dv = dv;
     a.dbeta = dbeta; a.dalpha = dalpha; a.dlam = dlambda; a.dh0 = dh0;
@@ -174,7 +172,6 @@ int qdelta_chunk_bwd(const qd_shape* shape, const void* q, const void* k, const 
     a.stream = (cudaStream_t)stream;
     if (tc_supported(*shape)) {
         a.TL = tc_layout(*shape);
-        if (workspace_bytes < a.TL.bwd_end) return QD_ERR_WORKSPACE;
         if (!(flags & QD_BWD_REUSE_FWD)) {
             // recompute what a saving forward leaves behind; its o goes to the dDelta section, which
             // the reverse chain overwrites afterwards
