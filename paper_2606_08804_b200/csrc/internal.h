@@ -56,6 +56,19 @@ struct TcLayout {
 TcLayout tc_layout(const qd_shape& s);
 bool tc_supported(const qd_shape& s);
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may begin before the previous kernel of the
+// stream has finished and orders itself with grid_dep_wait() (see sm100.cuh).
+template <class... KArgs, class... Args>
+cudaError_t launch_overlapped(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 struct ChunkArgs {
     qd_shape s;
     const void *q, *k, *v, *beta, *alpha, *lam;

@@ -49,6 +49,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32
     return false;
 }
 
+// ---- programmatic dependent launch ------------------------------------------------------------------------------
+// A kernel launched with cudaLaunchAttributeProgrammaticStreamSerialization may begin while the kernel before it in
+// the stream is still running.  grid_dep_wait() returns once that kernel has completed and its writes are visible
+// (at once if the launch had no such relation); everything before it may only touch data that is older than the
+// preceding kernel.  grid_dep_launch() lets the kernel after this one begin; the kernels here call it right after
+// their own wait, so a kernel that has begun can rely on everything up to its predecessor's predecessor.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- fences ------------------------------------------------------------------------------------
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA, UMMA operand reads)
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }

@@ -131,6 +131,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
 #pragma unroll
             for (int i = 0; i < 32; ++i) dh[i] = 0.f;
         }
+        grid_dep_wait();                  // the loads of dhT (an input) are in flight; everything below depends on earlier kernels
+        grid_dep_launch();
         // my 32 columns of the operand tile: 64-column block wg >> 1, 16-byte chunks 4 (wg & 1) ..
         unsigned char* myH = sdH + (wg >> 1) * 16384;
         const int hc0 = (wg & 1) * 4;
@@ -189,6 +191,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
     } else if (warp == kMmaWarp) {
         // ---------------------------------- MMA-issue warp ----------------------------------
         const bool lead = (tid & 31) == 0;
+        grid_dep_wait();
+        grid_dep_launch();
         const uint32_t adH = smem_u32(sdH), adD = smem_u32(sdD);
         for (int it = 0; it < p.N; ++it) {
             const uint32_t st = smem_u32(smem + (it & 1) * kStage);
@@ -217,6 +221,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
     } else {
         // ---------------------------------- TMA warp ----------------------------------
         const bool lead = (tid & 31) == 0;
+        grid_dep_wait();
+        grid_dep_launch();
         // iteration `it` processes chunk n = N-1-it
         auto issue_load = [&](int it) {
             const int n = p.N - 1 - it;
@@ -463,9 +469,22 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         // =============================== issuing warp: TMA copies and MMAs ===============================
         const bool lead = lane == 0;
         if (lead && (int)blockIdx.x < p.total) {
-            issue_early(blockIdx.x);
-            issue_late(blockIdx.x, 0); issue_late(blockIdx.x, 1); issue_late(blockIdx.x, 2);
+            // first chunk: everything that the reverse chain (the kernel before this one) does not write is fetched
+            // before waiting for it -- inputs, and tiles of kernels that had finished before the reverse chain began
+            const int ch = blockIdx.x;
+            const int n_ = ch % p.N, bh_ = ch / p.N;
+            const int yc = (int)(((size_t)bh_ * p.N + n_) * D);
+            issue_early(ch);
+            issue_late(ch, 0);
+            mbar_expect_tx_only(&bar_late, 32768 + 16384);
+            for (int blk = 0; blk < 2; ++blk) tma_load_2d(sm + oH + blk * 16384, &mapHs, blk * 64, yc, &bar_late);
+            tma_load_2d(sm + oDt, &mapDt, 0, yc, &bar_late);
+            grid_dep_wait();
+            mbar_expect_tx(&bar_late, 32768 + 16384);
+            for (int blk = 0; blk < 2; ++blk) tma_load_2d(sm + odH + blk * 16384, &mapdHs, blk * 64, yc, &bar_late);
+            tma_load_2d(sm + odDt, &mapdDt, 0, yc, &bar_late);
         }
+        grid_dep_wait();
         for (int ch_id = blockIdx.x, it = 0; ch_id < p.total; ch_id += gridDim.x, ++it) {
             const int n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
             const int row0 = (int)((size_t)b * p.T + (size_t)n * C);
@@ -562,6 +581,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     // ======================================== epilogue threads ========================================
     auto csync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(kNbC), "r"(kBwdCompute) : "memory"); };   // warps arrive converged
     if ((int)blockIdx.x < p.total) fetch_coef(blockIdx.x);
+    grid_dep_wait();                    // coefficients and log-decays are older than the reverse chain; the results below are not
 
     for (int ch_id = blockIdx.x, it = 0; ch_id < p.total; ch_id += gridDim.x, ++it) {
     const int n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
@@ -946,8 +966,8 @@ cudaError_t tc_chain_bwd(const ChunkArgs& a) {
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_chain_bwd, kChainSmem);
     if (e != cudaSuccess) return e;
-    k_tc_chain_bwd<<<(unsigned)BH, kChainThreads, kChainSmem, a.stream>>>(mWt, mdO, mQg, mK, mP, mdHs, mdDt, p);
-    return cudaGetLastError();
+    return launch_overlapped(k_tc_chain_bwd, dim3((unsigned)BH), dim3(kChainThreads), kChainSmem, a.stream,
+                             mWt, mdO, mQg, mK, mP, mdHs, mdDt, p);
 }
 
 cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
@@ -985,9 +1005,8 @@ cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     const unsigned grid = (unsigned)std::min<uint64_t>(BH * N, (uint64_t)sms);
-    k_tc_chunk_bwd<<<grid, kBwdThreads, kBwdSmem, a.stream>>>(mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs,
-                                                                               mdQ, mdK, mdV, p);
-    return cudaGetLastError();
+    return launch_overlapped(k_tc_chunk_bwd, dim3(grid), dim3(kBwdThreads), kBwdSmem, a.stream, mQ, mK, mV, mdO, mMt, mP,
+                             mDt, mdDt, mHs, mdHs, mdQ, mdK, mdV, p);
 }
 
 }  // namespace qd

@@ -101,6 +101,7 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     const uint32_t tbase = tmem_slot;
 
     QD_TL(0);
+    grid_dep_launch();                // the kernel after this one may set itself up while the last CTAs of this one run
     if (tid == 0) {
         mbar_expect_tx(&bar_load, 3 * 32768);
         const int y = (int)tok0;
@@ -440,6 +441,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
 #pragma unroll
             for (int i = 0; i < 32; ++i) h[i] = 0.f;
         }
+        grid_dep_wait();                  // the loads of h0 (an input) are in flight; everything below depends on the prep kernel
+        grid_dep_launch();
         // my 32 columns of the operand tile: 64-column block wg >> 1, 16-byte chunks 4 (wg & 1) ..
         unsigned char* myH = sH + (wg >> 1) * 16384;
         const int hc0 = (wg & 1) * 4;
@@ -548,6 +551,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
     } else if (warp == kMmaWarp) {
         // ---------------------------------- MMA-issue warp ----------------------------------
         const bool lead = (tid & 31) == 0;
+        grid_dep_wait();
+        grid_dep_launch();
         const uint32_t aH = smem_u32(sH), aD = smem_u32(sD), aDs = smem_u32(sDs);
         for (int n = 0; n < p.N; ++n) {
             const uint32_t st = smem_u32(smem + (n & 1) * kStage);
@@ -586,6 +591,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
     } else {
         // ---------------------------------- TMA warp ----------------------------------
         const bool lead = (tid & 31) == 0;
+        grid_dep_wait();                  // the tiles and the log-decays read below are written by the prep kernel
+        grid_dep_launch();
         auto issue_load = [&](int n) {
             unsigned char* st = smem + (n & 1) * kStage;
             uint64_t* bar = &bar_load[n & 1];
@@ -749,8 +756,8 @@ cudaError_t tc_chain_fwd(const ChunkArgs& a) {
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_chain_fwd, kChainSmem);
     if (e != cudaSuccess) return e;
-    k_tc_chain_fwd<<<(unsigned)BH, kChainThreads, kChainSmem, a.stream>>>(mWt, mUt, mQg, mK, mP, mHs, mDt, mO, p);
-    return cudaGetLastError();
+    return launch_overlapped(k_tc_chain_fwd, dim3((unsigned)BH), dim3(kChainThreads), kChainSmem, a.stream,
+                             mWt, mUt, mQg, mK, mP, mHs, mDt, mO, p);
 }
 
 }  // namespace qd
