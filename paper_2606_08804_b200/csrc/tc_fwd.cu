@@ -65,7 +65,7 @@ __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u6
 //   scan / coefficients   thread t < 128 owns token t
 //   row-wise elementwise  16 threads per 256-byte row (coalesced), 16 rows per pass
 //   Gram epilogue         thread (row = t & 127, half = t >> 7) owns 32 columns of its TMEM lane
-//   triangular inverse    lane pair (t >> 1, t < 128) owns columns j0 < 32 and j0 + 32 of one chunk, parity t & 1 the 8-row blocks
+//   triangular inverse    lane quad (t >> 2, t < 128) owns columns j0 + 16 k (j0 < 16) of one chunk, quad lane t & 3 the 8-row blocks t & 3 and (t & 3) + 4
 //   final epilogue        thread (d = t & 127, which = t >> 7) owns one row of U~^T resp. W~^T
 __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
                                                              const __grid_constant__ CUtensorMap mapK,
@@ -227,44 +227,44 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     tc_fence_before();
     __syncthreads();
     QD_TL(5);
-    // M_c = (I + A_c)^-1 by right-looking substitution, columns in registers.  A lane pair of the first four warps
-    // owns two columns of one chunk, j0 < 32 and j1 = j0 + 32 (the same loads of A serve both); the lane of parity
-    // `par` owns the 8-row blocks 2s + par.  Once m[i] is final its owner hands it to the partner lane and every
-    // later row gets its update m[r] -= A[r][i] m[i]; rows <= i of a block see A = 0 exactly.  Column j1 is zero
-    // above row 32, so it joins at step 32 and keeps only its blocks 4..7.  The loads of A are warp-wide
-    // broadcasts, and shared-memory wavefronts are what bounds this phase: hence two columns per load.
-    const int q = tid >> 1, par = tid & 1, ic = (q >> 5) & 1, j0 = q & 31, j1 = j0 + 32;
-    float m0[4][8], m1[2][8];
+    // M_c = (I + A_c)^-1 by right-looking substitution, columns in registers.  A lane quad of the first four warps
+    // owns four columns of one chunk, j0 + 16 k with j0 < 16 (the same loads of A serve all four); lane `ql` of the
+    // quad owns the 8-row blocks ql and ql + 4.  Once m[i] is final its owner hands it to the other three lanes and
+    // every later row gets its update m[r] -= A[r][i] m[i]; rows <= i of a block see A = 0 exactly, so whole blocks
+    // are updated.  Column j0 + 16 k is zero above row 16 k and joins at step 16 k; blocks 0..3 are final after step
+    // 30.  The loads of A are warp-wide broadcasts, and shared-memory wavefronts are what bounds this phase: hence
+    // four columns per load (32 FMAs for two 16-byte loads).
+    const int qd4 = tid >> 2, ql = tid & 3, ic = (qd4 >> 4) & 1, j0 = qd4 & 15;
+    float m[2][4][8];
     if (tid < 128) {
-        const float* Ac = sA + ic * C * C + par * 8;
+        const float* Ac = sA + ic * C * C + ql * 8;
 #pragma unroll
-        for (int s = 0; s < 4; ++s)
+        for (int sb = 0; sb < 2; ++sb)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) m0[s][e] = ((2 * s + par) * 8 + e == j0) ? 1.f : 0.f;
+            for (int k = 0; k < 4; ++k)
 #pragma unroll
-        for (int s = 0; s < 2; ++s)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) m1[s][e] = ((2 * s + 4 + par) * 8 + e == j1) ? 1.f : 0.f;
+                for (int e = 0; e < 8; ++e) m[sb][k][e] = ((ql + 4 * sb) * 8 + e == j0 + 16 * k) ? 1.f : 0.f;
 #pragma unroll
         for (int i = 0; i < C - 1; ++i) {
-            const int src = (lane & ~1) | ((i >> 3) & 1);
-            const float mi0 = __shfl_sync(0xffffffffu, m0[i >> 4][i & 7], src);
-            float mi1 = 0.f;
-            if (i >= 32) mi1 = __shfl_sync(0xffffffffu, m1[(i >> 4) - 2][i & 7], src);
+            const int bi = i >> 3;                              // block of the pivot row; its owner is quad lane bi & 3
+            const int src = (lane & ~3) | (bi & 3);
+            float mi[4];
 #pragma unroll
-            for (int s = (i + 1) >> 4; s < 4; ++s) {
-                const float4 a0 = *reinterpret_cast<const float4*>(Ac + i * C + s * 16);
-                const float4 a1 = *reinterpret_cast<const float4*>(Ac + i * C + s * 16 + 4);
-                m0[s][0] = fmaf(-a0.x, mi0, m0[s][0]); m0[s][1] = fmaf(-a0.y, mi0, m0[s][1]);
-                m0[s][2] = fmaf(-a0.z, mi0, m0[s][2]); m0[s][3] = fmaf(-a0.w, mi0, m0[s][3]);
-                m0[s][4] = fmaf(-a1.x, mi0, m0[s][4]); m0[s][5] = fmaf(-a1.y, mi0, m0[s][5]);
-                m0[s][6] = fmaf(-a1.z, mi0, m0[s][6]); m0[s][7] = fmaf(-a1.w, mi0, m0[s][7]);
-                if (i >= 32) {
-                    float* mm = m1[s >= 2 ? s - 2 : 0];
-                    mm[0] = fmaf(-a0.x, mi1, mm[0]); mm[1] = fmaf(-a0.y, mi1, mm[1]);
-                    mm[2] = fmaf(-a0.z, mi1, mm[2]); mm[3] = fmaf(-a0.w, mi1, mm[3]);
-                    mm[4] = fmaf(-a1.x, mi1, mm[4]); mm[5] = fmaf(-a1.y, mi1, mm[5]);
-                    mm[6] = fmaf(-a1.z, mi1, mm[6]); mm[7] = fmaf(-a1.w, mi1, mm[7]);
+            for (int k = 0; k < 4; ++k)
+                mi[k] = (i >= 16 * k) ? __shfl_sync(0xffffffffu, m[bi >> 2][k][i & 7], src) : 0.f;
+#pragma unroll
+            for (int sb = (i < 31 ? 0 : 1); sb < 2; ++sb) {
+                const float4 a0 = *reinterpret_cast<const float4*>(Ac + i * C + sb * 32);
+                const float4 a1 = *reinterpret_cast<const float4*>(Ac + i * C + sb * 32 + 4);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (i >= 16 * k) {
+                        float* mm = m[sb][k];
+                        mm[0] = fmaf(-a0.x, mi[k], mm[0]); mm[1] = fmaf(-a0.y, mi[k], mm[1]);
+                        mm[2] = fmaf(-a0.z, mi[k], mm[2]); mm[3] = fmaf(-a0.w, mi[k], mm[3]);
+                        mm[4] = fmaf(-a1.x, mi[k], mm[4]); mm[5] = fmaf(-a1.y, mi[k], mm[5]);
+                        mm[6] = fmaf(-a1.z, mi[k], mm[6]); mm[7] = fmaf(-a1.w, mi[k], mm[7]);
+                    }
                 }
             }
         }
@@ -277,21 +277,18 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         unsigned char* t1 = sT + 16384 + ic * 8192;
         bf16* mt = p.Mt ? p.Mt + ((size_t)bh * p.N + 2 * pr + ic) * C * C : nullptr;
 #pragma unroll
-        for (int col = 0; col < 2; ++col) {
-            const int j = col ? j1 : j0;
+        for (int k = 0; k < 4; ++k) {
+            const int j = j0 + 16 * k;
             const float beta = sbeta[ic * C + j], bg = beta * __expf(sg[ic * C + j]);
 #pragma unroll
-            for (int s = 0; s < 4; ++s) {
-                const int kb = 2 * s + par;
-                float mv[8], a[8], bq[8];
+            for (int sb = 0; sb < 2; ++sb) {
+                const int kb = ql + 4 * sb;
+                float a[8], bq[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    mv[e] = col ? (s >= 2 ? m1[s >= 2 ? s - 2 : 0][e] : 0.f) : m0[s][e];
-                    a[e] = mv[e] * beta; bq[e] = mv[e] * bg;
-                }
+                for (int e = 0; e < 8; ++e) { a[e] = m[sb][k][e] * beta; bq[e] = m[sb][k][e] * bg; }
                 sts128(t0 + sw128_chunk(j, kb), pack8(a));
                 sts128(t1 + sw128_chunk(j, kb), pack8(bq));
-                if (mt) *reinterpret_cast<uint4*>(mt + (size_t)j * C + kb * 8) = pack8(mv);
+                if (mt) *reinterpret_cast<uint4*>(mt + (size_t)j * C + kb * 8) = pack8(m[sb][k]);
             }
         }
     }
