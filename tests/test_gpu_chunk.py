@@ -168,3 +168,62 @@ def test_tensor_core_forward_regimes(regime):
 def test_tensor_core_forward_single_pair_no_h0():
     cfg = replace(gen.CONFIGS["cfg1"], B=1, H=1, T=128, h0=False, seed=19)
     _fwd_check(cfg)
+
+
+def test_tensor_core_optional_inputs_absent():
+    # bf16, d = 128, T a multiple of 128 (the tcgen05 kernels) with alpha = lambda = h0 = dhT = NULL, each alone and
+    # all together; backward both with its own forward recomputation and on the forward's saved workspace
+    from paper_2606_08804_b200 import binding as qd
+    cfg = replace(gen.CONFIGS["cfg2"], B=2, H=2, T=256, seed=23)
+    d = gen.make_chunk_inputs(cfg)
+    variants = [dict(alpha=None), dict(lam=None), dict(h0=None), dict(dhT=None),
+                dict(alpha=None, lam=None, h0=None, dhT=None)]
+    for drop in variants:
+        d2 = dict(d, **drop)
+        t = gu.dev_inputs(d2, cfg.dtype)
+        ro, rh = gu.oracle_fwd(d2)
+        ref = gu.oracle_bwd(d2)
+        for reuse in (False, True):
+            o, hT, ws = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], save_for_bwd=reuse)
+            g = qd.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], t["dO"], t["dhT"],
+                             workspace=ws if reuse else None, reuse_fwd=reuse)
+            torch.cuda.synchronize()
+            assert qd.workspace_status(ws) == 0
+            assert gu.rel_err(o, ro) <= 2e-2 and gu.rel_err(hT, rh) <= 2e-2, drop
+            for n in ("dq", "dk", "dv", "dbeta", "dalpha", "dlam", "dh0"):
+                if g.get(n) is None:            # d alpha / d lambda of an absent input
+                    continue
+                assert gu.rel_err(g[n], ref[n]) <= 2e-2, (drop, reuse, n)
+            assert (g["dalpha"] is None) == (d2["alpha"] is None) and (g["dlam"] is None) == (d2["lam"] is None)
+
+
+def test_back_to_back_launches_without_host_sync():
+    # The kernels of a step are launched so that each may begin while its predecessor drains.  Many steps in a row on
+    # one workspace, no host synchronisation in between, alternating two input sets: every step's results must equal
+    # the results of the same step run alone.
+    from paper_2606_08804_b200 import binding as qd
+    cfgs = [replace(gen.CONFIGS["cfg2"], B=2, H=3, T=384, seed=s) for s in (31, 32)]
+    ts = [gu.dev_inputs(gen.make_chunk_inputs(c), c.dtype) for c in cfgs]
+
+    def run(t, ws=None, out=None):
+        o, hT, ws = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], save_for_bwd=True,
+                                 workspace=ws)
+        g = qd.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], t["dO"], t["dhT"],
+                         workspace=ws, reuse_fwd=True, out=out)
+        return o, hT, g, ws
+
+    alone = []
+    for t in ts:
+        o, hT, g, _ = run(t)
+        torch.cuda.synchronize()
+        alone.append([o.clone(), hT.clone()] + [g[n].clone() for n in sorted(g)])
+    ws = qd.alloc_workspace(qd.make_shape(ts[0]["q"], ts[0]["v"], 64), True, "cuda")
+    got = []
+    for i in range(12):
+        o, hT, g, _ = run(ts[i & 1], ws)
+        got.append([o, hT] + [g[n] for n in sorted(g)])
+    torch.cuda.synchronize()
+    assert qd.workspace_status(ws) == 0
+    for i, res in enumerate(got):
+        for x, y in zip(res, alone[i & 1]):
+            assert torch.equal(x, y), i
