@@ -73,9 +73,39 @@ def stage_bytes_per_token_head(dk, dv, C):
     }
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu capture summarised in
-# profiles/tc_kernels_dram_traffic_cfg2.md (full-size cfg2); other workloads: not captured
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch: NOT measured by this run (a profiler cannot run inside the
+# timed program); constants from the ncu capture summarised in profiles/tc_kernels_dram_traffic_cfg2.md (full-size
+# cfg2).  Other workloads: not captured.
 NCU_TRAFFIC_BYTES = {"cfg2": {"prep": 421.9e6, "chain_fwd": 532.8e6, "chain_bwd": 469.2e6, "chunk_bwd": 926.2e6}}
+NCU_TRAFFIC_SOURCE = "constant from profiles/tc_kernels_dram_traffic_cfg2.md (ncu, one launch each); not measured by this run"
+# which pass of the path a kernel belongs to (its share of the algorithmic bytes of SURVEY section 8(d))
+STAGE_PASS = {"prep": "fwd", "chain_fwd": "fwd", "chain_bwd": "bwd", "chunk_bwd": "bwd"}
+
+
+def path_roofline(cfg, pk, fwd=True, bwd=True):
+    """Roofline time of the path on one GPU: max(algorithmic bytes / HBM, algorithmic FLOPs / bf16 peak), both for the
+    measured peaks of this machine and for the nominal 8 TB/s and 2.25 PFLOP/s."""
+    th = cfg.B * cfg.T * cfg.H
+    fb, bb = path_bytes_per_token_head(cfg.dk, cfg.dv)
+    ff, fbw = path_flops_per_token_head(cfg.dk, cfg.dv, cfg.chunk)
+    nstates = (2 if fwd else 0) + (2 if bwd else 0)            # h0, hT / dhT, dh0: fp32 [dk x dv] per sequence
+    nbytes = ((fb if fwd else 0) + (bb if bwd else 0)) * th + nstates * cfg.dk * cfg.dv * 4 * cfg.B * cfg.H
+    flops = ((ff if fwd else 0) + (fbw if bwd else 0)) * th
+    t_meas = max(nbytes / (pk["hbm_gbs"] * 1e9), flops / (pk["bf16_tflops"] * 1e12))
+    t_nom = max(nbytes / 8.0e12, flops / 2.25e15)
+    return {"bytes_per_step": nbytes, "flops_per_step": flops, "roofline_ms": t_meas * 1e3, "roofline_ms_nominal": t_nom * 1e3,
+            "bound": "hbm" if nbytes / (pk["hbm_gbs"] * 1e9) >= flops / (pk["bf16_tflops"] * 1e12) else "tensor"}
+
+
+def region_stats(times_ms, steps, mhz):
+    """Median / min / max of repeated K-step regions (ms per step) and the clock-normalised figure."""
+    per = sorted(t / steps for t in times_ms)
+    med = per[len(per) // 2]
+    out = {"regions": len(per), "steps_per_region": steps, "ms_per_step_median": med, "ms_per_step_min": per[0],
+           "ms_per_step_max": per[-1], "spread": (per[-1] - per[0]) / med}
+    if mhz:
+        out["ms_x_mhz_median"] = med * mhz          # time x median SM clock: compares runs taken at different clocks
+    return out
 
 
 class ClockSampler(threading.Thread):
@@ -147,8 +177,79 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
-def workload_name(cfg):
-    return "%s: bf16 fwd+bwd B=%d H=%d T=%d dk=%d dv=%d chunk=%d" % (cfg.name, cfg.B, cfg.H, cfg.T, cfg.dk, cfg.dv, cfg.chunk)
+def workload_name(cfg, backward=True):
+    return "%s: bf16 %s B=%d H=%d T=%d dk=%d dv=%d chunk=%d" % (cfg.name, "fwd+bwd" if backward else "fwd", cfg.B, cfg.H, cfg.T,
+                                                                 cfg.dk, cfg.dv, cfg.chunk)
+
+
+class Workload:
+    """Device-resident inputs, outputs and workspace of one chunkwise configuration, and its step."""
+
+    def __init__(self, torch, qd, gen, cfg, seed, backward=True, drop=()):
+        d = gen.make_chunk_inputs(cfg, seed=seed)
+        bf = torch.bfloat16
+        self.host, self.dev = {}, {}
+        for n in ("q", "k", "v", "beta", "alpha", "lam", "dO"):
+            if d.get(n) is not None:
+                self.host[n] = torch.from_numpy(d[n]).to(bf).pin_memory()
+        for n in ("h0", "dhT"):
+            if d.get(n) is not None:
+                self.host[n] = torch.from_numpy(d[n]).pin_memory()
+        for n, t in self.host.items():
+            self.dev[n] = t.to("cuda", non_blocking=True)
+        for n in ("q", "k", "v", "beta", "alpha", "lam", "dO", "h0", "dhT"):
+            self.dev.setdefault(n, None)
+        for n in drop:                                  # variant runs: the optional input is absent (NULL)
+            self.dev[n] = None
+        self.cfg, self.qd, self.backward = cfg, qd, backward
+        B, T, H, dk, dv = cfg.B, cfg.T, cfg.H, cfg.dk, cfg.dv
+        self.shape = qd.make_shape(self.dev["q"], self.dev["v"], cfg.chunk)
+        self.ws = qd.alloc_workspace(self.shape, backward, "cuda")
+        self.o = torch.empty((B, T, H, dv), dtype=bf, device="cuda")
+        self.hT = torch.empty((B, H, dk, dv), dtype=torch.float32, device="cuda")
+        self.grads = {}
+
+    def step(self):
+        d, qd, cfg = self.dev, self.qd, self.cfg
+        qd.chunk_fwd(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"], chunk=cfg.chunk,
+                     save_for_bwd=self.backward, workspace=self.ws, o=self.o, hT=self.hT)
+        if self.backward:
+            qd.chunk_bwd(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"], d["dO"], d["dhT"],
+                         chunk=cfg.chunk, workspace=self.ws, reuse_fwd=True, out=self.grads)
+
+
+def time_regions(torch, step, steps, regions, barrier):
+    """`regions` back-to-back regions of exactly `steps` steps, each bracketed by CUDA events on the launching stream."""
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(regions)]
+    barrier()
+    for e0, e1 in evs:
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+    barrier()
+    return [e0.elapsed_time(e1) for e0, e1 in evs]
+
+
+def extra_workload(torch, qd, gen, cfg, pk, pk_kind, backward, steps, regions, drop=()):
+    """A further configuration timed like the headline one (rank 0, one GPU): ms per step, tokens/s, roofline fraction."""
+    w = Workload(torch, qd, gen, cfg, cfg.seed, backward=backward, drop=drop)
+    for _ in range(3):
+        w.step()
+    torch.cuda.synchronize()
+    assert qd.workspace_status(w.ws) == 0, "device-side status word is set"
+    times = time_regions(torch, w.step, steps, regions, torch.cuda.synchronize)
+    st = region_stats(times, steps, None)
+    rl = path_roofline(cfg, pk, fwd=True, bwd=backward)
+    ms = st["ms_per_step_median"]
+    out = {"workload": workload_name(cfg, backward), "ms_per_step": ms, "tokens_per_s": cfg.B * cfg.T / (ms * 1e-3),
+           "roofline_ms": rl["roofline_ms"], "frac": rl["roofline_ms"] / ms, "frac_nominal": rl["roofline_ms_nominal"] / ms,
+           "peak_kind": "of " + pk_kind, "regions": st}
+    if drop:
+        out["absent_inputs"] = list(drop)
+    del w
+    torch.cuda.empty_cache()
+    return out
 
 
 def run_ours(args, cfg):
@@ -173,50 +274,25 @@ def run_ours(args, cfg):
         torch.cuda.synchronize()
 
     # ---- inputs: pinned host copies and device copies ------------------------------------------
-    d = gen.make_chunk_inputs(cfg, seed=sharding.rank_seed(cfg.seed, rank))
-    bf, f32 = torch.bfloat16, torch.float32
-    host, dev = {}, {}
-    for n in ("q", "k", "v", "beta", "alpha", "lam", "dO"):
-        host[n] = torch.from_numpy(d[n]).to(bf).pin_memory()
-    for n in ("h0", "dhT"):
-        host[n] = torch.from_numpy(d[n]).pin_memory()
-    for n, t in host.items():
-        dev[n] = t.to("cuda", non_blocking=True)
-    del d
+    w = Workload(torch, qd, gen, cfg, sharding.rank_seed(cfg.seed, rank), backward=True)
+    host, dev, ws, o, hT, grads, step = w.host, w.dev, w.ws, w.o, w.hT, w.grads, w.step
     B, T, H, dk, dv = cfg.B, cfg.T, cfg.H, cfg.dk, cfg.dv
-    shape = qd.make_shape(dev["q"], dev["v"], cfg.chunk)
-    ws = qd.alloc_workspace(shape, True, "cuda")
-    o = torch.empty((B, T, H, dv), dtype=bf, device="cuda")
-    hT = torch.empty((B, H, dk, dv), dtype=f32, device="cuda")
-    grads = {}
-
-    def step():
-        qd.chunk_fwd(dev["q"], dev["k"], dev["v"], dev["beta"], dev["alpha"], dev["lam"], dev["h0"],
-                     chunk=cfg.chunk, save_for_bwd=True, workspace=ws, o=o, hT=hT)
-        qd.chunk_bwd(dev["q"], dev["k"], dev["v"], dev["beta"], dev["alpha"], dev["lam"], dev["h0"],
-                     dev["dO"], dev["dhT"], chunk=cfg.chunk, workspace=ws, reuse_fwd=True, out=grads)
-
-    for _ in range(max(args.warmup, 3)):
+    assert qd.chunk_path(w.shape) == "tensor_core"
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
         step()
     barrier()
     assert qd.workspace_status(ws) == 0, "device-side status word is set"
 
-    # ---- timed region: K steps, CUDA events on the launching stream -------------------------------
-    # The four kernels of a step are launched so that each may set itself up while the one before it drains
-    # (programmatic dependent launch).  Events between the launches would serialise them again, so the per-kernel
-    # durations behind `roofline` come from a second pass over the same K steps, right after the timed one.
+    # ---- timed regions: each is exactly K steps between two CUDA events on the launching stream; `regions` of them
+    # run back to back so that the figure is the sustained one (power cap, clocks settled), the median is reported.
+    # The four kernels of a step are launched so that each may set itself up while the one before it drains; events
+    # between the launches would serialise them, so the per-kernel durations come from a separate pass afterwards.
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.25)
     qd.profile_enable(False)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    barrier()
-    ms = e0.elapsed_time(e1)
+    times = time_regions(torch, step, args.steps, max(1, args.regions), barrier)
     qd.profile_read(reset=True)
     qd.profile_enable(True)
     for _ in range(args.steps):
@@ -224,19 +300,22 @@ def run_ours(args, cfg):
     barrier()
     qd.profile_enable(False)
     stages = qd.profile_read(reset=True)
-    # the timed region lasts milliseconds, nvidia-smi answers in ~0.1 s: keep the same step loop running
-    # (untimed) for a second or so, so that the clock samples are taken under this load
+    # nvidia-smi answers in ~0.1 s: keep the same step loop running (untimed) a little longer so that enough clock
+    # samples are taken under this load
     t_probe = time.perf_counter()
-    while time.perf_counter() - t_probe < 1.5:
+    while time.perf_counter() - t_probe < 1.0:
         for _ in range(20):
             step()
         torch.cuda.synchronize()
     sampler.stop_flag.set()
     sampler.join()
-    ms, tokens_total = sharding.aggregate(ms, B * T * args.steps, "cuda")   # slowest rank, all ranks' tokens
+    clocks = sampler.summary()
+    med_ms = sorted(times)[len(times) // 2]
+    ms, tokens_total = sharding.aggregate(med_ms, B * T * args.steps, "cuda")   # slowest rank, all ranks' tokens
     ms_step = ms / args.steps
     tokens_step = tokens_total // args.steps
     value = sharding.throughput(tokens_total, ms)
+    regions = region_stats(times, args.steps, clocks.get("sm_mhz"))
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region ------------
     out_host = {"o": torch.empty_like(o, device="cpu").pin_memory(), "hT": torch.empty_like(hT, device="cpu").pin_memory()}
@@ -249,94 +328,125 @@ def run_ours(args, cfg):
     # step i computes (PCIe is full duplex).  Every step still uploads all of its inputs and downloads all of
     # its results inside the timed region.
     s_in, s_cmp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
-    dev2 = [dev, {n: torch.empty_like(t) for n, t in dev.items()}]
-    o2, hT2, g2 = [o, torch.empty_like(o)], [hT, torch.empty_like(hT)], [grads, {}]
-    qd.chunk_bwd(dev["q"], dev["k"], dev["v"], dev["beta"], dev["alpha"], dev["lam"], dev["h0"],
-                 dev["dO"], dev["dhT"], chunk=cfg.chunk, workspace=ws, reuse_fwd=True, out=g2[1])   # allocate set 1
-    torch.cuda.synchronize()
-    ev = lambda: torch.cuda.Event()
-    in_done, cmp_done, out_done = {}, {}, {}
-
-    def e2e_step(i):
-        k = i & 1
-        with torch.cuda.stream(s_in):
-            if i - 2 in cmp_done:
-                s_in.wait_event(cmp_done[i - 2])          # the inputs of step i-2 are no longer needed
-            for n, t in host.items():
-                dev2[k][n].copy_(t, non_blocking=True)
-            in_done[i] = ev(); in_done[i].record(s_in)
-        with torch.cuda.stream(s_cmp):
-            s_cmp.wait_event(in_done[i])
-            if i - 2 in out_done:
-                s_cmp.wait_event(out_done[i - 2])         # the results of step i-2 have left the device
-            d = dev2[k]
-            qd.chunk_fwd(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"],
-                         chunk=cfg.chunk, save_for_bwd=True, workspace=ws, o=o2[k], hT=hT2[k])
-            qd.chunk_bwd(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"],
-                         d["dO"], d["dhT"], chunk=cfg.chunk, workspace=ws, reuse_fwd=True, out=g2[k])
-            cmp_done[i] = ev(); cmp_done[i].record(s_cmp)
-        with torch.cuda.stream(s_out):
-            s_out.wait_event(cmp_done[i])
-            out_host["o"].copy_(o2[k], non_blocking=True)
-            out_host["hT"].copy_(hT2[k], non_blocking=True)
-            for n, t in g2[k].items():
-                out_host[n].copy_(t, non_blocking=True)
-            out_done[i] = ev(); out_done[i].record(s_out)
-
     e2e_steps = 0 if args.no_extras else max(4, min(args.steps, 10))
-    for i in range(2 if e2e_steps else 0):
-        e2e_step(i)
-    barrier()
-    in_done.clear(); cmp_done.clear(); out_done.clear()
-    e0.record(s_in)
-    for i in range(e2e_steps):
-        e2e_step(i)
-    e1.record(s_out)
-    barrier()
-    ems = e0.elapsed_time(e1) if e2e_steps else float("nan")
-    ems, _ = sharding.aggregate(ems, 0, "cuda")
-    e2e_value = tokens_step / (ems / e2e_steps * 1e-3) if e2e_steps else None
+    e2e_value = None
+    if e2e_steps:
+        dev2 = [dev, {n: torch.empty_like(t) for n, t in dev.items()}]
+        o2, hT2, g2 = [o, torch.empty_like(o)], [hT, torch.empty_like(hT)], [grads, {}]
+        qd.chunk_bwd(dev["q"], dev["k"], dev["v"], dev["beta"], dev["alpha"], dev["lam"], dev["h0"],
+                     dev["dO"], dev["dhT"], chunk=cfg.chunk, workspace=ws, reuse_fwd=True, out=g2[1])   # allocate set 1
+        torch.cuda.synchronize()
+        ev = lambda: torch.cuda.Event()
+        in_done, cmp_done, out_done = {}, {}, {}
 
-    # ---- roofline of the dominant kernel and of the whole path -----------------------------------
+        def e2e_step(i):
+            k = i & 1
+            with torch.cuda.stream(s_in):
+                if i - 2 in cmp_done:
+                    s_in.wait_event(cmp_done[i - 2])          # the inputs of step i-2 are no longer needed
+                for n, t in host.items():
+                    dev2[k][n].copy_(t, non_blocking=True)
+                in_done[i] = ev(); in_done[i].record(s_in)
+            with torch.cuda.stream(s_cmp):
+                s_cmp.wait_event(in_done[i])
+                if i - 2 in out_done:
+                    s_cmp.wait_event(out_done[i - 2])         # the results of step i-2 have left the device
+                d = dev2[k]
+                qd.chunk_fwd(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"],
+                             chunk=cfg.chunk, save_for_bwd=True, workspace=ws, o=o2[k], hT=hT2[k])
+                qd.chunk_bwd(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"],
+                             d["dO"], d["dhT"], chunk=cfg.chunk, workspace=ws, reuse_fwd=True, out=g2[k])
+                cmp_done[i] = ev(); cmp_done[i].record(s_cmp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(cmp_done[i])
+                out_host["o"].copy_(o2[k], non_blocking=True)
+                out_host["hT"].copy_(hT2[k], non_blocking=True)
+                for n, t in g2[k].items():
+                    out_host[n].copy_(t, non_blocking=True)
+                out_done[i] = ev(); out_done[i].record(s_out)
+
+        for i in range(2):
+            e2e_step(i)
+        barrier()
+        in_done.clear(); cmp_done.clear(); out_done.clear()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s_in)
+        for i in range(e2e_steps):
+            e2e_step(i)
+        e1.record(s_out)
+        barrier()
+        ems = e0.elapsed_time(e1)
+        ems, _ = sharding.aggregate(ems, 0, "cuda")
+        e2e_value = tokens_step / (ems / e2e_steps * 1e-3)
+        del dev2, o2, hT2, g2
+
+    # ---- roofline: the whole path (what the target is stated on) and the dominant kernel ----------------------
     pk, pk_kind = peaks()
     th = B * T * H                                     # token-heads one launch processes
-    sb = stage_bytes_per_token_head(dk, dv, cfg.chunk)
-    chunk_stages = {n: v for n, v in stages.items() if n in sb and v[1] > 0}
-    dom = max(chunk_stages, key=lambda n: chunk_stages[n][0])
-    dom_ms = chunk_stages[dom][0] / chunk_stages[dom][1]
-    ach = sb[dom] * th / (dom_ms * 1e-3) / 1e9
-    roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / pk["hbm_gbs"], "traffic": NCU_TRAFFIC_BYTES.get(cfg.name, {}).get(dom), "peak_kind": "of " + pk_kind,
-                "ms_per_launch": dom_ms, "algorithmic_bytes_per_launch": sb[dom] * th}
+    rl = path_roofline(cfg, pk)
+    chunk_stages = {n: v for n, v in stages.items() if n in STAGE_PASS and v[1] > 0}
+    stage_ms = {n: v[0] / v[1] for n, v in chunk_stages.items()}
+    path = dict(rl, frac=rl["roofline_ms"] / ms_step, frac_nominal=rl["roofline_ms_nominal"] / ms_step,
+                peak_kind="of " + pk_kind, stage_ms_per_launch=stage_ms,
+                note="whole fwd+bwd step against max(algorithmic bytes / HBM, algorithmic FLOPs / bf16 peak); "
+                     "target 0.50")
+    dom = max(stage_ms, key=lambda n: stage_ms[n])
     fb, bb = path_bytes_per_token_head(dk, dv)
-    ff, fbw = path_flops_per_token_head(dk, dv, cfg.chunk)
-    state_io = 4 * dk * dv * 4 * B * H
-    t_bytes = ((fb + bb) * th + state_io) / (pk["hbm_gbs"] * 1e9)
-    t_flops = (ff + fbw) * th / (pk["bf16_tflops"] * 1e12)
-    per_rank_ms = ms_step
-    path = {"bytes_per_step": (fb + bb) * th + state_io, "flops_per_step": (ff + fbw) * th,
-            "roofline_ms": max(t_bytes, t_flops) * 1e3, "frac": max(t_bytes, t_flops) * 1e3 / per_rank_ms,
-            "peak_kind": "of " + pk_kind,
-            "roofline_ms_nominal": max(((fb + bb) * th + state_io) / 8.0e12, (ff + fbw) * th / 2.25e15) * 1e3,
-            "frac_nominal": max(((fb + bb) * th + state_io) / 8.0e12, (ff + fbw) * th / 2.25e15) * 1e3 / per_rank_ms,
-            "stage_ms_per_launch": {n: v[0] / v[1] for n, v in chunk_stages.items()}}
+    # algorithmic bytes of the pass the dominant kernel belongs to (forward 1030 B, backward 1810 B per token-head at
+    # d = 128, plus that pass's two fp32 states per sequence); the kernels of a pass share them, so each kernel's
+    # fraction is an upper bound on what the pass reaches
+    pass_bytes = (fb if STAGE_PASS[dom] == "fwd" else bb) * th + 2 * dk * dv * 4 * B * H
+    ach = pass_bytes / (stage_ms[dom] * 1e-3) / 1e9
+    sb = stage_bytes_per_token_head(dk, dv, cfg.chunk)
+    roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / pk["hbm_gbs"], "peak_kind": "of " + pk_kind, "ms_per_launch": stage_ms[dom],
+                "algorithmic_bytes_per_launch": pass_bytes,
+                "algorithmic_bytes_are": "the %s pass's bytes of the path (inputs read once, outputs written once), not "
+                                         "the intermediates this decomposition stages" % STAGE_PASS[dom],
+                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name, {}).get(dom),
+                "traffic_source": NCU_TRAFFIC_SOURCE if cfg.name in NCU_TRAFFIC_BYTES else None,
+                # what this kernel would take if it moved only its own staged bytes at the HBM peak
+                "stage_floor": {n: {"bytes_per_launch": sb[n] * th, "ms_at_peak": sb[n] * th / (pk["hbm_gbs"] * 1e6),
+                                    "achieved_gbs_of_staged_bytes": sb[n] * th / (stage_ms[n] * 1e-3) / 1e9}
+                                for n in stage_ms}}
     launches = int(sum(v[1] for v in stages.values()))
+
+    extras = {}
+    if rank == 0 and world == 1 and not args.no_extras:
+        del w, host, dev, ws, o, hT, grads, out_host
+        torch.cuda.empty_cache()
+        # forward only at the headline shape (configuration 1) and the long-context configuration 3
+        extras["forward_only"] = extra_workload(torch, qd, gen, gen.CONFIGS["cfg1"], pk, pk_kind, False, 20, 5)
+        if cfg.name != "cfg3":
+            extras["long_context"] = extra_workload(torch, qd, gen, gen.CONFIGS["cfg3"], pk, pk_kind, True, 5, 5)
+        # the update rule's special cases as absent inputs: lambda = NULL is the gated delta rule (Eq. 3), alpha = NULL
+        # drops the forget gate, both together give DeltaNet (Eq. 2)
+        base = ms_step
+        var = {}
+        for name, drop in (("lambda_absent", ("lam",)), ("alpha_absent", ("alpha",)), ("both_absent", ("lam", "alpha"))):
+            r = extra_workload(torch, qd, gen, cfg, pk, pk_kind, True, 20, 3, drop=drop)
+            var[name] = {"ms_per_step": r["ms_per_step"], "speedup_vs_full_rule": base / r["ms_per_step"]}
+        extras["variants"] = var
 
     # ---- decode step (separate configuration), in place over a long run of steps ------------------
     decode = bench_decode(args, qd, gen, torch, pk, pk_kind) if (rank == 0 and not args.no_extras) else None
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(cfg), "l2": "inputs larger than L2 (no flush)",
-                       "clock_sampling": "nvidia-smi during the timed steps and 1.5 s more of the same step loop",
-                       "kernel_timing": "per-kernel CUDA events in a second pass over the same K steps (events between "
-                                        "launches would serialise the overlapped launches of the timed pass)",
+                       "timing": "median of %d back-to-back regions of exactly %d steps, CUDA events on the launching "
+                                 "stream, max over ranks" % (len(times), args.steps),
+                       "clock_sampling": "nvidia-smi during the timed regions and 1 s more of the same step loop",
+                       "kernel_timing": "per-kernel CUDA events in a separate pass over K steps (events between "
+                                        "launches would serialise the overlapped launches of the timed regions)",
                        "tokens_per_step": tokens_step, "parallelism": "batch sharded over %d rank(s), no collective" % world},
-            "clocks": sampler.summary(),
+            "clocks": clocks, "regions": regions,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "steps": e2e_steps, "pipelining": "upload, compute and download of consecutive steps overlap on three streams"},
-            "gpu_launches": launches, "roofline": roofline, "roofline_path": path, "decode": decode}
+            "gpu_launches": launches, "roofline": roofline, "roofline_path": path,
+            "decode": decode}
+    line.update(extras)
     if rank == 0:
         if world == 1 and not args.no_extras:
             cores = os.cpu_count() or 1
@@ -394,7 +504,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--only", default="all", choices=["all", "decode"],
                     help="'decode': time only the decode step (small runs for profiler captures)")
-    ap.add_argument("--decode-steps", type=int, default=200)
+    ap.add_argument("--regions", type=int, default=21,
+                    help="how many back-to-back regions of --steps steps are timed (the median is reported)")
+    ap.add_argument("--decode-steps", type=int, default=1000, help="configuration 4 runs 1000 sequential steps")
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "small"],
                     help="cfg2: headline (default); cfg3: long context; small: B=2 of cfg2 for profiler captures")
     ap.add_argument("--no-extras", action="store_true", help="skip the end-to-end, decode and CPU-baseline legs")

@@ -20,6 +20,11 @@
  *     dbeta,dalpha,dlambda and every state are fp32.
  *   - The caller owns every buffer, including the workspace whose size it queries.  The library
  *     never allocates, frees or synchronises; all work is enqueued on `stream`.
+ *   - Ordering: a call reads its inputs only after everything enqueued on `stream` before the call has
+ *     completed, and everything enqueued on `stream` after the call sees its outputs complete -- ordinary
+ *     stream order.  (Internally the kernels of one call overlap their set-up with the tail of the kernel
+ *     before them; none of them touches caller data, or workspace contents it depends on, before that
+ *     kernel has completed.)  Work on OTHER streams needs events as usual.
  *   - Inputs are read-only.  Outputs are fully overwritten.  q,k,v,o,dO,dq,dk,dv, the
  *     states and the workspace must be 16-byte aligned; coefficient tensors (and the decode step's o)
  *     need only the alignment of their element type.
@@ -28,7 +33,11 @@
  *     Conditions found on the device (a bounded wait that ran out) are written to the first
  *     32-bit word of the workspace and can be read with qdelta_workspace_status after the
  *     caller has synchronised the stream.
- *   - Supported shapes: chunk = 64, T a multiple of chunk, dk and dv in {64, 128}.
+ *   - Supported shapes: chunk = 64, any T >= 1, dk and dv in {64, 128}.  A sequence length that is not a
+ *     multiple of the chunk is completed, inside the library, with tokens that leave the recurrence
+ *     untouched (beta = 0, alpha = 1); tensors are never read or written beyond their T rows.
+ *     bf16 with dk = dv = 128 runs on the tensor cores (tcgen05); fp32, and bf16 with another head
+ *     dimension, run on plain fp32 FMA kernels (qdelta_chunk_path tells which).
  */
 #ifndef QDELTA_H_
 #define QDELTA_H_
@@ -41,7 +50,7 @@ extern "C" {
 
 typedef enum {
     QD_OK = 0,
-    QD_ERR_INVALID_ARG = 1,   /* null required pointer, non-positive size, T % chunk != 0, misaligned pointer */
+    QD_ERR_INVALID_ARG = 1,   /* null required pointer, non-positive size, misaligned pointer, unknown flag */
     QD_ERR_UNSUPPORTED = 2,   /* (dk, dv, chunk, dtype) outside the supported set */
     QD_ERR_WORKSPACE = 3,     /* workspace null or smaller than qdelta_chunk_workspace_bytes */
     QD_ERR_CUDA = 4,          /* a CUDA runtime call (launch, attribute) failed */
@@ -66,6 +75,10 @@ typedef struct {
 } qd_shape;
 
 typedef struct CUstream_st *qd_stream;   /* a cudaStream_t */
+
+/* Which kernels serve `shape` (the paper has no counterpart; a query for tests and benchmarks):
+ * 1 = tensor-core kernels, 0 = fp32 FMA kernels, -1 = invalid or unsupported shape. */
+int qdelta_chunk_path(const qd_shape *shape);
 
 /* Bytes of device workspace the chunkwise calls need for this shape (0 on invalid shape).
  * for_backward != 0: the size qdelta_chunk_bwd (and a QD_FWD_SAVE_FOR_BWD forward) needs. */

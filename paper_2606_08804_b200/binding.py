@@ -18,7 +18,7 @@ QD_FWD_SAVE_FOR_BWD, QD_BWD_REUSE_FWD = 1, 2
 EXPORTS = ("qdelta_chunk_workspace_bytes", "qdelta_chunk_fwd", "qdelta_chunk_bwd",
            "qdelta_recurrent_step", "qdelta_workspace_status", "qdelta_status_string",
            "qdelta_profile_enable", "qdelta_profile_stage_count", "qdelta_profile_stage_name",
-           "qdelta_profile_read", "qdelta_chunk_fwd_static")
+           "qdelta_profile_read", "qdelta_chunk_fwd_static", "qdelta_chunk_path")
 
 
 class QdShape(ctypes.Structure):
@@ -45,6 +45,8 @@ def load():
     vp, sz, u, i = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint, ctypes.c_int
     lib.qdelta_chunk_workspace_bytes.restype = sz
     lib.qdelta_chunk_workspace_bytes.argtypes = [ctypes.POINTER(QdShape), i]
+    lib.qdelta_chunk_path.restype = i
+    lib.qdelta_chunk_path.argtypes = [ctypes.POINTER(QdShape)]
     lib.qdelta_chunk_fwd.restype = i
     lib.qdelta_chunk_fwd.argtypes = [ctypes.POINTER(QdShape)] + [vp] * 9 + [vp, sz, u, vp]
     lib.qdelta_chunk_bwd.restype = i
@@ -128,6 +130,14 @@ def chunk_workspace_bytes(shape: QdShape, for_backward: bool) -> int:
     if n == 0:
         raise QdeltaError("unsupported or invalid shape for the chunkwise kernels")
     return int(n)
+
+
+def chunk_path(shape: QdShape) -> str:
+    """Which kernels serve this shape: "tensor_core" (tcgen05) or "fp32" (plain FMA)."""
+    r = load().qdelta_chunk_path(ctypes.byref(shape))
+    if r < 0:
+        raise QdeltaError("unsupported or invalid shape for the chunkwise kernels")
+    return "tensor_core" if r == 1 else "fp32"
 
 
 def alloc_workspace(shape: QdShape, for_backward: bool, device) -> torch.Tensor:

@@ -17,7 +17,7 @@ LIB = os.path.join(_HERE, "libqdelta.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "--use_fast_math" if False else "-DQD_NO_FAST_MATH", "-Xcompiler", "-fPIC", "-Xptxas", "-v",
+    "-Xcompiler", "-fPIC", "-Xptxas", "-v",
     "-I", os.path.join(_ROOT, "include"),
 ]
 

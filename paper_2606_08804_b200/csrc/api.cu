@@ -1,8 +1,6 @@
 // C-ABI entry points: argument validation, workspace carving, kernel sequencing.
 #include "internal.h"
 
-#include <cstdio>
-#include <cstdlib>
 #include <vector>
 
 namespace qd {
@@ -11,7 +9,7 @@ static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 WsLayout ws_layout(const qd_shape& s) {
     WsLayout L{};
-    const size_t BH = (size_t)s.B * s.H, T = s.T, N = T / kChunk;
+    const size_t BH = (size_t)s.B * s.H, T = (size_t)simt_padded_T(s), N = T / kChunk;
     const size_t io = s.dtype == QD_BF16 ? 2 : 4;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return o; };
@@ -34,14 +32,13 @@ WsLayout ws_layout(const qd_shape& s) {
     return L;
 }
 
-static int check_shape(const qd_shape* s) {
+int check_shape(const qd_shape* s) {
     if (!s) return QD_ERR_INVALID_ARG;
     if (s->B <= 0 || s->T <= 0 || s->H <= 0 || s->dk <= 0 || s->dv <= 0 || s->chunk <= 0) return QD_ERR_INVALID_ARG;
     if (s->dtype != QD_F32 && s->dtype != QD_BF16) return QD_ERR_UNSUPPORTED;
     if (s->chunk != kChunk) return QD_ERR_UNSUPPORTED;
     if ((s->dk != 64 && s->dk != 128) || (s->dv != 64 && s->dv != 128)) return QD_ERR_UNSUPPORTED;
-    if (s->T % s->chunk != 0) return QD_ERR_INVALID_ARG;
-    if ((long long)s->B * s->H * (s->T / s->chunk) > 0x7fffffffLL / 4) return QD_ERR_UNSUPPORTED;
+    if ((long long)s->B * s->H * ((s->T + 127) / 128 * 2) > 0x7fffffffLL / 4) return QD_ERR_UNSUPPORTED;
     return QD_OK;
 }
 
@@ -82,14 +79,7 @@ struct StageTimer {
 
 template <class F> static cudaError_t timed(int stage, cudaStream_t s, F f) {
     StageTimer t(stage, s);
-    cudaError_t e = f();
-    // QDELTA_DEBUG=1 (debugging aid, breaks the "never synchronises" rule on purpose): wait for the
-    // stage and say which one failed
-    if (getenv("QDELTA_DEBUG")) {
-        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
-        if (e != cudaSuccess) fprintf(stderr, "[qdelta] stage %s: %s\n", kStageNames[stage], cudaGetErrorString(e));
-    }
-    return e;
+    return f();
 }
 
 }  // namespace qd
@@ -107,6 +97,11 @@ size_t qdelta_chunk_workspace_bytes(const qd_shape* shape, int for_backward) {
     }
     WsLayout L = ws_layout(*shape);
     return for_backward ? L.bwd_end : L.fwd_end;
+}
+
+int qdelta_chunk_path(const qd_shape* shape) {
+    if (check_shape(shape) != QD_OK) return -1;
+    return tc_supported(*shape) ? 1 : 0;
 }
 
 int qdelta_chunk_fwd(const qd_shape* shape, const void* q, const void* k, const void* v, const void* beta,
@@ -180,6 +175,7 @@ int qdelta_chunk_bwd(const qd_shape* shape, const void* q, const void* k, const 
             a.hT = nullptr;
             if (timed(ST_PREP, a.stream, [&] { return tc_prep(a); }) != cudaSuccess) return QD_ERR_CUDA;
             if (timed(ST_CHAIN_FWD, a.stream, [&] { return tc_chain_fwd(a); }) != cudaSuccess) return QD_ERR_CUDA;
+            a.own_predecessor = true;      // the reverse chain follows this library's forward chain in the stream
         }
         if (timed(ST_CHAIN_BWD, a.stream, [&] { return tc_chain_bwd(a); }) != cudaSuccess) return QD_ERR_CUDA;
         if (timed(ST_CHUNK_BWD, a.stream, [&] { return tc_chunk_bwd(a); }) != cudaSuccess) return QD_ERR_CUDA;

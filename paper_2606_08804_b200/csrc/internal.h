@@ -35,6 +35,8 @@ struct WsLayout {
 };
 
 WsLayout ws_layout(const qd_shape& s);
+// QD_OK, or the error code every entry point reports for this shape (host-side validation only).
+int check_shape(const qd_shape* s);
 
 // Workspace of the tensor-core path (bf16, d_k = d_v = 128).  Sections start on 1024-byte boundaries.
 struct TcLayout {
@@ -55,6 +57,15 @@ struct TcLayout {
 };
 TcLayout tc_layout(const qd_shape& s);
 bool tc_supported(const qd_shape& s);
+// Rows per sequence in the tensor-core workspace: T rounded up to a whole number of chunk PAIRS (the preparation kernel
+// takes two chunks at a time).  The rows past T behave as tokens with beta = 0, alpha = 1, q = k = v = 0, which leave the
+// recurrence of Section 3.3.1 untouched; TMA supplies the zeros and drops the stores.
+inline int simt_padded_T(const qd_shape& s) { return (s.T + kChunk - 1) / kChunk * kChunk; }   // fp32 path: whole chunks
+inline int tc_padded_T(const qd_shape& s) { return (s.T + 2 * kChunk - 1) / (2 * kChunk) * (2 * kChunk); }
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize for `kernel`: set when first needed on a device, and again only if a
+// later call needs more.
+cudaError_t set_max_smem_once(const void* kernel, size_t bytes);
 
 // Launch with the programmatic-stream-serialization attribute: the kernel may begin before the previous kernel of the
 // stream has finished and orders itself with grid_dep_wait() (see sm100.cuh).
@@ -84,6 +95,7 @@ struct ChunkArgs {
     WsLayout L;
     TcLayout TL;
     bool save;       // forward: keep hs and D
+    bool own_predecessor;   // backward: the kernel enqueued before the reverse chain is this library's forward chain
     cudaStream_t stream;
 };
 

@@ -22,7 +22,7 @@
 
 #include <mutex>
 
-#include "../../include/qdelta.h"
+#include "internal.h"
 
 namespace {
 
@@ -56,10 +56,11 @@ int scratch_for_current_device(void** out) {
 extern "C" int qdelta_chunk_fwd_static(const qd_shape* shape, const void* q, const void* k, const void* v,
                                        const void* beta, const void* alpha, const void* lambda, const float* h0,
                                        void* o, float* hT, unsigned* status_out, qd_stream stream) {
-    if (!shape) return QD_ERR_INVALID_ARG;
+    const int src = qd::check_shape(shape);                         // the same code qdelta_chunk_fwd reports for a bad shape
+    if (src != QD_OK) return src;
     if (status_out && ((uintptr_t)status_out & 3)) return QD_ERR_INVALID_ARG;
     const size_t need = qdelta_chunk_workspace_bytes(shape, 0);
-    if (need == 0) return QD_ERR_INVALID_ARG;                       // the shape itself is not valid
+    if (need == 0) return QD_ERR_INVALID_ARG;
     if (need > kStaticScratchBytes) return QD_ERR_STATIC_SCRATCH;    // larger than the built-in array
     void* scratch = nullptr;
     const int rc = scratch_for_current_device(&scratch);

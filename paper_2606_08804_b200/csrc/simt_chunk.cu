@@ -22,7 +22,8 @@ constexpr int DS = kSliceSimt;
 constexpr int NT = 256;
 
 struct Ptrs {
-    int B, T, H, dk, dv, N;
+    int B, T, Tp, H, dk, dv, N;      // the workspace holds Tp = 64 N >= T rows per sequence; rows past T are tokens with
+                                     // beta = 0, alpha = 1, q = k = v = dO = 0 (exact no-ops of the recurrence)
     const void *q, *k, *v, *beta, *alpha, *lam, *dO;
     const float *h0, *dhT;
     void *o, *dq, *dk_, *dv_;
@@ -71,14 +72,14 @@ __device__ __forceinline__ float warp_sum(float x) {
 
 // Coefficients of one chunk into shared memory: beta, lambda, alpha, g (cumulative log alpha).
 template <typename IO>
-__device__ __forceinline__ void load_coeffs(const Ptrs& p, size_t row0, float* sbeta, float* slam,
+__device__ __forceinline__ void load_coeffs(const Ptrs& p, size_t row0, int live, float* sbeta, float* slam,
                                             float* salpha, float* sg) {
     const int t = threadIdx.x;
     if (t < C) {
         const size_t r = row0 + (size_t)t * p.H;
-        sbeta[t] = ld((const IO*)p.beta, r);
-        slam[t] = p.lam ? ld((const IO*)p.lam, r) : 0.f;
-        salpha[t] = p.alpha ? ld((const IO*)p.alpha, r) : 1.f;
+        sbeta[t] = t < live ? ld((const IO*)p.beta, r) : 0.f;
+        slam[t] = (t < live && p.lam) ? ld((const IO*)p.lam, r) : 0.f;
+        salpha[t] = (t < live && p.alpha) ? ld((const IO*)p.alpha, r) : 1.f;
     }
     __syncthreads();
     if (t == 0) {
@@ -112,13 +113,14 @@ __global__ void __launch_bounds__(NT) k_prep(Ptrs p) {
     const int ch = blockIdx.x, n = ch % p.N, bh = ch / p.N, b = bh / p.H, hh = bh % p.H;
     const int dk = p.dk, dv = p.dv, H = p.H;
     const size_t row0 = ((size_t)b * p.T + (size_t)n * C) * H + hh;   // token row of local r: row0 + r*H
-    const size_t wrow0 = (size_t)bh * p.T + (size_t)n * C;            // workspace row of local r: wrow0 + r
+    const size_t wrow0 = (size_t)bh * p.Tp + (size_t)n * C;           // workspace row of local r: wrow0 + r
+    const int live = min(C, p.T - n * C);                              // tokens of this chunk inside the sequence
     const IO *q = (const IO*)p.q, *k = (const IO*)p.k, *v = (const IO*)p.v;
-    load_coeffs<IO>(p, row0, sbeta, slam, salpha, sg);
+    load_coeffs<IO>(p, row0, live, sbeta, slam, salpha, sg);
     if (threadIdx.x < C) p.g[wrow0 + threadIdx.x] = sg[threadIdx.x];
 
-    auto Qf = [&](int r, int d) { return ld(q, (row0 + (size_t)r * H) * dk + d); };
-    auto Kf = [&](int r, int d) { return ld(k, (row0 + (size_t)r * H) * dk + d); };
+    auto Qf = [&](int r, int d) { return r < live ? ld(q, (row0 + (size_t)r * H) * dk + d) : 0.f; };
+    auto Kf = [&](int r, int d) { return r < live ? ld(k, (row0 + (size_t)r * H) * dk + d) : 0.f; };
     auto Xf = [&](int r, int d) { return fmaf(slam[r], Qf(r, d), Kf(r, d)); };
     // A = strictLower(beta_r Gamma_ri (x_r . k_i))
     mm<4, 4>(C, C, dk, Xf, [&](int d, int i) { return Kf(i, d); },
@@ -134,7 +136,7 @@ __global__ void __launch_bounds__(NT) k_prep(Ptrs p) {
     invert_unit_lower(sA, sM);
     __syncthreads();
     auto Tf = [&](int r, int i) { return sM[r * LD + i] * sbeta[i]; };
-    mm<4, 4>(C, dv, C, Tf, [&](int i, int j) { return ld(v, (row0 + (size_t)i * H) * dv + j); },
+    mm<4, 4>(C, dv, C, Tf, [&](int i, int j) { return i < live ? ld(v, (row0 + (size_t)i * H) * dv + j) : 0.f; },
              [&](int r, int j, float acc) { st((IO*)p.U, (wrow0 + r) * dv + j, acc); });
     mm<4, 4>(C, dk, C, Tf, [&](int i, int d) { return expf(sg[i]) * Xf(i, d); },
              [&](int r, int d, float acc) { st((IO*)p.W, (wrow0 + r) * dk + d, acc); });
@@ -159,7 +161,8 @@ __global__ void __launch_bounds__(NT) k_chain_fwd(Ptrs p) {
     }
     for (int n = 0; n < p.N; ++n) {
         const size_t row0 = ((size_t)b * p.T + (size_t)n * C) * H + hh;
-        const size_t wrow0 = (size_t)bh * p.T + (size_t)n * C;
+        const size_t wrow0 = (size_t)bh * p.Tp + (size_t)n * C;
+        const int live = min(C, p.T - n * C);
         if (threadIdx.x < C) sg[threadIdx.x] = p.g[wrow0 + threadIdx.x];
         __syncthreads();
         if (p.save) {
@@ -175,19 +178,19 @@ __global__ void __launch_bounds__(NT) k_chain_fwd(Ptrs p) {
                      if (p.save) st((IO*)p.D, (wrow0 + r) * dv + j0 + j, d);
                  });
         // inter-chunk part of the output: diag(gamma) Q h
-        mm<2, 4>(C, DS, dk, [&](int r, int i) { return ld(q, (row0 + (size_t)r * H) * dk + i); }, hf,
+        mm<2, 4>(C, DS, dk, [&](int r, int i) { return r < live ? ld(q, (row0 + (size_t)r * H) * dk + i) : 0.f; }, hf,
                  [&](int r, int j, float acc) { sO[r * DS + j] = expf(sg[r]) * acc; });
         __syncthreads();
         // intra-chunk part: P Delta
         mm<2, 4>(C, DS, C, [&](int r, int s) { return ld((const IO*)p.P, (wrow0 + r) * C + s); },
                  [&](int s, int j) { return sD[s * DS + j]; },
                  [&](int r, int j, float acc) {
-                     st((IO*)p.o, (row0 + (size_t)r * H) * dv + j0 + j, sO[r * DS + j] + acc);
+                     if (r < live) st((IO*)p.o, (row0 + (size_t)r * H) * dv + j0 + j, sO[r * DS + j] + acc);
                  });
         // h <- gamma_C h + K->^T Delta
         const float gC = sg[C - 1];
         mm<4, 4>(dk, DS, C,
-                 [&](int i, int r) { return ld(k, (row0 + (size_t)r * H) * dk + i) * expf(gC - sg[r]); },
+                 [&](int i, int r) { return r < live ? ld(k, (row0 + (size_t)r * H) * dk + i) * expf(gC - sg[r]) : 0.f; },
                  [&](int r, int j) { return sD[r * DS + j]; },
                  [&](int i, int j, float acc) { sh[i * DS + j] = fmaf(expf(gC), sh[i * DS + j], acc); });
         __syncthreads();
@@ -212,12 +215,13 @@ __global__ void __launch_bounds__(NT) k_chain_bwd(Ptrs p) {
     float* sg = sKD + C * DS;        // [C]
     const int nsl = dv / DS, sl = blockIdx.x % nsl, j0 = sl * DS, bh = blockIdx.x / nsl, b = bh / H, hh = bh % H;
     const IO *q = (const IO*)p.q, *k = (const IO*)p.k, *dO = (const IO*)p.dO;
-    const size_t BHT = (size_t)p.B * H * p.T, BHN = (size_t)p.B * H * p.N;
+    const size_t BHT = (size_t)p.B * H * p.Tp, BHN = (size_t)p.B * H * p.N;
     for (int e = threadIdx.x; e < dk * DS; e += NT)
         sdh[e] = p.dhT ? p.dhT[((size_t)bh * dk + e / DS) * dv + j0 + e % DS] : 0.f;
     for (int n = p.N - 1; n >= 0; --n) {
         const size_t row0 = ((size_t)b * p.T + (size_t)n * C) * H + hh;
-        const size_t wrow0 = (size_t)bh * p.T + (size_t)n * C;
+        const size_t wrow0 = (size_t)bh * p.Tp + (size_t)n * C;
+        const int live = min(C, p.T - n * C);
         if (threadIdx.x < C) sg[threadIdx.x] = p.g[wrow0 + threadIdx.x];
         __syncthreads();
         // keep dh of this chunk's exit state; partial <dh, h_entry>_F over this slice
@@ -242,7 +246,7 @@ __global__ void __launch_bounds__(NT) k_chain_bwd(Ptrs p) {
         const float gC = sg[C - 1];
         // K-> dh
         mm<2, 4>(C, DS, dk,
-                 [&](int s, int i) { return ld(k, (row0 + (size_t)s * H) * dk + i) * expf(gC - sg[s]); },
+                 [&](int s, int i) { return s < live ? ld(k, (row0 + (size_t)s * H) * dk + i) * expf(gC - sg[s]) : 0.f; },
                  [&](int i, int j) { return sdh[i * DS + j]; },
                  [&](int s, int j, float acc) {
                      sdD[s * DS + j] = acc;
@@ -251,7 +255,7 @@ __global__ void __launch_bounds__(NT) k_chain_bwd(Ptrs p) {
         __syncthreads();
         // + P^T dO   (same thread owns the same (s,j) as above: tile shapes are identical)
         mm<2, 4>(C, DS, C, [&](int s, int r) { return ld((const IO*)p.P, (wrow0 + r) * C + s); },
-                 [&](int r, int j) { return ld(dO, (row0 + (size_t)r * H) * dv + j0 + j); },
+                 [&](int r, int j) { return r < live ? ld(dO, (row0 + (size_t)r * H) * dv + j0 + j) : 0.f; },
                  [&](int s, int j, float acc) {
                      const float d = sdD[s * DS + j] + acc;
                      sdD[s * DS + j] = d;
@@ -266,11 +270,11 @@ __global__ void __launch_bounds__(NT) k_chain_bwd(Ptrs p) {
         // dh_in = gamma_C dh + (diag(gamma) Q)^T dO - W<-^T dDelta    (one product over 2C terms)
         mm<4, 4>(dk, DS, 2 * C,
                  [&](int i, int kk) {
-                     return kk < C ? ld(q, (row0 + (size_t)kk * H) * dk + i) * expf(sg[kk])
+                     return kk < C ? (kk < live ? ld(q, (row0 + (size_t)kk * H) * dk + i) * expf(sg[kk]) : 0.f)
                                    : -ld((const IO*)p.W, (wrow0 + kk - C) * dk + i);
                  },
                  [&](int kk, int j) {
-                     return kk < C ? ld(dO, (row0 + (size_t)kk * H) * dv + j0 + j) : sdD[(kk - C) * DS + j];
+                     return kk < C ? (kk < live ? ld(dO, (row0 + (size_t)kk * H) * dv + j0 + j) : 0.f) : sdD[(kk - C) * DS + j];
                  },
                  [&](int i, int j, float acc) { sdh[i * DS + j] = fmaf(expf(gC), sdh[i * DS + j], acc); });
         __syncthreads();
@@ -305,19 +309,20 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
     const IO *q = (const IO*)p.q, *k = (const IO*)p.k, *v = (const IO*)p.v, *dO = (const IO*)p.dO;
     float* sc = p.scratch + (size_t)blockIdx.x * 4 * C * dk;
     float *dW = sc, *dXg = sc + C * dk, *dX = sc + 2 * C * dk, *dQ1 = sc + 3 * C * dk;
-    const size_t BHT = (size_t)p.B * H * p.T, BHN = (size_t)p.B * H * p.N;
+    const size_t BHT = (size_t)p.B * H * p.Tp, BHN = (size_t)p.B * H * p.N;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     for (int ch = blockIdx.x; ch < nchunks; ch += gridDim.x) {
         const int n = ch % p.N, bh = ch / p.N, b = bh / H, hh = bh % H;
         const size_t row0 = ((size_t)b * p.T + (size_t)n * C) * H + hh;
-        const size_t wrow0 = (size_t)bh * p.T + (size_t)n * C;
+        const size_t wrow0 = (size_t)bh * p.Tp + (size_t)n * C;
+        const int live = min(C, p.T - n * C);
         const float* hs = p.hs + ((size_t)bh * p.N + n) * dk * dv;
         const float* dhs = p.dhs + ((size_t)bh * p.N + n) * dk * dv;
-        auto Qf = [&](int r, int d) { return ld(q, (row0 + (size_t)r * H) * dk + d); };
-        auto Kf = [&](int r, int d) { return ld(k, (row0 + (size_t)r * H) * dk + d); };
-        auto Vf = [&](int r, int j) { return ld(v, (row0 + (size_t)r * H) * dv + j); };
-        auto dOf = [&](int r, int j) { return ld(dO, (row0 + (size_t)r * H) * dv + j); };
+        auto Qf = [&](int r, int d) { return r < live ? ld(q, (row0 + (size_t)r * H) * dk + d) : 0.f; };
+        auto Kf = [&](int r, int d) { return r < live ? ld(k, (row0 + (size_t)r * H) * dk + d) : 0.f; };
+        auto Vf = [&](int r, int j) { return r < live ? ld(v, (row0 + (size_t)r * H) * dv + j) : 0.f; };
+        auto dOf = [&](int r, int j) { return r < live ? ld(dO, (row0 + (size_t)r * H) * dv + j) : 0.f; };
         auto Xf = [&](int r, int d) { return fmaf(slam[r], Qf(r, d), Kf(r, d)); };
         auto Df = [&](int r, int j) { return ld((const IO*)p.D, (wrow0 + r) * dv + j); };
         auto dDf = [&](int r, int j) { return ld((const IO*)p.dD, (wrow0 + r) * dv + j); };
@@ -325,9 +330,9 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
         // S0 coefficients
         if (tid < C) {
             const size_t r = row0 + (size_t)tid * H;
-            sbeta[tid] = ld((const IO*)p.beta, r);
-            slam[tid] = p.lam ? ld((const IO*)p.lam, r) : 0.f;
-            salpha[tid] = p.alpha ? ld((const IO*)p.alpha, r) : 1.f;
+            sbeta[tid] = tid < live ? ld((const IO*)p.beta, r) : 0.f;
+            slam[tid] = (tid < live && p.lam) ? ld((const IO*)p.lam, r) : 0.f;
+            salpha[tid] = (tid < live && p.alpha) ? ld((const IO*)p.alpha, r) : 1.f;
             sg[tid] = p.g[wrow0 + tid];
         }
         __syncthreads();
@@ -358,7 +363,7 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
         // S5 dV = T^T dDelta, dXg = T^T dW<-, dbeta = colsum(dT o M)
         auto TTf = [&](int s, int r) { return m1[r * LD + s] * sbeta[s]; };
         mm<4, 4>(C, dv, C, TTf, [&](int r, int j) { return dDf(r, j); },
-                 [&](int s, int j, float acc) { st((IO*)p.dv_, (row0 + (size_t)s * H) * dv + j, acc); });
+                 [&](int s, int j, float acc) { if (s < live) st((IO*)p.dv_, (row0 + (size_t)s * H) * dv + j, acc); });
         mm<4, 4>(C, dk, C, TTf, [&](int r, int i) { return dW[r * dk + i]; },
                  [&](int s, int i, float acc) { dXg[s * dk + i] = acc; });
         if (tid < C) {
@@ -413,12 +418,12 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
                      return kk < C ? Xf(kk, d) : (kk < 2 * C ? Qf(kk - C, d) : dhs[(size_t)d * dv + kk - 2 * C]);
                  },
                  [&](int i, int d, float acc) {
-                     st((IO*)p.dk_, (row0 + (size_t)i * H) * dk + d, acc + dX[i * dk + d]);
+                     if (i < live) st((IO*)p.dk_, (row0 + (size_t)i * H) * dk + d, acc + dX[i * dk + d]);
                  });
         mm<4, 4>(C, dk, C, [&](int r, int s) { return m3[r * LD + s]; }, Kf,
                  [&](int r, int d, float acc) {
-                     st((IO*)p.dq, (row0 + (size_t)r * H) * dk + d,
-                        acc + dQ1[r * dk + d] + slam[r] * dX[r * dk + d]);
+                     if (r < live)
+                         st((IO*)p.dq, (row0 + (size_t)r * H) * dk + d, acc + dQ1[r * dk + d] + slam[r] * dX[r * dk + d]);
                  });
         for (int r = warp; r < C; r += NT / 32) {
             float a1 = 0.f, a2 = 0.f, a3 = 0.f;
@@ -449,7 +454,7 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
             for (int r = C - 1; r >= 0; --r) { acc += sdg[r]; sdg[r] = acc; }
         }
         __syncthreads();
-        if (tid < C) {
+        if (tid < live) {
             const size_t r = row0 + (size_t)tid * H;
             p.dbeta[r] = sdbeta[tid];
             if (p.dlam) p.dlam[r] = sdlam[tid];
@@ -461,7 +466,7 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
 
 Ptrs make_ptrs(const ChunkArgs& a) {
     Ptrs p{};
-    p.B = a.s.B; p.T = a.s.T; p.H = a.s.H; p.dk = a.s.dk; p.dv = a.s.dv; p.N = a.s.T / kChunk;
+    p.B = a.s.B; p.T = a.s.T; p.Tp = simt_padded_T(a.s); p.H = a.s.H; p.dk = a.s.dk; p.dv = a.s.dv; p.N = p.Tp / kChunk;
     p.q = a.q; p.k = a.k; p.v = a.v; p.beta = a.beta; p.alpha = a.alpha; p.lam = a.lam; p.dO = a.dO;
     p.h0 = a.h0; p.dhT = a.dhT; p.o = a.o; p.dq = a.dq; p.dk_ = a.dk; p.dv_ = a.dv;
     p.hT = a.hT; p.dbeta = a.dbeta; p.dalpha = a.dalpha; p.dlam = a.dlam; p.dh0 = a.dh0;
@@ -476,9 +481,7 @@ Ptrs make_ptrs(const ChunkArgs& a) {
 }
 
 template <class K>
-cudaError_t set_smem(K kern, size_t bytes) {
-    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-}
+cudaError_t set_smem(K kern, size_t bytes) { return set_max_smem_once(reinterpret_cast<const void*>(kern), bytes); }
 
 }  // namespace
 

@@ -39,14 +39,30 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after `limit` polls (each poll may itself block for a short,
-// hardware-defined time).  Returns false on expiry; the caller records the failure and leaves.
-constexpr uint32_t kWaitLimit = 1u << 22;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit = kWaitLimit) {
+// Bounded wait: gives up about `limit_ns` nanoseconds of the global timer after it began (each poll may itself block
+// for a short, hardware-defined time).  Returns false on expiry; the caller records the failure and leaves.  One second
+// is several hundred times the longest kernel of this library and far inside any host-side watchdog.  Reading the
+// global timer is slow (a wait that looked at it on every poll made the chunk-backward kernel 6 % slower), so the
+// timer is read only every kPollsPerTimerRead unsuccessful polls; ordinary waits end long before the first read.
+// The low 32 bits of the timer wrap every 4.29 s, so differences below that are exact.
+__device__ __forceinline__ uint32_t global_timer_lo() {
+    uint32_t t;
+    asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t));
+    return t;
+}
+constexpr uint32_t kWaitLimitNs = 1000u * 1000u * 1000u;
+constexpr uint32_t kPollsPerTimerRead = 64;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit_ns = kWaitLimitNs) {
+    uint32_t t0 = 0;
 #pragma unroll 1
-    for (uint32_t i = 0; i < limit; ++i)
+    for (uint32_t polls = 1;; ++polls) {
         if (mbar_try_wait(bar, parity)) return true;
-    return false;
+        if ((polls & (kPollsPerTimerRead - 1)) == 0) {
+            const uint32_t now = global_timer_lo();
+            if (polls == kPollsPerTimerRead) t0 = now;
+            else if (now - t0 > limit_ns) return false;
+        }
+    }
 }
 
 // ---- programmatic dependent launch ------------------------------------------------------------------------------
@@ -71,6 +87,23 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y)
         : "memory");
+}
+// 3-D tiled copies of the token-major tensors [B][T][H*D]: x = column (elements, a multiple of 8), t = token,
+// b = batch index.  Rows at t >= T are outside the tensor: a load fills them with zeros, a store skips them --
+// which is how a sequence length that is not a multiple of the chunk is handled (t is never negative).
+__device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* map, int x, int t, int b, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(t), "r"(b)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, const void* smem_src, int x, int t, int b) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(smem_u32(smem_src)), "r"(x), "r"(t), "r"(b)
+                 : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int x, int t, int b) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(map), "r"(x), "r"(t), "r"(b) : "memory");
 }
 // Prefetch of a tile into L2 (no shared-memory destination, no completion to wait for).
 __device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
@@ -256,10 +289,13 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 }  // namespace sm100
 
-// ---- host side: tensor maps ----------------------------------------------------------------------
+// ---- host side: tensor maps (tmap.cu) ---------------------------------------------------------------
 // 2-D bf16 tensor [rows][cols] with row pitch `pitch_bytes`, boxes of [box_rows][64] elements,
 // 128-byte swizzle.  Returns false if the driver entry point is missing or the encode fails.
 bool make_tmap_bf16_2d(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t pitch_bytes,
                        uint32_t box_rows);
+// 3-D map of a token-major bf16 tensor [B][T][H*D] (q, k, v, o, dO and the gradients), boxes of
+// [1][box_rows][64]; coordinates (column, token, batch).
+bool make_tmap_tokens(CUtensorMap* map, const void* base, int B, int T, int H, int D, uint32_t box_rows);
 
 }  // namespace qd

@@ -49,7 +49,8 @@ __device__ __forceinline__ void fold(float* v, int lane, int off) {
 
 // =================================================================================================
 struct ChainBwdParams {
-    int T, H, N;
+    int Tp, H, N;              // Tp = 64 N rows per sequence in the workspace
+    int dhT_early;             // the kernel before this one in the stream is the library's own: dhT is older than it
     const float* g;
     const float* dhT;
     float* dh0;
@@ -118,11 +119,15 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
         if (s_abort) return;
         if (!mbar_wait(bar, parity)) { s_abort = 1; *p.status = QD_ERR_TIMEOUT; }
     };
-    const float* gseq = p.g + (size_t)bh * p.T;
+    const float* gseq = p.g + (size_t)bh * p.Tp;
 
     if (warp < kMmaWarp) {
         // ---------------------------------- compute warps ----------------------------------
         float dh[32];     // dh^T[j = l][32 wg .. 32 wg + 31]
+        // dhT is an input of the call.  When the kernel before this one is the library's own forward chain, dhT is older
+        // than that kernel and may be read while it drains; otherwise the predecessor may be the very kernel that wrote
+        // dhT, whose writes are only guaranteed visible after the wait.
+        if (!p.dhT_early) grid_dep_wait();
         if (p.dhT) {
             const float* src = p.dhT + (size_t)bh * D * D + (size_t)(32 * wg) * D + l;
 #pragma unroll
@@ -131,7 +136,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
 #pragma unroll
             for (int i = 0; i < 32; ++i) dh[i] = 0.f;
         }
-        grid_dep_wait();                  // the loads of dhT (an input) are in flight; everything below depends on earlier kernels
+        if (p.dhT_early) grid_dep_wait();  // the loads of dhT are in flight; everything below depends on earlier kernels
         grid_dep_launch();
         // my 32 columns of the operand tile: 64-column block wg >> 1, 16-byte chunks 4 (wg & 1) ..
         unsigned char* myH = sdH + (wg >> 1) * 16384;
@@ -230,15 +235,14 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
             uint64_t* bar = &bar_load[it & 1];
             mbar_expect_tx(bar, kStage);
             const int yc = (int)(((size_t)bh * p.N + n) * D);
-            const int yt = (int)((size_t)bh * p.T + (size_t)n * C);
-            const int yi = (int)((size_t)b * p.T + (size_t)n * C);
+            const int yt = (int)((size_t)bh * p.Tp + (size_t)n * C);
             tma_load_2d(st, &mapWt, 0, yc, bar);
-            tma_load_2d(st + 16384, &mapdO, hh * D, yi, bar);
-            tma_load_2d(st + 16384 + 8192, &mapdO, hh * D + 64, yi, bar);
+            tma_load_3d(st + 16384, &mapdO, hh * D, n * C, b, bar);          // rows past the end of the sequence: zeros
+            tma_load_3d(st + 16384 + 8192, &mapdO, hh * D + 64, n * C, b, bar);
             tma_load_2d(st + 32768, &mapQg, 0, yt, bar);
             tma_load_2d(st + 32768 + 8192, &mapQg, 64, yt, bar);
-            tma_load_2d(st + 49152, &mapK, hh * D, yi, bar);
-            tma_load_2d(st + 49152 + 8192, &mapK, hh * D + 64, yi, bar);
+            tma_load_3d(st + 49152, &mapK, hh * D, n * C, b, bar);
+            tma_load_3d(st + 49152 + 8192, &mapK, hh * D + 64, n * C, b, bar);
             tma_load_2d(st + 65536, &mapP, 0, yt, bar);
         };
         if (lead) { issue_load(0); if (p.N > 1) issue_load(1); }
@@ -290,12 +294,11 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
 
 // =================================================================================================
 struct ChunkBwdParams {
-    int T, H, N, total;        // total = B*H*N chunks
+    int T, Tp, H, N, BH, total;   // T tokens per sequence, Tp = 64 N rows per sequence in the workspace; total = BH*N chunks
     const bf16 *beta, *alpha, *lam;
     const float* g;
     float *dbeta, *dalpha, *dlam;
     unsigned* status;
-    long long* timeline;       // diagnostic builds only (QD_CTA_TIMELINE): start time of every chunk
 };
 
 // shared-memory map of k_tc_chunk_bwd (bytes from the 1024-aligned base)
@@ -314,14 +317,6 @@ constexpr int kBwdThreads = kBwdCompute + 32;            // + one warp that issu
 // named barriers of k_tc_chunk_bwd: 1 = the epilogue threads among themselves; the others are raised by the
 // epilogue threads (bar.arrive) when an operand tile is complete and awaited by the issuing warp (bar.sync)
 constexpr int kNbC = 1, kNbX = 2, kNbDW = 3, kNbDTb = 4, kNbN = 5, kNbDXK = 6, kNbOut = 7, kNbDV = 8, kNbScr = 9;
-
-// Optional phase timestamps (build with -DQD_PHASE_CLOCKS -DQD_CLK_CTA=<chunk>): thread 0 of the CTA that owns that chunk
-// writes clock64() values into bytes 64.. of the workspace status section.
-#ifdef QD_PHASE_CLOCKS
-#define QD_CLK(i) do { if (ch_id == QD_CLK_CTA && threadIdx.x == 0) ((long long*)((char*)p.status + 64))[i] = clock64(); } while (0)
-#else
-#define QD_CLK(i) do { } while (0)
-#endif
 
 // Column sums across the 32 lanes of a warp for 8 columns: returns, in every lane, the warp-wide sum of
 // column col8_of_lane(lane) (four lanes hold each column).
@@ -389,30 +384,33 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     // The tiles of a chunk arrive in two groups.  "early": V, dO, M^T, P -- their regions are dead once the
     // last products of the previous chunk have finished; "late": Q, Delta^T, dDelta^T, h^T, dh^T -- regions
     // that the previous chunk uses up to its end (staging tiles of the stores, scratch of the reductions).
+    // Work item `ch` is chunk n_ of sequence bh_, sequence-major.  (Chunk-major numbering, which would take the tiles the
+    // reverse chain wrote last first, was measured 10 % slower.)
+    auto item = [&](int ch, int& n_, int& bh_) { bh_ = ch / p.N; n_ = ch - bh_ * p.N; };
     auto issue_early = [&](int ch) {
-        const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
-        const int yi = (int)((size_t)b_ * p.T + (size_t)n_ * C), yt = (int)((size_t)bh_ * p.T + (size_t)n_ * C);
-        const int ym = (int)(((size_t)bh_ * p.N + n_) * C);
+        int n_, bh_; item(ch, n_, bh_);
+        const int b_ = bh_ / p.H, hh_ = bh_ % p.H;
+        const int yt = (int)((size_t)bh_ * p.Tp + (size_t)n_ * C);
         mbar_expect_tx(&bar_load, kBwdEarlyBytes);
-        for (int blk = 0; blk < 2; ++blk) {
-            tma_load_2d(sm + oV + blk * 8192, &mapV, hh_ * D + blk * 64, yi, &bar_load);
-            tma_load_2d(sm + odO + blk * 8192, &mapdO, hh_ * D + blk * 64, yi, &bar_load);
+        for (int blk = 0; blk < 2; ++blk) {       // token rows past the end of the sequence arrive as zeros
+            tma_load_3d(sm + oV + blk * 8192, &mapV, hh_ * D + blk * 64, n_ * C, b_, &bar_load);
+            tma_load_3d(sm + odO + blk * 8192, &mapdO, hh_ * D + blk * 64, n_ * C, b_, &bar_load);
         }
-        tma_load_2d(sm + oMt, &mapMt, 0, ym, &bar_load);
+        tma_load_2d(sm + oMt, &mapMt, 0, yt, &bar_load);
         tma_load_2d(sm + oP, &mapP, 0, yt, &bar_load);
     };
     // The late group goes in three batches as its regions fall free: part 0 = Q, K (after the last epilogue),
     // part 1 = h^T, dh^T (after the last products and the column sums have read the scratch that aliases them), part 2 = Delta^T,
     // dDelta^T (after the stores have read the staging tiles).  Only the last batch arrives on the barrier.
     auto issue_late = [&](int ch, int part) {
-        const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
-        const int yi = (int)((size_t)b_ * p.T + (size_t)n_ * C);
+        int n_, bh_; item(ch, n_, bh_);
+        const int b_ = bh_ / p.H, hh_ = bh_ % p.H;
         const int yc = (int)(((size_t)bh_ * p.N + n_) * D);
         if (part == 0) {
             mbar_expect_tx_only(&bar_late, 2 * 16384);
             for (int blk = 0; blk < 2; ++blk) {
-                tma_load_2d(sm + oQ + blk * 8192, &mapQ, hh_ * D + blk * 64, yi, &bar_late);
-                tma_load_2d(sm + oK + blk * 8192, &mapK, hh_ * D + blk * 64, yi, &bar_late);
+                tma_load_3d(sm + oQ + blk * 8192, &mapQ, hh_ * D + blk * 64, n_ * C, b_, &bar_late);
+                tma_load_3d(sm + oK + blk * 8192, &mapK, hh_ * D + blk * 64, n_ * C, b_, &bar_late);
             }
         } else if (part == 1) {
             mbar_expect_tx_only(&bar_late, 2 * 32768);
@@ -429,12 +427,12 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     // the late group of a chunk into L2 only, issued a chunk time before its load: the load, which can only be
     // issued at the very end of the previous chunk and is waited for at once, then finds the tiles in L2
     auto prefetch_late = [&](int ch) {
-        const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
-        const int yi = (int)((size_t)b_ * p.T + (size_t)n_ * C);
+        int n_, bh_; item(ch, n_, bh_);
+        const int b_ = bh_ / p.H, hh_ = bh_ % p.H;
         const int yc = (int)(((size_t)bh_ * p.N + n_) * D);
         for (int blk = 0; blk < 2; ++blk) {
-            tma_prefetch_2d(&mapQ, hh_ * D + blk * 64, yi);
-            tma_prefetch_2d(&mapK, hh_ * D + blk * 64, yi);
+            tma_prefetch_3d(&mapQ, hh_ * D + blk * 64, n_ * C, b_);
+            tma_prefetch_3d(&mapK, hh_ * D + blk * 64, n_ * C, b_);
             tma_prefetch_2d(&mapHs, blk * 64, yc);
             tma_prefetch_2d(&mapdHs, blk * 64, yc);
         }
@@ -445,12 +443,14 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     float cf_beta = 0.f, cf_lam = 0.f, cf_alpha = 1.f, cf_g = 0.f;
     auto fetch_coef = [&](int ch) {
         if (tid < C) {
-            const int n_ = ch % p.N, bh_ = ch / p.N, b_ = bh_ / p.H, hh_ = bh_ % p.H;
+            int n_, bh_; item(ch, n_, bh_);
+            const int b_ = bh_ / p.H, hh_ = bh_ % p.H;
+            const bool live = n_ * C + tid < p.T;             // tokens past the end of the sequence: beta = 0, alpha = 1
             const size_t cr = ((size_t)b_ * p.T + (size_t)n_ * C + tid) * p.H + hh_;
-            cf_beta = __bfloat162float(p.beta[cr]);
-            cf_lam = p.lam ? __bfloat162float(p.lam[cr]) : 0.f;
-            cf_alpha = p.alpha ? __bfloat162float(p.alpha[cr]) : 1.f;
-            cf_g = p.g[(size_t)bh_ * p.T + (size_t)n_ * C + tid];
+            cf_beta = live ? __bfloat162float(p.beta[cr]) : 0.f;
+            cf_lam = (live && p.lam) ? __bfloat162float(p.lam[cr]) : 0.f;
+            cf_alpha = (live && p.alpha) ? __bfloat162float(p.alpha[cr]) : 1.f;
+            cf_g = p.g[(size_t)bh_ * p.Tp + (size_t)n_ * C + tid];
         }
     };
     // bounded wait; once any wait has expired every later wait returns at once and the kernel drains: all
@@ -472,7 +472,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             // first chunk: everything that the reverse chain (the kernel before this one) does not write is fetched
             // before waiting for it -- inputs, and tiles of kernels that had finished before the reverse chain began
             const int ch = blockIdx.x;
-            const int n_ = ch % p.N, bh_ = ch / p.N;
+            int n_, bh_; item(ch, n_, bh_);
             const int yc = (int)(((size_t)bh_ * p.N + n_) * D);
             issue_early(ch);
             issue_late(ch, 0);
@@ -486,8 +486,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         }
         grid_dep_wait();
         for (int ch_id = blockIdx.x, it = 0; ch_id < p.total; ch_id += gridDim.x, ++it) {
-            const int n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
-            const int row0 = (int)((size_t)b * p.T + (size_t)n * C);
+            int n, bh; item(ch_id, n, bh);
+            const int b = bh / p.H, hh = bh % p.H;
             const int next_id = ch_id + gridDim.x;
             const uint32_t ph = it & 1;
             if (s_latch) break;
@@ -518,8 +518,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             }
             nb_sync(kNbDV, kBwdThreads);                                 // the dv staging tile is complete, T6 has been read
             if (lead) {
-                tma_store_2d(&mapdV, sm + oStDv, hh * D, row0);
-                tma_store_2d(&mapdV, sm + oStDv + 8192, hh * D + 64, row0);
+                tma_store_3d(&mapdV, sm + oStDv, hh * D, n * C, b);          // rows past the end of the sequence are skipped
+                tma_store_3d(&mapdV, sm + oStDv + 8192, hh * D + 64, n * C, b);
                 tma_store_commit();
                 tc_fence_after();
                 umma_product<false, false>(T6, adW, 16384, aMt, 8192, C, C, false);         // dW<-^T M         [i][s]
@@ -558,10 +558,10 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             }
             nb_sync(kNbOut, kBwdThreads);                                // the dk and dq staging tiles are complete
             if (lead) {
-                tma_store_2d(&mapdK, sm + oStDk, hh * D, row0);
-                tma_store_2d(&mapdK, sm + oStDk + 8192, hh * D + 64, row0);
-                tma_store_2d(&mapdQ, sm + oStDq, hh * D, row0);
-                tma_store_2d(&mapdQ, sm + oStDq + 8192, hh * D + 64, row0);
+                tma_store_3d(&mapdK, sm + oStDk, hh * D, n * C, b);
+                tma_store_3d(&mapdK, sm + oStDk + 8192, hh * D + 64, n * C, b);
+                tma_store_3d(&mapdQ, sm + oStDq, hh * D, n * C, b);
+                tma_store_3d(&mapdQ, sm + oStDq + 8192, hh * D + 64, n * C, b);
                 tma_store_commit();
                 fence_proxy_async();                                     // the epilogue's reads of Q precede the copy into its region
                 if (next_id < p.total && !s_abort) issue_late(next_id, 0);
@@ -584,16 +584,13 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     grid_dep_wait();                    // coefficients and log-decays are older than the reverse chain; the results below are not
 
     for (int ch_id = blockIdx.x, it = 0; ch_id < p.total; ch_id += gridDim.x, ++it) {
-    const int n = ch_id % p.N, bh = ch_id / p.N, b = bh / p.H, hh = bh % p.H;
+    int n, bh; item(ch_id, n, bh);
+    const int b = bh / p.H, hh = bh % p.H;
     const size_t row0 = (size_t)b * p.T + (size_t)n * C;          // token row in the [B*T] view
+    const int live = min(C, p.T - n * C);                          // tokens of this chunk inside the sequence (may be <= 0)
     const int next_id = ch_id + gridDim.x;
     const uint32_t ph = it & 1;
     if (s_latch) break;
-
-    QD_CLK(0);
-#ifdef QD_CTA_TIMELINE
-    if (tid == 0) { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); p.timeline[ch_id] = t; }
-#endif
     if (tid < C) {
         sbeta[tid] = cf_beta;
         slam[tid] = cf_lam;
@@ -608,7 +605,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     }
     wait(&bar_load, ph);
     wait(&bar_late, ph);
-    QD_CLK(1);
     // ---- X = K + lambda Q (the products that do not read X are already running); partial <dh,h>_F -------
     {
         constexpr int kPer = 16 / (kBwdCompute / 64);     // 16-byte chunks of a row per thread
@@ -640,7 +636,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
 #pragma unroll
         for (int e = 0; e < 8; ++e) dhh_part = fmaf(a[e], c8[e], dhh_part);
     }
-    QD_CLK(2);
     // ---- dW<-^T = -h dDelta^T: row i = l as an operand tile (region of its own: dO is still being read) -----
     wait(&bm_a, ph);
     tc_fence_after();
@@ -656,7 +651,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     nb_arrive(kNbDW, kBwdThreads);
     wait(&bm_b, ph);
     tc_fence_after();
-    QD_CLK(3);
     float* sPP = reinterpret_cast<float*>(sm + oPP);
     {
         // my columns in groups of 8 (one 16-byte bf16 chunk each)
@@ -676,7 +670,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     fence_proxy_async();
     tc_fence_before();
     nb_arrive(kNbDV, kBwdThreads);
-    QD_CLK(4);
     float* sAA = reinterpret_cast<float*>(sm + oAA);
     // One group of 8 columns of the dA epilogue for row r; tA = dA, tX = X K^T, both with row r on this thread's lane.
     auto dA_group = [&](uint32_t tA, uint32_t tX, int g8, int r, float& db, float& rAA) {
@@ -743,7 +736,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     } else {
     wait(&bm_2, ph);
     tc_fence_after();
-    QD_CLK(5);
     if (l < C) {
         // dT^T row s = l, my 32 values of r;  M[r][s] = line s of Mt
         const int s = l;
@@ -772,7 +764,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     fence_proxy_async();
     tc_fence_before();
     nb_arrive(kNbDTb, kBwdThreads);
-    QD_CLK(6);
     // ---- N~ = dT diag(beta) M^T, copied out as an operand tile --------------------------------------
     wait(&bm_3, ph);
     tc_fence_after();
@@ -788,11 +779,9 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     fence_proxy_async();
     tc_fence_before();
     nb_arrive(kNbN, kBwdThreads);
-    QD_CLK(8);
     // ---- dA = -M^T N~ -----------------------------------------------------------------------------
     wait(&bm_4, ph);
     tc_fence_after();
-    QD_CLK(9);
     {
         const int r = l;
         float rAA = 0.f, db = 0.f;
@@ -804,7 +793,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     fence_proxy_async();
     tc_fence_before();
     nb_arrive(kNbDXK, kBwdThreads);
-    QD_CLK(10);
     // ---- the last products; meanwhile the column sums of dA o A and dP o P (kBwdCompute/64 threads per column)
     // and the coefficients of the next chunk -------------------------------------------------------------------
     csync();
@@ -842,12 +830,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             rPP += srow[0][w4][r]; dbt += srow[1][w4][r] + srow[4][w4][r]; t2 += srow[2][w4][r]; rAA += srow[3][w4][r] + srow[5][w4][r];
         }
         dg_pre = rPP - cPP + t2 + rAA - cAA;
-        p.dbeta[(row0 + r) * p.H + hh] = dbt;
+        if (r < live) p.dbeta[(row0 + r) * p.H + hh] = dbt;
     }
     if (next_id < p.total) fetch_coef(next_id);
     wait(&bm_5, ph);
     tc_fence_after();
-    QD_CLK(11);
     {
         const int i = l;                                            // d_k index; my 32 tokens c0..c0+31 in groups of 8
         unsigned char* stk = sm + oStDk + (i >> 6) * 8192;
@@ -893,7 +880,6 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     tc_fence_before();
     nb_arrive(kNbOut, kBwdThreads);
     csync();
-    QD_CLK(12);
     // ---- decay gradient ----------------------------------------------------------------------------
     if (tid < C) {
         const int r = tid;
@@ -902,7 +888,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         for (int w4 = 0; w4 < 4; ++w4) { kd += sred[0][w4][r]; dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
         sdg[r] = t1 + dg_pre - kd;
         skd[r] = kd;                            // summed below into dg of the last token
-        if (p.dlam) p.dlam[(row0 + r) * p.H + hh] = dl;
+        if (p.dlam && r < live) p.dlam[(row0 + r) * p.H + hh] = dl;
     }
     csync();
     if (tid < 32) {
@@ -924,13 +910,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             if (lane + o < 32) sfx += t;
         }
         if (p.dalpha) {
-            p.dalpha[(row0 + 2 * lane) * p.H + hh] = sfx / salpha[2 * lane];
-            p.dalpha[(row0 + 2 * lane + 1) * p.H + hh] = (sfx - a) / salpha[2 * lane + 1];
+            if (2 * lane < live) p.dalpha[(row0 + 2 * lane) * p.H + hh] = sfx / salpha[2 * lane];
+            if (2 * lane + 1 < live) p.dalpha[(row0 + 2 * lane + 1) * p.H + hh] = (sfx - a) / salpha[2 * lane + 1];
         }
     }
-    QD_CLK(13);
     __syncthreads();                     // every read of this chunk's tiles and scratch is done
-    QD_CLK(14);
     }  // chunk loop
     }  // epilogue threads
     tc_fence_before();
@@ -940,27 +924,26 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
 }
 
 template <class K>
-cudaError_t set_smem(K kern, size_t bytes) {
-    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-}
+cudaError_t set_smem(K kern, size_t bytes) { return set_max_smem_once(reinterpret_cast<const void*>(kern), bytes); }
 
 }  // namespace
 
 cudaError_t tc_chain_bwd(const ChunkArgs& a) {
     const qd_shape& s = a.s;
-    const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
-    const uint64_t icols = (uint64_t)s.H * D, irows = (uint64_t)s.B * s.T;
+    const int Tp = tc_padded_T(s);
+    const uint64_t BH = (uint64_t)s.B * s.H, N = Tp / kChunk;
     CUtensorMap mWt, mdO, mQg, mK, mP, mdHs, mdDt;
     if (!make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, BH * N * D, 128, 128) ||
-        !make_tmap_bf16_2d(&mdO, a.dO, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mQg, a.ws + a.TL.Qg, D, BH * s.T, D * 2, 64) ||
-        !make_tmap_bf16_2d(&mK, a.k, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * s.T, 128, 64) ||
+        !make_tmap_tokens(&mdO, a.dO, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_bf16_2d(&mQg, a.ws + a.TL.Qg, D, BH * Tp, D * 2, 64) ||
+        !make_tmap_tokens(&mK, a.k, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * Tp, 128, 64) ||
         !make_tmap_bf16_2d(&mdHs, a.ws + a.TL.dhsT, D, BH * N * D, D * 2, 128) ||
         !make_tmap_bf16_2d(&mdDt, a.ws + a.TL.dDt, 64, BH * N * D, 128, 128))
         return cudaErrorInvalidValue;
     ChainBwdParams p{};
-    p.T = s.T; p.H = s.H; p.N = (int)N;
+    p.Tp = Tp; p.H = s.H; p.N = (int)N;
+    p.dhT_early = a.own_predecessor ? 1 : 0;
     p.g = (const float*)(a.ws + a.TL.g);
     p.dhT = a.dhT; p.dh0 = a.dh0;
     p.status = (unsigned*)(a.ws + a.TL.status);
@@ -972,35 +955,32 @@ cudaError_t tc_chain_bwd(const ChunkArgs& a) {
 
 cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
     const qd_shape& s = a.s;
-    const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
-    const uint64_t icols = (uint64_t)s.H * D, irows = (uint64_t)s.B * s.T;
+    const int Tp = tc_padded_T(s);
+    const uint64_t BH = (uint64_t)s.B * s.H, N = Tp / kChunk;
     CUtensorMap mQ, mK, mV, mdO, mMt, mP, mDt, mdDt, mHs, mdHs, mdQ, mdK, mdV;
-    if (!make_tmap_bf16_2d(&mdQ, a.dq, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mdK, a.dk, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mdV, a.dv, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mQ, a.q, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mK, a.k, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mV, a.v, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mdO, a.dO, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mMt, a.ws + a.TL.Mt, 64, BH * s.T, 128, 64) ||
-        !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * s.T, 128, 64) ||
+    if (!make_tmap_tokens(&mdQ, a.dq, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_tokens(&mdK, a.dk, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_tokens(&mdV, a.dv, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_tokens(&mQ, a.q, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_tokens(&mK, a.k, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_tokens(&mV, a.v, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_tokens(&mdO, a.dO, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_bf16_2d(&mMt, a.ws + a.TL.Mt, 64, BH * Tp, 128, 64) ||
+        !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * Tp, 128, 64) ||
         !make_tmap_bf16_2d(&mDt, a.ws + a.TL.Dt, 64, BH * N * D, 128, 128) ||
         !make_tmap_bf16_2d(&mdDt, a.ws + a.TL.dDt, 64, BH * N * D, 128, 128) ||
         !make_tmap_bf16_2d(&mHs, a.ws + a.TL.hsT, D, BH * N * D, D * 2, 128) ||
         !make_tmap_bf16_2d(&mdHs, a.ws + a.TL.dhsT, D, BH * N * D, D * 2, 128))
         return cudaErrorInvalidValue;
     ChunkBwdParams p{};
-    p.T = s.T; p.H = s.H; p.N = (int)N; p.total = (int)(BH * N);
+    p.T = s.T; p.Tp = Tp; p.H = s.H; p.N = (int)N; p.BH = (int)BH; p.total = (int)(BH * N);
     p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
     p.g = (const float*)(a.ws + a.TL.g);
     p.dbeta = a.dbeta; p.dalpha = a.dalpha; p.dlam = a.dlam;
     p.status = (unsigned*)(a.ws + a.TL.status);
-#ifdef QD_CTA_TIMELINE
-    p.timeline = (long long*)(a.ws + a.TL.Ut);      // U~^T is not read by the backward kernels
-#endif
     cudaError_t e = set_smem(k_tc_chunk_bwd, kBwdSmem);
     if (e != cudaSuccess) return e;
-    // persistent: one CTA per SM walks the chunks with stride gridDim.x
+    // persistent: one CTA per SM walks the work items with stride gridDim.x
     int dev = 0, sms = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;

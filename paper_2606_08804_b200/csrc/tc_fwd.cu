@@ -38,28 +38,18 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 
 // =================================================================================================
 struct PrepParams {
-    int T, H, N;
+    int T, Tp, H, N, BH;       // T tokens per sequence; the workspace holds Tp = 64 N >= T rows per sequence (N even)
     const bf16 *beta, *alpha, *lam;
     float* g;
     bf16 *Qg, *P;
     bf16* Mt;                  // optional: ((I+A)^-1)^T per chunk, [column i][row r]; kept for the backward
     unsigned* status;
-    long long* timeline;       // diagnostic builds only (QD_CTA_TIMELINE): 16 stamp slots per CTA
 };
 
 // 96 KB: Q (later X, in place) | K (later A in fp32, then the T tiles) | V; at the end the first and the
 // last 32 KB stage U~^T and W~^T for their TMA stores.  Two CTAs fit on one SM.
 constexpr int kPrepSmem = 3 * 32768 + 1024;
 constexpr int kPrepThreads = 256;
-
-// Optional per-CTA timeline (build with -DQD_CTA_TIMELINE; the workspace must be backward-sized): thread 0 of
-// every CTA writes the global nanosecond timer at each phase boundary into the (then unused) entry-state section.
-#ifdef QD_CTA_TIMELINE
-__device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
-#define QD_TL(i) do { if (threadIdx.x == 0) p.timeline[(size_t)blockIdx.x * 16 + (i)] = gtime(); } while (0)
-#else
-#define QD_TL(i) do { } while (0)
-#endif
 
 // One CTA prepares a pair of chunks (128 tokens) of one head.  Thread roles change by phase:
 //   scan / coefficients   thread t < 128 owns token t
@@ -83,12 +73,13 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     __shared__ float sg[128], sbeta[128], slam[128], swsum[4];
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int pairs = p.N / 2, bh = blockIdx.x / pairs, pr = blockIdx.x % pairs;
+    // CTAs are numbered pair-major, last pair first: the forward chain, which starts with chunk 0 of every sequence,
+    // then finds the tiles written last (and K, read last) still in L2
+    const int pairs = p.N / 2, pr = pairs - 1 - (int)blockIdx.x / p.BH, bh = (int)blockIdx.x % p.BH;
     const int b = bh / p.H, hh = bh % p.H;
-    const size_t tok0 = (size_t)b * p.T + (size_t)pr * 128;          // first row in the [B*T] view
-    const size_t wtok0 = (size_t)bh * p.T + (size_t)pr * 128;        // first row in the [BH*T] view
+    const int t0 = pr * 128;                                         // first token of the pair
+    const size_t wtok0 = (size_t)bh * p.Tp + (size_t)t0;             // first row in the workspace's [BH*Tp] view
 
-    QD_TL(10);
     if (tid == 0) {
         mbar_init(&bar_load, 1);
         mbar_init(&bar_mma, 1);
@@ -100,23 +91,23 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     tc_fence_after();
     const uint32_t tbase = tmem_slot;
 
-    QD_TL(0);
     grid_dep_launch();                // the kernel after this one may set itself up while the last CTAs of this one run
     if (tid == 0) {
         mbar_expect_tx(&bar_load, 3 * 32768);
-        const int y = (int)tok0;
-        for (int blk = 0; blk < 2; ++blk) {
-            tma_load_2d(sQ + blk * 16384, &mapQ, hh * D + blk * 64, y, &bar_load);
-            tma_load_2d(sK + blk * 16384, &mapK, hh * D + blk * 64, y, &bar_load);
-            tma_load_2d(sV + blk * 16384, &mapV, hh * D + blk * 64, y, &bar_load);
+        for (int blk = 0; blk < 2; ++blk) {          // rows at t >= T arrive as zeros
+            tma_load_3d(sQ + blk * 16384, &mapQ, hh * D + blk * 64, t0, b, &bar_load);
+            tma_load_3d(sK + blk * 16384, &mapK, hh * D + blk * 64, t0, b, &bar_load);
+            tma_load_3d(sV + blk * 16384, &mapV, hh * D + blk * 64, t0, b, &bar_load);
         }
     }
     // coefficients of token tid; in-chunk cumulative log-decay by a two-warp scan per chunk
     if (tid < 128) {
-        const size_t crow = (tok0 + tid) * p.H + hh;
-        sbeta[tid] = __bfloat162float(p.beta[crow]);
-        slam[tid] = p.lam ? __bfloat162float(p.lam[crow]) : 0.f;
-        const float alpha = p.alpha ? __bfloat162float(p.alpha[crow]) : 1.f;
+        // a token past the end of the sequence is an exact no-op of the recurrence: beta = 0, alpha = 1 (and q = k = v = 0)
+        const bool live = t0 + tid < p.T;
+        const size_t crow = ((size_t)b * p.T + t0 + tid) * p.H + hh;
+        sbeta[tid] = live ? __bfloat162float(p.beta[crow]) : 0.f;
+        slam[tid] = (live && p.lam) ? __bfloat162float(p.lam[crow]) : 0.f;
+        const float alpha = (live && p.alpha) ? __bfloat162float(p.alpha[crow]) : 1.f;
         float g = logf(alpha);
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -138,7 +129,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         if (warp == 0) tmem_dealloc(tbase, 256);
         return;
     }
-    QD_TL(1);
     if (tid == 0) {
         tc_fence_after();
         // G2 = Q K^T -> columns [128,256)
@@ -168,7 +158,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         if (warp == 0) tmem_dealloc(tbase, 256);
         return;
     }
-    QD_TL(2);
     // X = K + lambda Q, in place over Q (K-major swizzled layout)
 #pragma unroll 4
     for (int it = 0; it < 8; ++it) {
@@ -185,7 +174,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    QD_TL(3);
     if (tid == 0) {
         tc_fence_after();
         // G1 = X K^T -> columns [0,128)
@@ -199,7 +187,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         return;
     }
     tc_fence_after();
-    QD_TL(4);
     // A = strictLower(beta_r Gamma_ri (x_r . k_i)) -> shared fp32, transposed;  P = Gamma_ri (q_r . k_i), i <= r -> workspace
     {
         const int row = tid & 127, half = tid >> 7, c = row >> 6, r = row & 63;
@@ -226,7 +213,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
-    QD_TL(5);
     // M_c = (I + A_c)^-1 by right-looking substitution, columns in registers.  A lane quad of the first four warps
     // owns four columns of one chunk, j0 + 16 k with j0 < 16 (the same loads of A serve all four); lane `ql` of the
     // quad owns the 8-row blocks ql and ql + 4.  Once m[i] is final its owner hands it to the other three lanes and
@@ -270,7 +256,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         }
     }
     __syncthreads();
-    QD_TL(6);
     // T_c = M_c diag(beta), T_c diag(gamma): line j of the MN-major tiles holds column j over the rows
     if (tid < 128) {
         unsigned char* t0 = sT + ic * 8192;
@@ -295,7 +280,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    QD_TL(7);
     if (tid == 0) {
         tc_fence_after();
         for (int cc = 0; cc < 2; ++cc) {
@@ -314,7 +298,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         return;
     }
     tc_fence_after();
-    QD_TL(8);
     // row d = tid & 127 of U~^T (threads < 128) resp. W~^T (the others), both chunks: staged as swizzled
     // [128][64] tiles over the dead Q/X and V regions, then written by TMA
     {
@@ -333,7 +316,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
-    QD_TL(9);
     if (tid == 0) {
         const int y = (int)(((size_t)bh * p.N + 2 * pr) * D);
         tma_store_2d(&mapUt, sQ, 0, y);
@@ -347,12 +329,11 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         __syncwarp();
         tmem_dealloc(tbase, 256);
     }
-    QD_TL(11);
 }
 
 // =================================================================================================
 struct ChainParams {
-    int T, H, N;
+    int Tp, H, N;              // Tp = 64 N rows per sequence in the workspace
     const float* g;
     const float* h0;
     float* hT;
@@ -425,7 +406,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         if (s_abort) return;
         if (!mbar_wait(bar, parity)) { s_abort = 1; *p.status = QD_ERR_TIMEOUT; }
     };
-    const float* gseq = p.g + (size_t)bh * p.T;
+    const float* gseq = p.g + (size_t)bh * p.Tp;
 
     if (warp < kMmaWarp) {
         // ---------------------------------- compute warps ----------------------------------
@@ -466,20 +447,10 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             nb_arrive(kBarO, kNb);
         };
 
-#ifdef QD_PHASE_CLOCKS
-#define QD_C(i) do { if (blockIdx.x == 5 && tid == 0 && n == 10) ((long long*)((char*)p.status + 64))[i] = clock64(); } while (0)
-#define QD_M(i) do { if (blockIdx.x == 5 && lead && n == 10) ((long long*)((char*)p.status + 64))[12 + (i)] = clock64(); } while (0)
-#else
-#define QD_C(i) do { } while (0)
-#define QD_M(i) do { } while (0)
-#endif
         for (int n = 0; n < p.N; ++n) {
-            QD_C(0);
             const unsigned char* st = smem + (n & 1) * kStage;
-            QD_C(1);
             wait(&bar_load[n & 1], (n >> 1) & 1);
             wait(&bar_a, n & 1);
-            QD_C(2);
             tc_fence_after();
             // decay ratios of my 16 tokens
             float sc[16];
@@ -515,13 +486,10 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             tc_fence_before();
             fence_proxy_async();
             nb_arrive(kBarD, kNb); nb_arrive(kBarDt, kNb);
-            QD_C(3);
             // in the shadow of the H product: output epilogue of the previous chunk
             if (n > 0) { wait(&bar_o, (n - 1) & 1); tc_fence_after(); o_stage(n - 1); }
-            QD_C(4);
             // h^T <- gamma_C h^T + acc (my 32 d_k columns), refresh the bf16 operand copy
             wait(&bar_b, n & 1);
-            QD_C(5);
             tc_fence_after();
             {
                 float v[32];
@@ -535,7 +503,6 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             tc_fence_before();
             fence_proxy_async();
             nb_arrive(kBarH, kNb); nb_arrive(kBarHt, kNb);
-            QD_C(6);
         }
         wait(&bar_o, (p.N - 1) & 1);
         tc_fence_after();
@@ -554,34 +521,27 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         for (int n = 0; n < p.N; ++n) {
             const uint32_t st = smem_u32(smem + (n & 1) * kStage);
             const uint32_t tO = tO0 + 64 * (n & 1);
-            QD_M(0);
             if (lead) wait(&bar_load[n & 1], (n >> 1) & 1);
             nb_sync(kBarH, kNb);                          // h^T operand of chunk n is in place
-            QD_M(1);
             if (lead) {
                 tc_fence_after();
                 // Delta-accumulator = h^T Wt (B: MN-major, lines = d_k)
                 umma_product<false, true>(tD, aH, 16384, st, 8192, C, D, false);
                 umma_commit(&bar_a);
-                QD_M(2);
                 // O-accumulator = h^T Qg^T (B: K-major); it reads the state tile, so the commit behind the
                 // H product below (which releases that tile) must cover it
                 umma_product<false, false>(tO, aH, 16384, st + 32768, 8192, C, D, false);
             }
-            QD_M(3);
             nb_sync(kBarD, kNb);                          // Delta^T operands of chunk n are in place
-            QD_M(4);
             if (lead) {
                 tc_fence_after();
                 // H-accumulator = scaled Delta^T K (B: MN-major, lines = tokens)
                 umma_product<false, true>(tH, aDs, 16384, st + 49152, 8192, D, C, false);
                 umma_commit(&bar_b);
-                QD_M(5);
                 // O-accumulator += Delta^T P^T (B: K-major [r][s])
                 umma_product<false, false>(tO, aD, 16384, st + 65536, 8192, C, C, true);
                 umma_commit(&bar_o);
                 umma_commit(&bar_e);
-                QD_M(6);
             }
         }
         nb_sync(kBarH, kNb);                              // final arrival of the compute warps
@@ -595,14 +555,13 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             uint64_t* bar = &bar_load[n & 1];
             mbar_expect_tx(bar, kStage);
             const int yc = (int)(((size_t)bh * p.N + n) * D);
-            const int yt = (int)((size_t)bh * p.T + (size_t)n * C);
+            const int yt = (int)((size_t)bh * p.Tp + (size_t)n * C);
             tma_load_2d(st, &mapWt, 0, yc, bar);
             tma_load_2d(st + 16384, &mapUt, 0, yc, bar);
             tma_load_2d(st + 32768, &mapQg, 0, yt, bar);
             tma_load_2d(st + 32768 + 8192, &mapQg, 64, yt, bar);
-            const int yk = (int)((size_t)b * p.T + (size_t)n * C);
-            tma_load_2d(st + 49152, &mapK, hh * D, yk, bar);
-            tma_load_2d(st + 49152 + 8192, &mapK, hh * D + 64, yk, bar);
+            tma_load_3d(st + 49152, &mapK, hh * D, n * C, b, bar);
+            tma_load_3d(st + 49152 + 8192, &mapK, hh * D + 64, n * C, b, bar);
             tma_load_2d(st + 65536, &mapP, 0, yt, bar);
         };
         if (lead) { issue_load(0); if (p.N > 1) issue_load(1); }
@@ -642,9 +601,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
             if (n > 0) {
                 nb_sync(kBarO, kNb);                      // output tile of chunk n-1 staged
                 if (lead) {
-                    const int yo = (int)((size_t)b * p.T + (size_t)(n - 1) * C);
-                    tma_store_2d(&mapO, sO, hh * D, yo);
-                    tma_store_2d(&mapO, sO + 8192, hh * D + 64, yo);
+                    tma_store_3d(&mapO, sO, hh * D, (n - 1) * C, b);      // rows past the end of the sequence are skipped
+                    tma_store_3d(&mapO, sO + 8192, hh * D + 64, (n - 1) * C, b);
                     tma_store_commit();                   // group: output of chunk n-1
                 }
             }
@@ -657,9 +615,8 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         if (lead) { tma_store_wait_read_n<0>(); mbar_arrive(&bar_o); }
         nb_sync(kBarO, kNb);                              // output tile of the last chunk staged
         if (lead) {
-            const int yo = (int)((size_t)b * p.T + (size_t)(p.N - 1) * C);
-            tma_store_2d(&mapO, sO, hh * D, yo);
-            tma_store_2d(&mapO, sO + 8192, hh * D + 64, yo);
+            tma_store_3d(&mapO, sO, hh * D, (p.N - 1) * C, b);
+            tma_store_3d(&mapO, sO + 8192, hh * D + 64, (p.N - 1) * C, b);
             tma_store_commit();
             tma_store_wait_all();
             if (s_abort) { mbar_wait(&bar_load[0], 0); mbar_wait(&bar_load[1], 0); }
@@ -671,20 +628,18 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
 }
 
 template <class K>
-cudaError_t set_smem(K kern, size_t bytes) {
-    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-}
+cudaError_t set_smem(K kern, size_t bytes) { return set_max_smem_once(reinterpret_cast<const void*>(kern), bytes); }
 
 }  // namespace
 
 bool tc_supported(const qd_shape& s) {
-    return s.dtype == QD_BF16 && s.dk == 128 && s.dv == 128 && s.chunk == kChunk && s.T % 128 == 0 &&
-           (long long)s.B * s.H * s.T * 128 < 0x7fffffffLL * 64;
+    return s.dtype == QD_BF16 && s.dk == 128 && s.dv == 128 && s.chunk == kChunk &&
+           (long long)s.B * s.H * tc_padded_T(s) * 128 < 0x7fffffffLL * 64;
 }
 
 TcLayout tc_layout(const qd_shape& s) {
     TcLayout L{};
-    const size_t BH = (size_t)s.B * s.H, T = s.T;
+    const size_t BH = (size_t)s.B * s.H, T = (size_t)tc_padded_T(s);
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = (off + bytes + 1023) & ~(size_t)1023; return o; };
     L.status = take(256);
@@ -707,23 +662,20 @@ TcLayout tc_layout(const qd_shape& s) {
 cudaError_t tc_prep(const ChunkArgs& a) {
     const qd_shape& s = a.s;
     CUtensorMap mQ, mK, mV, mUt, mWt;
-    const uint64_t rows = (uint64_t)s.B * s.T, cols = (uint64_t)s.H * D;
-    const uint64_t trows = (uint64_t)s.B * s.H * (s.T / kChunk) * D;          // rows of the [chunk][d][64] tiles
-    if (!make_tmap_bf16_2d(&mQ, a.q, cols, rows, cols * 2, 128) || !make_tmap_bf16_2d(&mK, a.k, cols, rows, cols * 2, 128) ||
-        !make_tmap_bf16_2d(&mV, a.v, cols, rows, cols * 2, 128) ||
+    const int Tp = tc_padded_T(s);
+    const uint64_t trows = (uint64_t)s.B * s.H * (Tp / kChunk) * D;          // rows of the [chunk][d][64] tiles
+    if (!make_tmap_tokens(&mQ, a.q, s.B, s.T, s.H, D, 128) || !make_tmap_tokens(&mK, a.k, s.B, s.T, s.H, D, 128) ||
+        !make_tmap_tokens(&mV, a.v, s.B, s.T, s.H, D, 128) ||
         !make_tmap_bf16_2d(&mUt, a.ws + a.TL.Ut, 64, trows, 128, 128) ||
         !make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, trows, 128, 128))
         return cudaErrorInvalidValue;
     PrepParams p{};
-    p.T = s.T; p.H = s.H; p.N = s.T / kChunk;
+    p.T = s.T; p.Tp = Tp; p.H = s.H; p.N = Tp / kChunk; p.BH = s.B * s.H;
     p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
     p.g = (float*)(a.ws + a.TL.g);
     p.Qg = (bf16*)(a.ws + a.TL.Qg); p.P = (bf16*)(a.ws + a.TL.P);
     p.Mt = a.save ? (bf16*)(a.ws + a.TL.Mt) : nullptr;
     p.status = (unsigned*)(a.ws + a.TL.status);
-#ifdef QD_CTA_TIMELINE
-    p.timeline = (long long*)(a.ws + a.TL.hsT);
-#endif
     cudaError_t e = set_smem(k_tc_prep, kPrepSmem);
     if (e != cudaSuccess) return e;
     const int grid = s.B * s.H * (p.N / 2);
@@ -733,20 +685,20 @@ cudaError_t tc_prep(const ChunkArgs& a) {
 
 cudaError_t tc_chain_fwd(const ChunkArgs& a) {
     const qd_shape& s = a.s;
-    const uint64_t BH = (uint64_t)s.B * s.H, N = s.T / kChunk;
-    const uint64_t icols = (uint64_t)s.H * D, irows = (uint64_t)s.B * s.T;
+    const int Tp = tc_padded_T(s);
+    const uint64_t BH = (uint64_t)s.B * s.H, N = Tp / kChunk;
     CUtensorMap mWt, mUt, mQg, mK, mP, mHs, mDt, mO;
     if (!make_tmap_bf16_2d(&mHs, a.ws + a.TL.hsT, D, BH * N * D, D * 2, 128) ||
         !make_tmap_bf16_2d(&mDt, a.ws + a.TL.Dt, 64, BH * N * D, 128, 128) ||
-        !make_tmap_bf16_2d(&mO, a.o, icols, irows, icols * 2, 64) ||
+        !make_tmap_tokens(&mO, a.o, s.B, s.T, s.H, D, 64) ||
         !make_tmap_bf16_2d(&mWt, a.ws + a.TL.Wt, 64, BH * N * D, 128, 128) ||
         !make_tmap_bf16_2d(&mUt, a.ws + a.TL.Ut, 64, BH * N * D, 128, 128) ||
-        !make_tmap_bf16_2d(&mQg, a.ws + a.TL.Qg, D, BH * s.T, D * 2, 64) ||
-        !make_tmap_bf16_2d(&mK, a.k, icols, irows, icols * 2, 64) ||
-        !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * s.T, 128, 64))
+        !make_tmap_bf16_2d(&mQg, a.ws + a.TL.Qg, D, BH * Tp, D * 2, 64) ||
+        !make_tmap_tokens(&mK, a.k, s.B, s.T, s.H, D, 64) ||
+        !make_tmap_bf16_2d(&mP, a.ws + a.TL.P, 64, BH * Tp, 128, 64))
         return cudaErrorInvalidValue;
     ChainParams p{};
-    p.T = s.T; p.H = s.H; p.N = (int)N;
+    p.Tp = Tp; p.H = s.H; p.N = (int)N;
     p.g = (const float*)(a.ws + a.TL.g);
     p.h0 = a.h0; p.hT = a.hT;
     p.save = a.save ? 1 : 0;

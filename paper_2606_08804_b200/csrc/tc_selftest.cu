@@ -1,34 +1,13 @@
-// Unit check of the sm_100a primitives: one CTA computes D[128 x N] = Aop * Bop^T over a
-// contraction of K with tcgen05.mma from 128-byte-swizzled shared-memory tiles, in each of the four
-// operand-major combinations the kernels use, with tiles filled either by TMA or by threads.
-// Also hosts the tensor-map encoder.
+// Unit checks of the sm_100a primitives.
+//  * one CTA computes D[128 x N] = Aop * Bop^T over a contraction of K with tcgen05.mma from
+//    128-byte-swizzled shared-memory tiles, in each of the four operand-major combinations the kernels
+//    use, with tiles filled either by TMA or by threads;
+//  * one CTA waits, with a short limit, on an mbarrier that nothing ever arrives on: the path every kernel
+//    takes when a bounded wait runs out (record QD_ERR_TIMEOUT, release tensor memory, return).
 #include "internal.h"
 #include "sm100.cuh"
 
-#include <cudaTypedefs.h>
-
 namespace qd {
-
-bool make_tmap_bf16_2d(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint64_t pitch_bytes,
-                       uint32_t box_rows) {
-    static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
-    if (!encode) {
-        void* fn = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
-            qres != cudaDriverEntryPointSuccess || !fn)
-            return false;
-        encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
-    }
-    cuuint64_t dims[2] = {cols, rows};
-    cuuint64_t strides[1] = {pitch_bytes};
-    cuuint32_t box[2] = {64, box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
 
 namespace {
 using namespace sm100;
@@ -155,82 +134,51 @@ extern "C" int qdelta_selftest_umma(const void* A, const void* B, float* D, int 
     if (!make_tmap_bf16_2d(&mA, A, a.CA, a.RA, (uint64_t)a.CA * 2, a.RA)) return QD_ERR_CUDA;
     if (!make_tmap_bf16_2d(&mB, B, a.CB, a.RB, (uint64_t)a.CB * 2, a.RB)) return QD_ERR_CUDA;
     const size_t smem = 65536 + 1024;
-    if (cudaFuncSetAttribute(k_selftest, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return QD_ERR_CUDA;
+    if (set_max_smem_once(reinterpret_cast<const void*>(k_selftest), smem) != cudaSuccess) return QD_ERR_CUDA;
     k_selftest<<<1, 128, smem, (cudaStream_t)stream>>>(mA, mB, a);
     return cudaGetLastError() == cudaSuccess ? QD_OK : QD_ERR_CUDA;
 }
 
-// ---- MMA issue-rate probe (timing only; operands are zeros) ------------------------------------------
 namespace qd {
 namespace {
 using namespace sm100;
 
-// `nthr` issuing threads (lane 0 of warps 0..nthr-1), each issuing `reps` products D[128 x N] += A B^T (K = 128,
-// 8 instructions, descriptors precomputed, fully unrolled) into its own accumulator.
-template <int N, bool TS>
-__global__ void __launch_bounds__(128) k_mma_rate(int nthr, int reps, long long* out) {
-    extern __shared__ __align__(1024) unsigned char smem_raw[];
-    unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+// Every thread waits on a barrier that is never completed.  out[0] <- QD_ERR_TIMEOUT when the wait gave up (QD_OK if it
+// did not, which would be a bug), out[1] <- nanoseconds thread 0 spent in the wait.
+__global__ void __launch_bounds__(128) k_selftest_timeout(unsigned* out, unsigned limit_ns) {
     __shared__ uint64_t bar;
     __shared__ uint32_t tmem_slot;
+    __shared__ int expired;
     const int tid = threadIdx.x, warp = tid >> 5;
-    for (int i = tid; i < (32768 + 65536) / 16; i += 128) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
-    if (tid == 0) { mbar_init(&bar, (uint32_t)nthr); mbar_init_fence(); }
-    if (warp == 0) { tmem_alloc(&tmem_slot, 512); tmem_relinquish(); }
-    fence_proxy_async();
+    if (tid == 0) {
+        mbar_init(&bar, 1);
+        mbar_init_fence();
+        expired = 0;
+    }
+    if (warp == 0) { tmem_alloc(&tmem_slot, 32); tmem_relinquish(); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tb = tmem_slot;
-    if ((tid & 31) == 0 && warp < nthr) {
-        const uint32_t sa = smem_u32(smem), sb = smem_u32(smem + 32768);
-        constexpr uint32_t idesc = make_idesc(128, N, false, false);
-        const uint64_t a0 = desc_kmajor(sa), b0 = desc_kmajor(sb);
-        constexpr uint32_t b_blk = (uint32_t)N * 128u;
-        const uint32_t tA = tb + 448;
-        const uint32_t d = tb + (uint32_t)warp * (N > 64 ? 64u : (uint32_t)N);   // accumulators may overlap for N = 256: timing only
-        uint64_t ad[8], bd[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            ad[k] = a0 + (((uint32_t)(k >> 2) * 16384u + (uint32_t)(k & 3) * 32u) >> 4);
-            bd[k] = b0 + (((uint32_t)(k >> 2) * b_blk + (uint32_t)(k & 3) * 32u) >> 4);
-        }
-        const long long t0 = clock64();
-#pragma unroll 1
-        for (int r = 0; r < reps; ++r) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                if (TS) umma_ts(d, tA + k * 8, bd[k], idesc, true);
-                else umma_ss(d, ad[k], bd[k], idesc, true);
-            }
-        }
-        const long long t1 = clock64();
-        umma_commit(&bar);
-        mbar_wait(&bar, 0);
-        const long long t2 = clock64();
-        if (warp == 0) { out[0] = t1 - t0; out[1] = t2 - t0; }
+    const uint32_t tbase = tmem_slot;
+    const uint32_t t0 = global_timer_lo();
+    if (!mbar_wait(&bar, 0, limit_ns)) expired = 1;
+    const uint32_t t1 = global_timer_lo();
+    __syncthreads();
+    if (tid == 0) {
+        out[0] = expired ? (unsigned)QD_ERR_TIMEOUT : (unsigned)QD_OK;
+        out[1] = t1 - t0;
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tb, 512);
+    if (warp == 0) tmem_dealloc(tbase, 32);
 }
 
 }  // namespace
 }  // namespace qd
 
-// Timing probe, not part of the public header.  out[0] = cycles thread 0 needed to issue, out[1] = cycles until
-// every issuing thread's products have completed.
-extern "C" int qdelta_selftest_mma_rate(int N, int nthr, int ts, int reps, long long* out, qd_stream stream) {
-    using namespace qd;
-    if (!out || nthr < 1 || nthr > 4 || (N != 64 && N != 128 && N != 256)) return QD_ERR_INVALID_ARG;
-    const size_t smem = 32768 + 65536 + 1024;
-    auto launch = [&](auto kern) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return (int)QD_ERR_CUDA;
-        kern<<<1, 128, smem, (cudaStream_t)stream>>>(nthr, reps, out);
-        return cudaGetLastError() == cudaSuccess ? (int)QD_OK : (int)QD_ERR_CUDA;
-    };
-    if (N == 64) return ts ? launch(k_mma_rate<64, true>) : launch(k_mma_rate<64, false>);
-    if (N == 128) return ts ? launch(k_mma_rate<128, true>) : launch(k_mma_rate<128, false>);
-    return ts ? launch(k_mma_rate<256, true>) : launch(k_mma_rate<256, false>);
+// Not part of the public header: used by the GPU tests.  out: device pointer to two 32-bit words.
+extern "C" int qdelta_selftest_timeout(unsigned* out, unsigned limit_ns, qd_stream stream) {
+    if (!out || limit_ns == 0 || limit_ns > 100u * 1000u * 1000u) return QD_ERR_INVALID_ARG;   // at most 0.1 s
+    qd::k_selftest_timeout<<<1, 128, 0, (cudaStream_t)stream>>>(out, limit_ns);
+    return cudaGetLastError() == cudaSuccess ? QD_OK : QD_ERR_CUDA;
 }

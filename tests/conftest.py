@@ -24,3 +24,19 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """With QD_PARITY_LOG=<file>: dump the error figures the GPU parity tests collected (max-normalised, rms-relative,
+    worst sequence) as JSON."""
+    path = os.environ.get("QD_PARITY_LOG")
+    if not path:
+        return
+    try:
+        import json
+        import gpu_util
+    except Exception:
+        return
+    if gpu_util.LOG:
+        with open(path, "w") as f:
+            json.dump([dict(zip(("label", "tensor", "max", "rms", "per_seq"), r)) for r in gpu_util.LOG], f, indent=0)

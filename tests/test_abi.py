@@ -48,7 +48,10 @@ def test_static_forward_rejects_shapes_beyond_its_scratch(lib):
     big = QdShape(8, 2048, 16, 128, 128, 64, 1)
     rc = lib.qdelta_chunk_fwd_static(ctypes.byref(big), fake, fake, fake, fake, None, None, None, fake, None, None, None)
     assert rc == 6 and "STATIC_SCRATCH" in status_string(rc)
-    bad = QdShape(8, 2000, 16, 128, 128, 64, 1)
+    # a bad shape is reported with the code qdelta_chunk_fwd gives it
+    bad = QdShape(8, 2048, 16, 96, 128, 64, 1)
+    assert lib.qdelta_chunk_fwd_static(ctypes.byref(bad), fake, fake, fake, fake, None, None, None, fake, None, None, None) == 2
+    bad = QdShape(8, 0, 16, 128, 128, 64, 1)
     assert lib.qdelta_chunk_fwd_static(ctypes.byref(bad), fake, fake, fake, fake, None, None, None, fake, None, None, None) == 1
     ok = QdShape(1, 2048, 16, 128, 128, 64, 1)
     assert lib.qdelta_chunk_fwd_static(ctypes.byref(ok), fake, fake, fake, fake, None, None, None, fake, None, fake + 2, None) == 1
@@ -59,7 +62,15 @@ def test_workspace_size_and_shape_validation(lib):
     s = QdShape(8, 2048, 16, 128, 128, 64, 1)
     f, b = chunk_workspace_bytes(s, False), chunk_workspace_bytes(s, True)
     assert 0 < f < b and f % 256 == 0 and b % 256 == 0
-    for bad in (QdShape(8, 2000, 16, 128, 128, 64, 1), QdShape(8, 2048, 16, 96, 128, 64, 1),
+    # a sequence length that is not a multiple of the chunk is padded inside the workspace: T = 1985 .. 2048 need the same
+    assert chunk_workspace_bytes(QdShape(8, 2000, 16, 128, 128, 64, 1), True) == b
+    assert chunk_workspace_bytes(QdShape(8, 1920, 16, 128, 128, 64, 1), True) < b
+    assert chunk_workspace_bytes(QdShape(1, 100, 2, 64, 64, 64, 0), False) == chunk_workspace_bytes(QdShape(1, 128, 2, 64, 64, 64, 0), False)
+    assert lib.qdelta_chunk_path(ctypes.byref(s)) == 1 and lib.qdelta_chunk_path(ctypes.byref(QdShape(8, 2000, 16, 128, 128, 64, 1))) == 1
+    assert lib.qdelta_chunk_path(ctypes.byref(QdShape(1, 256, 2, 64, 64, 64, 0))) == 0
+    assert lib.qdelta_chunk_path(ctypes.byref(QdShape(1, 256, 2, 64, 64, 64, 1))) == 0
+    assert lib.qdelta_chunk_path(ctypes.byref(QdShape(1, 256, 2, 96, 64, 64, 1))) == -1
+    for bad in (QdShape(8, 2048, 16, 96, 128, 64, 1),
                 QdShape(8, 2048, 16, 128, 128, 32, 1), QdShape(0, 2048, 16, 128, 128, 64, 1),
                 QdShape(8, 2048, 16, 128, 128, 64, 7)):
         with pytest.raises(QdeltaError):
