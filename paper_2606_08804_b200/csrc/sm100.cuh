@@ -39,29 +39,27 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up about `limit_ns` nanoseconds of the global timer after it began (each poll may itself block
-// for a short, hardware-defined time).  Returns false on expiry; the caller records the failure and leaves.  One second
-// is several hundred times the longest kernel of this library and far inside any host-side watchdog.  Reading the
-// global timer is slow (a wait that looked at it on every poll made the chunk-backward kernel 6 % slower), so the
-// timer is read only every kPollsPerTimerRead unsuccessful polls; ordinary waits end long before the first read.
-// The low 32 bits of the timer wrap every 4.29 s, so differences below that are exact.
+// Bounded wait: gives up about `limit_ns` nanoseconds of the global timer after its first unsuccessful poll.  Returns
+// false on expiry; the caller records the failure and leaves.  One second is several hundred times the longest kernel
+// of this library and far inside any host-side watchdog.  The low 32 bits of the timer wrap every 4.29 s, so differences
+// below that are exact.  How often a waiting thread polls matters: polls are shared-memory traffic that competes with
+// the operand reads of the MMAs.  Measured on the chunk-backward kernel: a tight polling loop 0.347 ms, the timer read
+// every 64 polls 0.303 ms, the timer read after every poll (this loop) 0.289 ms; suspend-time hints on try_wait
+// (0.5 - 50 us) 0.292 ms and slower state chains.
 __device__ __forceinline__ uint32_t global_timer_lo() {
     uint32_t t;
     asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t));
     return t;
 }
 constexpr uint32_t kWaitLimitNs = 1000u * 1000u * 1000u;
-constexpr uint32_t kPollsPerTimerRead = 64;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit_ns = kWaitLimitNs) {
     uint32_t t0 = 0;
 #pragma unroll 1
-    for (uint32_t polls = 1;; ++polls) {
+    for (uint32_t polls = 0;; ++polls) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((polls & (kPollsPerTimerRead - 1)) == 0) {
-            const uint32_t now = global_timer_lo();
-            if (polls == kPollsPerTimerRead) t0 = now;
-            else if (now - t0 > limit_ns) return false;
-        }
+        const uint32_t now = global_timer_lo();          // also paces the polls
+        if (polls == 0) t0 = now;
+        else if (now - t0 > limit_ns) return false;
     }
 }
 

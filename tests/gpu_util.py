@@ -10,7 +10,7 @@ TOL = {"f32": 1e-4, "bf16": 2e-2}     # per tensor: max|gpu - ref| / max|ref|  (
 #   per_seq  max|gpu - ref| / max|ref| taken separately over every (batch, head) sequence, worst sequence reported
 #            (one large entry elsewhere in the tensor cannot hide a bad sequence).
 TOL_RMS = {"f32": 5e-5, "bf16": 1e-2}
-TOL_SEQ = {"f32": 2e-4, "bf16": 4e-2}
+TOL_SEQ = {"f32": 1e-4, "bf16": 2e-2}     # the contract's bar, but met by every sequence on its own
 LOG = []                               # (label, tensor name, max, rms, per_seq) of every comparison, dumped by conftest
 TDT = {"f32": torch.float32, "bf16": torch.bfloat16}
 
