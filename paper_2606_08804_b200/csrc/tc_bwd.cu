@@ -333,6 +333,11 @@ __device__ __forceinline__ void ld8(uint32_t taddr, float* v) { tmem_ld8(taddr, 
 
 // Two warpgroups: warpgroup w (threads 128w..128w+127) owns TMEM columns [32w, 32w+32) of every
 // 64-column accumulator; inside a warpgroup thread l owns TMEM lane l.
+// HAS_LAM = false: lambda is absent and d lambda is not asked for (the gated delta rule, Eq. 3): X = K, nothing is built,
+// no column sum for d lambda.  HAS_ALPHA = false: alpha is absent and d alpha is not asked for (no forget gate; with
+// HAS_LAM = false too this is DeltaNet, Eq. 2): every decay factor is 1 and none of the sums that only feed d alpha is
+// taken.  The <true, true> instance serves every other case (an absent input then reads as lambda = 0, alpha = 1).
+template <bool HAS_LAM, bool HAS_ALPHA>
 __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_constant__ CUtensorMap mapQ,
                                                               const __grid_constant__ CUtensorMap mapK,
                                                               const __grid_constant__ CUtensorMap mapV,
@@ -464,6 +469,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                    adDt = smem_u32(sm + odDt), aH = smem_u32(sm + oH), adH = smem_u32(sm + odH);
     const uint32_t adPG = smem_u32(sm + odPG), adTb = smem_u32(sm + odTb), adW = smem_u32(sm + odW),
                    aN = smem_u32(sm + oN), adXK = smem_u32(sm + odXK);
+    constexpr bool has_lam = HAS_LAM, has_alpha = HAS_ALPHA, want_dl = HAS_LAM, want_da = HAS_ALPHA;
+    const uint32_t aXe = has_lam ? aX : aK;
 
     if (tid >= kBwdCompute) {
         // =============================== issuing warp: TMA copies and MMAs ===============================
@@ -510,11 +517,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             if (lead) {
                 tc_fence_after();
                 // the product that the dependent chain waits for goes first, the two that are needed late after it
-                umma_product<false, true>(T3, aX, 8192, adW, 8192, C, D, false);            // X dW<-^T         [s][r]
+                umma_product<false, true>(T3, aXe, 8192, adW, 8192, C, D, false);           // X dW<-^T         [s][r]
                 umma_commit(&bm_2);
                 umma_product<true, true>(T5, adH, 16384, aDt, 8192, C, D, false);           // dh Delta^T       [i][s]
-                umma_product<false, false>(T0, aX, 8192, aK, 8192, C, D, false);            // X K^T            [r][i]
-                umma_product<false, false>(T7, aX - 8192, 8192, aK, 8192, C, D, false);     // once more, rows r on lanes 64 + r
+                umma_product<false, false>(T0, aXe, 8192, aK, 8192, C, D, false);           // X K^T            [r][i]
+                umma_product<false, false>(T7, aXe - 8192, 8192, aK, 8192, C, D, false);    // once more, rows r on lanes 64 + r
             }
             nb_sync(kNbDV, kBwdThreads);                                 // the dv staging tile is complete, T6 has been read
             if (lead) {
@@ -541,7 +548,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             if (lead) {
                 tc_fence_after();
                 umma_product<true, false>(T7, aK, 8192, adXK, 8192, C, C, false);           // (dXK K)^T        [i][r]
-                umma_product<true, true>(T1, aX, 8192, adXK, 8192, C, C, false);            // (dXK^T X)^T      [i][s]
+                umma_product<true, true>(T1, aXe, 8192, adXK, 8192, C, C, false);           // (dXK^T X)^T      [i][s]
                 umma_product<true, true>(T1, aQ, 8192, adPG, 8192, C, C, true);             // + (dPG^T Q)^T
                 umma_product<true, false>(T2, aK, 8192, adPG, 8192, C, C, false);           // (dPG K)^T        [i][r]
                 umma_commit(&bm_5);
@@ -606,7 +613,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     wait(&bar_load, ph);
     wait(&bar_late, ph);
     // ---- X = K + lambda Q (the products that do not read X are already running); partial <dh,h>_F -------
-    {
+    if (has_lam) {
         constexpr int kPer = 16 / (kBwdCompute / 64);     // 16-byte chunks of a row per thread
         const int r = tid & 63, part = tid >> 6;
         const float lm = slam[r];
@@ -626,6 +633,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     tc_fence_before();                                    // also orders the previous chunk's TMEM reads before the new products
     nb_arrive(kNbX, kBwdThreads);
     float dhh_part = 0.f;
+    if (want_da)
 #pragma unroll
     for (int cc = 0; cc < 16 / kNWG; ++cc) {
         const int ci = wg * (16 / kNWG) + cc;                // chunk 0..15 of line l
@@ -683,13 +691,13 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         for (int e = 0; e < 8; ++e) {
             const int s = cb + e;
             const bool on = s < r;
-            const float gm = on ? __expf(gr - sg[s]) : 0.f;
+            const float gm = on ? (has_alpha ? __expf(gr - sg[s]) : 1.f) : 0.f;
             const float d = on ? da[e] : 0.f;
             const float dgx = d * gm * xk[e];
             db += dgx;
             const float aa = br * dgx;
             rAA += aa;
-            sts32(&sAA[r * LDAA + s], aa);
+            if (want_da) sts32(&sAA[r * LDAA + s], aa);
             da[e] = d * br * gm;                               // dXK
         }
         sts128(sm + odXK + sw128_chunk(r, wg * kG8 + g8), pack8(da));
@@ -720,8 +728,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 const float dp = (s <= r) ? v[e] : 0.f;
                 const float pp = dp * pv[e];
                 rPP += pp;
-                sts32(&sPP[r * C + ((s + r) & (C - 1))], pp);   // rotated rows: 64 x 64 floats fit the h^T half exactly
-                pg[e] = (s <= r) ? dp * __expf(gr - sg[s]) : 0.f;
+                if (want_da) sts32(&sPP[r * C + ((s + r) & (C - 1))], pp);   // rotated rows: 64 x 64 floats fit the h^T half exactly
+                pg[e] = (s <= r) ? (has_alpha ? dp * __expf(gr - sg[s]) : dp) : 0.f;
             }
             sts128(sm + odPG + sw128_chunk(r, ck), pack8(pg));
         }
@@ -796,7 +804,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     // ---- the last products; meanwhile the column sums of dA o A and dP o P (kBwdCompute/64 threads per column)
     // and the coefficients of the next chunk -------------------------------------------------------------------
     csync();
-    {
+    if (want_da) {
         const float* sAAc = reinterpret_cast<const float*>(sm + oAA);
         const int r = tid & 63, part = tid >> 6;
         float cA = 0.f, cP = 0.f;
@@ -810,12 +818,14 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         scol[1][part][r] = cP;
     }
     nb_arrive(kNbScr, kBwdThreads);      // the scratch tiles over h^T and dh^T are dead from here on
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 16);
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 8);
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 4);
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 2);
-    dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 1);
-    if (lane == 0) swp[tid >> 5] = dhh_part;
+    if (want_da) {
+        dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 16);
+        dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 8);
+        dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 4);
+        dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 2);
+        dhh_part += __shfl_xor_sync(0xffffffffu, dhh_part, 1);
+        if (lane == 0) swp[tid >> 5] = dhh_part;
+    }
     csync();
     // everything of the decay gradient that does not wait for the last epilogue
     float dg_pre = 0.f;
@@ -867,12 +877,18 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 z[e] = q1 * qv;
                 dx[e] = dxe * qv;
             }
-            const float dls = col_reduce8(dx, lane), t1s = col_reduce8(z, lane), kds = col_reduce8(u, lane);
-            if ((lane & 3) == 0) {
-                const int col = cb + col8_of_lane(lane);
-                sred[0][wq][col] = kds;
-                sred[1][wq][col] = dls;
-                sred[2][wq][col] = t1s;
+            // column sums over the d_k index (across the lanes): d lambda, and the two that only the decay gradient needs
+            if (want_dl) {
+                const float dls = col_reduce8(dx, lane);
+                if ((lane & 3) == 0) sred[1][wq][cb + col8_of_lane(lane)] = dls;
+            }
+            if (want_da) {
+                const float t1s = col_reduce8(z, lane), kds = col_reduce8(u, lane);
+                if ((lane & 3) == 0) {
+                    const int col = cb + col8_of_lane(lane);
+                    sred[0][wq][col] = kds;
+                    sred[2][wq][col] = t1s;
+                }
             }
         }
     }
@@ -881,17 +897,17 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     nb_arrive(kNbOut, kBwdThreads);
     csync();
     // ---- decay gradient ----------------------------------------------------------------------------
-    if (tid < C) {
+    if (tid < C && (want_dl || want_da)) {
         const int r = tid;
         float kd = 0.f, dl = 0.f, t1 = 0.f;
 #pragma unroll
         for (int w4 = 0; w4 < 4; ++w4) { kd += sred[0][w4][r]; dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
         sdg[r] = t1 + dg_pre - kd;
         skd[r] = kd;                            // summed below into dg of the last token
-        if (p.dlam && r < live) p.dlam[(row0 + r) * p.H + hh] = dl;
+        if (want_dl && r < live) p.dlam[(row0 + r) * p.H + hh] = dl;
     }
     csync();
-    if (tid < 32) {
+    if (tid < 32 && want_da) {
         // warp 0: lane owns tokens 2*lane, 2*lane+1; d log alpha_i = sum_{r >= i} dg_r (suffix sums)
         const float a = sdg[2 * lane];
         float b2 = sdg[2 * lane + 1];
@@ -978,14 +994,18 @@ cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
     p.g = (const float*)(a.ws + a.TL.g);
     p.dbeta = a.dbeta; p.dalpha = a.dalpha; p.dlam = a.dlam;
     p.status = (unsigned*)(a.ws + a.TL.status);
-    cudaError_t e = set_smem(k_tc_chunk_bwd, kBwdSmem);
+    // the instance without lambda / without the forget gate needs the input AND its gradient to be absent
+    const bool lam = a.lam || a.dlam, alpha = a.alpha || a.dalpha;
+    auto kern = lam ? (alpha ? k_tc_chunk_bwd<true, true> : k_tc_chunk_bwd<true, false>)
+                    : (alpha ? k_tc_chunk_bwd<false, true> : k_tc_chunk_bwd<false, false>);
+    cudaError_t e = set_smem(kern, kBwdSmem);
     if (e != cudaSuccess) return e;
     // persistent: one CTA per SM walks the work items with stride gridDim.x
     int dev = 0, sms = 0;
     if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
     if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
     const unsigned grid = (unsigned)std::min<uint64_t>(BH * N, (uint64_t)sms);
-    return launch_overlapped(k_tc_chunk_bwd, dim3(grid), dim3(kBwdThreads), kBwdSmem, a.stream, mQ, mK, mV, mdO, mMt, mP,
+    return launch_overlapped(kern, dim3(grid), dim3(kBwdThreads), kBwdSmem, a.stream, mQ, mK, mV, mdO, mMt, mP,
                              mDt, mdDt, mHs, mdHs, mdQ, mdK, mdV, p);
 }
 

@@ -65,9 +65,13 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char *sQ = smem, *sK = smem + 32768, *sV = smem + 65536;
-    unsigned char* sX = sQ;                                     // X overwrites Q once Q K^T has been formed
-    float* sA = reinterpret_cast<float*>(sK);                   // A^T [2][column i][row r], aliases K once both Grams are read
-    unsigned char* sT = sK;                                     // [2] T_c, [2] T_c diag(gamma): 8 KB each, alias A
+    // lambda absent (the gated delta rule, Eq. 3): X = K, so nothing is built, both Gram products start at once, and
+    // the scratch that otherwise overwrites K overwrites Q instead
+    const bool has_lam = p.lam != nullptr;
+    unsigned char* sX = has_lam ? sQ : sK;                      // X overwrites Q once Q K^T has been formed
+    unsigned char* sScr = has_lam ? sK : sQ;                    // dead once both Grams are read (and diag(gamma)Q is written)
+    float* sA = reinterpret_cast<float*>(sScr);                 // A^T [2][column i][row r]
+    unsigned char* sT = sScr;                                   // [2] T_c, [2] T_c diag(gamma): 8 KB each, alias A
     __shared__ uint64_t bar_load, bar_mma;
     __shared__ uint32_t tmem_slot;
     __shared__ float sg[128], sbeta[128], slam[128], swsum[4];
@@ -131,8 +135,9 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     }
     if (tid == 0) {
         tc_fence_after();
-        // G2 = Q K^T -> columns [128,256)
+        // G2 = Q K^T -> columns [128,256);  without lambda also G1 = K K^T -> columns [0,128)
         umma_product<false, false>(tbase + 128, smem_u32(sQ), 16384, smem_u32(sK), 16384, 128, 128, false);
+        if (!has_lam) umma_product<false, false>(tbase, smem_u32(sK), 16384, smem_u32(sK), 16384, 128, 128, false);
         umma_commit(&bar_mma);
     }
     // row-wise work: 16 lanes cover one 256-byte row (chunk `ch` of 16 bytes each), 16 rows per pass
@@ -158,33 +163,35 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         if (warp == 0) tmem_dealloc(tbase, 256);
         return;
     }
-    // X = K + lambda Q, in place over Q (K-major swizzled layout)
+    if (has_lam) {
+        // X = K + lambda Q, in place over Q (K-major swizzled layout)
 #pragma unroll 4
-    for (int it = 0; it < 8; ++it) {
-        const int row = it * 16 + rsub;
-        const uint32_t off = coff + sw128_chunk(row, ch & 7);
-        const float lm = slam[row];
-        float qv[8], kv[8];
-        load8(sQ + off, qv);
-        load8(sK + off, kv);
+        for (int it = 0; it < 8; ++it) {
+            const int row = it * 16 + rsub;
+            const uint32_t off = coff + sw128_chunk(row, ch & 7);
+            const float lm = slam[row];
+            float qv[8], kv[8];
+            load8(sQ + off, qv);
+            load8(sK + off, kv);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) kv[e] = fmaf(lm, qv[e], kv[e]);
-        sts128(sX + off, pack8(kv));
-    }
-    fence_proxy_async();
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
-        tc_fence_after();
-        // G1 = X K^T -> columns [0,128)
-        umma_product<false, false>(tbase, smem_u32(sX), 16384, smem_u32(sK), 16384, 128, 128, false);
-        umma_commit(&bar_mma);
-    }
-    fail = !mbar_wait(&bar_mma, 1);
-    if (__syncthreads_or(fail)) {
-        if (tid == 0) *p.status = QD_ERR_TIMEOUT;
-        if (warp == 0) tmem_dealloc(tbase, 256);
-        return;
+            for (int e = 0; e < 8; ++e) kv[e] = fmaf(lm, qv[e], kv[e]);
+            sts128(sX + off, pack8(kv));
+        }
+        fence_proxy_async();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0) {
+            tc_fence_after();
+            // G1 = X K^T -> columns [0,128)
+            umma_product<false, false>(tbase, smem_u32(sX), 16384, smem_u32(sK), 16384, 128, 128, false);
+            umma_commit(&bar_mma);
+        }
+        fail = !mbar_wait(&bar_mma, 1);
+        if (__syncthreads_or(fail)) {
+            if (tid == 0) *p.status = QD_ERR_TIMEOUT;
+            if (warp == 0) tmem_dealloc(tbase, 256);
+            return;
+        }
     }
     tc_fence_after();
     // A = strictLower(beta_r Gamma_ri (x_r . k_i)) -> shared fp32, transposed;  P = Gamma_ri (q_r . k_i), i <= r -> workspace
@@ -291,7 +298,7 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         }
         umma_commit(&bar_mma);
     }
-    fail = !mbar_wait(&bar_mma, 0);
+    fail = !mbar_wait(&bar_mma, has_lam ? 0 : 1);          // third phase of the barrier with lambda, second without
     if (__syncthreads_or(fail)) {
         if (tid == 0) *p.status = QD_ERR_TIMEOUT;
         if (warp == 0) tmem_dealloc(tbase, 256);
@@ -338,6 +345,7 @@ struct ChainParams {
     const float* h0;
     float* hT;
     int save;                  // also store, per chunk, the bf16 entry state (mapHs) and Delta^T (mapDt)
+    int has_alpha;             // 0: no forget gate (alpha absent), every decay factor is 1
     unsigned* status;
 };
 
@@ -480,7 +488,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                         d1[e] = u[e] * sc[cc * 8 + e];
                     }
                     sts128(sD + off, pack8(u));
-                    sts128(sDs + off, pack8(d1));
+                    if (p.has_alpha) sts128(sDs + off, pack8(d1));      // without a forget gate the scaled copy is Delta itself
                 }
             }
             tc_fence_before();
@@ -517,7 +525,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         const bool lead = (tid & 31) == 0;
         grid_dep_wait();
         grid_dep_launch();
-        const uint32_t aH = smem_u32(sH), aD = smem_u32(sD), aDs = smem_u32(sDs);
+        const uint32_t aH = smem_u32(sH), aD = smem_u32(sD), aDs = p.has_alpha ? smem_u32(sDs) : smem_u32(sD);
         for (int n = 0; n < p.N; ++n) {
             const uint32_t st = smem_u32(smem + (n & 1) * kStage);
             const uint32_t tO = tO0 + 64 * (n & 1);
@@ -702,6 +710,7 @@ cudaError_t tc_chain_fwd(const ChunkArgs& a) {
     p.g = (const float*)(a.ws + a.TL.g);
     p.h0 = a.h0; p.hT = a.hT;
     p.save = a.save ? 1 : 0;
+    p.has_alpha = a.alpha ? 1 : 0;
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_chain_fwd, kChainSmem);
     if (e != cudaSuccess) return e;

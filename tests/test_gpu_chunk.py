@@ -307,3 +307,26 @@ def test_backward_right_behind_the_kernels_that_write_its_inputs():
         torch.cuda.synchronize()
         for n in ("dq", "dk", "dv", "dbeta", "dalpha", "dlam", "dh0"):
             gu.check(_label(cfg, " behind producers"), n, g[n], ref[n], cfg.dtype, state=(n == "dh0"))
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_gradients_of_absent_coefficients_on_request(dtype):
+    # alpha = NULL means alpha == 1 and lambda = NULL means lambda == 0; their gradients at those values are still
+    # defined and are written when the caller passes buffers for them
+    from paper_2606_08804_b200 import binding as qd
+    base = gen.CONFIGS["cfg2"] if dtype == "bf16" else replace(gen.CONFIGS["cfg0"], h0=True, backward=True)
+    cfg = replace(base, B=2, H=2, T=192, seed=67)
+    d = dict(gen.make_chunk_inputs(cfg), alpha=None, lam=None)
+    t = gu.dev_inputs(d, cfg.dtype)
+    ref = gu.oracle_bwd(d)
+    for reuse in (False, True):
+        ws = None
+        if reuse:
+            _, _, ws = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], None, None, t["h0"], save_for_bwd=True)
+        out = {"dalpha": torch.full((cfg.B, cfg.T, cfg.H), float("nan"), device="cuda"),
+               "dlam": torch.full((cfg.B, cfg.T, cfg.H), float("nan"), device="cuda")}
+        g = qd.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], None, None, t["h0"], t["dO"], t["dhT"], workspace=ws,
+                         reuse_fwd=reuse, out=out)
+        torch.cuda.synchronize()
+        for n in ("dq", "dk", "dv", "dbeta", "dalpha", "dlam", "dh0"):
+            gu.check(_label(cfg, " absent coefficients, gradients requested"), n, g[n], ref[n], cfg.dtype, state=(n == "dh0"))
