@@ -489,8 +489,27 @@ def bench_decode(args, qd, gen, torch, pk, pk_kind):
     nstates = cfg.B * cfg.H
     bytes_step = nstates * (2 * cfg.dk * cfg.dv * 4 + 2 * (2 * cfg.dk + cfg.dv) + 6 + 2 * cfg.dv)
     gbs = bytes_step / (ms * 1e-3) / 1e9
+    # multi-token step (S tokens per call share one read and one write of the state)
+    multi = {}
+    for S in (2, 4, 8):
+        tk = gen.make_decode_tokens(cfg, 100, S)
+        tk = {n: torch.from_numpy(np.ascontiguousarray(np.moveaxis(a, 0, 1))).to("cuda", bf) for n, a in tk.items()}
+        oS = torch.empty((cfg.B, S, cfg.H, cfg.dv), dtype=bf, device="cuda")
+        calls = max(50, nsteps // S)
+        for _ in range(5):
+            qd.recurrent_steps(tk["q"], tk["k"], tk["v"], tk["beta"], tk["alpha"], tk["lam"], state, oS)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(calls):
+            qd.recurrent_steps(tk["q"], tk["k"], tk["v"], tk["beta"], tk["alpha"], tk["lam"], state, oS)
+        e1.record()
+        torch.cuda.synchronize()
+        msS = e0.elapsed_time(e1) / calls
+        bytesS = nstates * (2 * cfg.dk * cfg.dv * 4 + S * (2 * (2 * cfg.dk + cfg.dv) + 6 + 2 * cfg.dv))
+        multi["S=%d" % S] = {"us_per_call": msS * 1e3, "tokens_per_s": cfg.B * S / (msS * 1e-3),
+                             "achieved_gbs": bytesS / (msS * 1e-3) / 1e9, "frac": bytesS / (msS * 1e-3) / 1e9 / pk["hbm_gbs"]}
     return {"workload": "cfg4: batch=%d H=%d dk=%d dv=%d fp32 state in place, bf16 tokens" % (cfg.B, cfg.H, cfg.dk, cfg.dv),
-            "steps": nsteps, "us_per_step": ms * 1e3, "tokens_per_s": cfg.B / (ms * 1e-3),
+            "steps": nsteps, "us_per_step": ms * 1e3, "tokens_per_s": cfg.B / (ms * 1e-3), "multi_token": multi,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / pk["hbm_gbs"], "peak_kind": "of " + pk_kind,
                          "algorithmic_bytes_per_launch": bytes_step, "state_larger_than_l2": True}}

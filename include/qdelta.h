@@ -29,7 +29,8 @@
  *     states and the workspace must be 16-byte aligned; coefficient tensors (and the decode step's o)
  *     need only the alignment of their element type.
  *   - Coefficient domains: beta, lambda in [0,1], alpha in (0,1] (Section 3.3.1); not checked on device.
- *   - Return value: QD_OK, or an error code reported synchronously; on error nothing was enqueued.
+ *   - Return value: QD_OK, or an error code reported synchronously.  After a validation error (every code but
+ *     QD_ERR_CUDA) nothing was enqueued; QD_ERR_CUDA means a CUDA call failed part-way, earlier kernels of the call may run.
  *     Conditions found on the device (a bounded wait that ran out) are written to the first
  *     32-bit word of the workspace and can be read with qdelta_workspace_status after the
  *     caller has synchronised the stream.
@@ -127,6 +128,20 @@ int qdelta_recurrent_step(int B, int H, int dk, int dv, int dtype,
                           const void *q, const void *k, const void *v,
                           const void *beta, const void *alpha, const void *lambda,
                           float *state, void *o, qd_stream stream);
+
+/*
+ * S consecutive tokens of the same recurrence (Section 3.3.1) per call, for multi-token / speculative decoding: the
+ * state is read once and written once for all S tokens instead of once per token.  Token tensors are token-major like
+ * those of the chunkwise calls:
+ *     q,k [B,S,H,dk]   v,o [B,S,H,dv]   beta/alpha/lambda [B,S,H]   (alpha, lambda may be NULL)
+ *     state [B,H,dk,dv] fp32, UPDATED IN PLACE to the state after the S-th token;  o_s is read out after token s.
+ * The result is bit-identical to S calls of qdelta_recurrent_step.  S >= 1; for long runs of tokens (a prompt) use
+ * qdelta_chunk_fwd with h0 / hT, which runs on the tensor cores.  Needs no workspace.
+ */
+int qdelta_recurrent_steps(int B, int S, int H, int dk, int dv, int dtype,
+                           const void *q, const void *k, const void *v,
+                           const void *beta, const void *alpha, const void *lambda,
+                           float *state, void *o, qd_stream stream);
 
 /* Copies the device status word of `workspace` to *status_out (a qd_status) with a blocking
  * 4-byte device-to-host copy on `stream`.  Returns QD_OK or QD_ERR_CUDA / QD_ERR_INVALID_ARG. */

@@ -18,7 +18,8 @@ QD_FWD_SAVE_FOR_BWD, QD_BWD_REUSE_FWD = 1, 2
 EXPORTS = ("qdelta_chunk_workspace_bytes", "qdelta_chunk_fwd", "qdelta_chunk_bwd",
            "qdelta_recurrent_step", "qdelta_workspace_status", "qdelta_status_string",
            "qdelta_profile_enable", "qdelta_profile_stage_count", "qdelta_profile_stage_name",
-           "qdelta_profile_read", "qdelta_chunk_fwd_static", "qdelta_chunk_path")
+           "qdelta_profile_read", "qdelta_chunk_fwd_static", "qdelta_chunk_path",
+           "qdelta_recurrent_steps")
 
 
 class QdShape(ctypes.Structure):
@@ -55,6 +56,8 @@ def load():
     lib.qdelta_chunk_fwd_static.argtypes = [ctypes.POINTER(QdShape)] + [vp] * 9 + [vp, vp]
     lib.qdelta_recurrent_step.restype = i
     lib.qdelta_recurrent_step.argtypes = [i] * 5 + [vp] * 8 + [vp]
+    lib.qdelta_recurrent_steps.restype = i
+    lib.qdelta_recurrent_steps.argtypes = [i] * 6 + [vp] * 8 + [vp]
     lib.qdelta_workspace_status.restype = i
     lib.qdelta_workspace_status.argtypes = [vp, ctypes.POINTER(i), vp]
     lib.qdelta_status_string.restype = ctypes.c_char_p
@@ -249,4 +252,22 @@ def recurrent_step(q, k, v, beta, alpha, lam, state, o=None):
         _ptr(lam, dt, (B, H), "lam"), _ptr(state, torch.float32, (B, H, dk, dv), "state"),
         _ptr(o, dt, (B, H, dv), "o"), _stream())
     _check(rc, "qdelta_recurrent_step")
+    return o
+
+
+def recurrent_steps(q, k, v, beta, alpha, lam, state, o=None):
+    """S decode tokens per call: q,k [B,S,H,dk], v [B,S,H,dv], coefficients [B,S,H]; `state` [B,H,dk,dv] fp32 is
+    updated in place to the state after the last token.  Returns o [B,S,H,dv]."""
+    lib = load()
+    B, S, H, dk = q.shape
+    dv = v.shape[-1]
+    dt = q.dtype
+    if o is None:
+        o = torch.empty((B, S, H, dv), dtype=dt, device=q.device)
+    rc = lib.qdelta_recurrent_steps(
+        B, S, H, dk, dv, _dtype_code(q), _ptr(q, dt, (B, S, H, dk), "q"), _ptr(k, dt, (B, S, H, dk), "k"),
+        _ptr(v, dt, (B, S, H, dv), "v"), _ptr(beta, dt, (B, S, H), "beta"), _ptr(alpha, dt, (B, S, H), "alpha"),
+        _ptr(lam, dt, (B, S, H), "lam"), _ptr(state, torch.float32, (B, H, dk, dv), "state"),
+        _ptr(o, dt, (B, S, H, dv), "o"), _stream())
+    _check(rc, "qdelta_recurrent_steps")
     return o

@@ -216,6 +216,27 @@ int qdelta_recurrent_step(int B, int H, int dk, int dv, int dtype, const void* q
     return QD_OK;
 }
 
+int qdelta_recurrent_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
+                           const void* beta, const void* alpha, const void* lambda, float* state, void* o,
+                           qd_stream stream) {
+    if (B <= 0 || H <= 0 || S <= 0) return QD_ERR_INVALID_ARG;
+    if (dtype != QD_F32 && dtype != QD_BF16) return QD_ERR_UNSUPPORTED;
+    if ((dk != 64 && dk != 128) || (dv != 64 && dv != 128)) return QD_ERR_UNSUPPORTED;
+    if (!q || !k || !v || !beta || !state || !o) return QD_ERR_INVALID_ARG;
+    if ((long long)B * H > 0x3fffffffLL || (long long)B * S * H > 0x7fffffffLL / 128) return QD_ERR_UNSUPPORTED;
+    const void* ptrs[] = {q, k, v, state};
+    for (const void* p : ptrs)
+        if (p && misaligned(p)) return QD_ERR_INVALID_ARG;
+    const void* coef[] = {beta, alpha, lambda, o};
+    for (const void* p : coef)
+        if (p && ((uintptr_t)p & (dtype == QD_BF16 ? 1 : 3))) return QD_ERR_INVALID_ARG;
+    if (timed(ST_DECODE, (cudaStream_t)stream, [&] {
+            return decode_steps(B, S, H, dk, dv, dtype, q, k, v, beta, alpha, lambda, state, o, (cudaStream_t)stream);
+        }) != cudaSuccess)
+        return QD_ERR_CUDA;
+    return QD_OK;
+}
+
 int qdelta_workspace_status(const void* workspace, int* status_out, qd_stream stream) {
     if (!workspace || !status_out) return QD_ERR_INVALID_ARG;
     unsigned w = 0;

@@ -80,6 +80,95 @@ __global__ void __launch_bounds__(NT) k_decode(int dv, const IO* __restrict__ q,
     }
 }
 
+// Several tokens per call (multi-token / speculative decoding): S consecutive tokens of every sequence go through the
+// same recurrence, one after the other, while the state slice stays in registers -- one read and one write of the state
+// for S tokens instead of S of each.  Token tensors are token-major [B, S, H, d] like those of the chunkwise calls.  The
+// arithmetic of one token is exactly that of k_decode, in the same order, so S tokens here give bit-identical results to
+// S single-token calls.
+template <typename IO, int DK, int DVS, int NT>
+__global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, const IO* __restrict__ q, const IO* __restrict__ k,
+                                                     const IO* __restrict__ v, const IO* __restrict__ beta,
+                                                     const IO* __restrict__ alpha, const IO* __restrict__ lam,
+                                                     float* __restrict__ state, IO* __restrict__ o) {
+    constexpr int C4 = DVS / 4, RP = NT / C4, NP = DK / RP;
+    static_assert(NT % C4 == 0 && DK % RP == 0, "bad decode tiling");
+    __shared__ float sx[DK], sq[DK], sk[DK];
+    __shared__ float redx[RP][DVS], redq[RP][DVS];
+    __shared__ float sdelta[DVS];
+    __shared__ float skq[NT / 32];
+    const int nsl = dv / DVS, bh = blockIdx.x / nsl, j0 = (blockIdx.x % nsl) * DVS, tid = threadIdx.x;
+    const int b = bh / H, hh = bh % H;
+    const int c4 = tid % C4, rg = tid / C4;
+
+    float4* base = reinterpret_cast<float4*>(state + (size_t)bh * DK * dv + j0) + c4;
+    const int rstride = dv / 4;
+    float4 h[NP];
+#pragma unroll
+    for (int pz = 0; pz < NP; ++pz) h[pz] = __ldcs(base + (size_t)(pz * RP + rg) * rstride);
+
+    for (int s = 0; s < S; ++s) {
+        const size_t row = ((size_t)b * S + s) * H + hh;        // token row of this head in the [B, S, H] view
+        const float be = ld(beta, row);
+        const float al = alpha ? ld(alpha, row) : 1.f;
+        const float la = lam ? ld(lam, row) : 0.f;
+        float kq = 0.f;
+        for (int i = tid; i < DK; i += NT) {
+            const float qi = ld(q, row * DK + i), ki = ld(k, row * DK + i);
+            sq[i] = qi; sk[i] = ki; sx[i] = fmaf(la, qi, ki);
+            kq = fmaf(ki, qi, kq);
+        }
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) kq += __shfl_xor_sync(0xffffffffu, kq, w);
+        if ((tid & 31) == 0) skq[tid >> 5] = kq;
+        __syncthreads();
+
+        float4 ax = make_float4(0.f, 0.f, 0.f, 0.f), aq = ax;
+#pragma unroll
+        for (int pz = 0; pz < NP; ++pz) {
+            const float xi = sx[pz * RP + rg], qi = sq[pz * RP + rg];
+            ax.x = fmaf(h[pz].x, xi, ax.x); ax.y = fmaf(h[pz].y, xi, ax.y);
+            ax.z = fmaf(h[pz].z, xi, ax.z); ax.w = fmaf(h[pz].w, xi, ax.w);
+            aq.x = fmaf(h[pz].x, qi, aq.x); aq.y = fmaf(h[pz].y, qi, aq.y);
+            aq.z = fmaf(h[pz].z, qi, aq.z); aq.w = fmaf(h[pz].w, qi, aq.w);
+        }
+        *reinterpret_cast<float4*>(&redx[rg][c4 * 4]) = ax;
+        *reinterpret_cast<float4*>(&redq[rg][c4 * 4]) = aq;
+        __syncthreads();
+        if (tid < DVS) {
+            float rx = 0.f, rq = 0.f, kqt = 0.f;
+#pragma unroll
+            for (int r = 0; r < RP; ++r) { rx += redx[r][tid]; rq += redq[r][tid]; }
+#pragma unroll
+            for (int w = 0; w < NT / 32; ++w) kqt += skq[w];
+            const float dl = be * (ld(v, row * dv + j0 + tid) - al * rx);
+            sdelta[tid] = dl;
+            st(o, row * dv + j0 + tid, fmaf(al, rq, kqt * dl));
+        }
+        __syncthreads();
+        const float4 dl = *reinterpret_cast<const float4*>(&sdelta[c4 * 4]);
+#pragma unroll
+        for (int pz = 0; pz < NP; ++pz) {
+            const float ki = sk[pz * RP + rg];
+            h[pz].x = fmaf(al, h[pz].x, ki * dl.x); h[pz].y = fmaf(al, h[pz].y, ki * dl.y);
+            h[pz].z = fmaf(al, h[pz].z, ki * dl.z); h[pz].w = fmaf(al, h[pz].w, ki * dl.w);
+        }
+        __syncthreads();                 // the token's shared arrays are rewritten by the next one
+    }
+#pragma unroll
+    for (int pz = 0; pz < NP; ++pz) __stcs(base + (size_t)(pz * RP + rg) * rstride, h[pz]);
+}
+
+template <typename IO, int DK>
+cudaError_t launch_multi(int B, int S, int H, int dv, const void* q, const void* k, const void* v, const void* beta,
+                         const void* alpha, const void* lam, float* state, void* o, cudaStream_t stream) {
+    constexpr int DVS = 64, NT = 128;
+    dim3 grid((unsigned)(dv / DVS) * (unsigned)(B * H));
+    k_decode_multi<IO, DK, DVS, NT><<<grid, NT, 0, stream>>>(S, H, dv, (const IO*)q, (const IO*)k, (const IO*)v,
+                                                             (const IO*)beta, (const IO*)alpha, (const IO*)lam,
+                                                             state, (IO*)o);
+    return cudaGetLastError();
+}
+
 template <typename IO, int DK>
 cudaError_t launch(int BH, int dv, const void* q, const void* k, const void* v, const void* beta,
                    const void* alpha, const void* lam, float* state, void* o, cudaStream_t stream) {
@@ -102,6 +191,17 @@ cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const 
     }
     if (dk == 128) return launch<float, 128>(BH, dv, q, k, v, beta, alpha, lam, state, o, stream);
     return launch<float, 64>(BH, dv, q, k, v, beta, alpha, lam, state, o, stream);
+}
+
+cudaError_t decode_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
+                         const void* beta, const void* alpha, const void* lam, float* state, void* o,
+                         cudaStream_t stream) {
+    if (dtype == QD_BF16) {
+        if (dk == 128) return launch_multi<__nv_bfloat16, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, stream);
+        return launch_multi<__nv_bfloat16, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, stream);
+    }
+    if (dk == 128) return launch_multi<float, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, stream);
+    return launch_multi<float, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, stream);
 }
 
 }  // namespace qd

@@ -115,6 +115,10 @@ cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const 
                         const void* beta, const void* alpha, const void* lam, float* state, void* o,
                         cudaStream_t stream);
 
+cudaError_t decode_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
+                         const void* beta, const void* alpha, const void* lam, float* state, void* o,
+                         cudaStream_t stream);
+
 // ---- storage-dtype helpers -------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float ld(const T* p, size_t i);
 template <> __device__ __forceinline__ float ld<float>(const float* p, size_t i) { return p[i]; }

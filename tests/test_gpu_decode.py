@@ -101,3 +101,64 @@ def test_decode_matches_chunk_forward_on_gpu():
     den = o.float().abs().max()
     assert ((o2.float() - o.float()).abs().max() / den).item() <= 2e-2
     assert ((state - hT).abs().max() / hT.abs().max()).item() <= 2e-2
+
+
+@pytest.mark.parametrize("dtype,dk,dv,S", [("bf16", 128, 128, 4), ("bf16", 128, 128, 1), ("bf16", 64, 128, 7), ("f32", 64, 64, 5)])
+def test_multi_token_step_is_the_single_step_repeated(dtype, dk, dv, S):
+    # S tokens in one call: bit-identical to S single-token calls, and equal to the oracle's recurrence
+    from paper_2606_08804_b200 import binding as qd
+    cfg = replace(gen.CONFIGS["cfg1"], B=3, H=5, T=S, dk=dk, dv=dv, dtype=dtype, regime="alpha_slow", seed=83)
+    d = gen.make_chunk_inputs(cfg)
+    t = gu.dev_inputs(d, cfg.dtype)
+    st_multi = gu.Guarded((cfg.B, cfg.H, dk, dv), torch.float32, fill=t["h0"])
+    o_multi = gu.Guarded((cfg.B, S, cfg.H, dv), gu.TDT[dtype])
+    qd.recurrent_steps(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], st_multi.t, o_multi.t)
+    st_single = t["h0"].clone()
+    outs = []
+    for s in range(S):
+        c = lambda x: x[:, s].contiguous()
+        outs.append(qd.recurrent_step(c(t["q"]), c(t["k"]), c(t["v"]), c(t["beta"]), c(t["alpha"]), c(t["lam"]), st_single))
+    torch.cuda.synchronize()
+    assert st_multi.intact() and o_multi.intact()
+    assert torch.equal(o_multi.t, torch.stack(outs, dim=1))
+    assert torch.equal(st_multi.t, st_single)
+    ro, rh = gu.oracle_fwd(d)
+    assert gu.rel_err(o_multi.t, ro) <= gu.TOL[dtype] and gu.rel_err(st_multi.t, rh) <= gu.TOL[dtype]
+
+
+def test_prefill_then_multi_token_decode():
+    # a prompt through the chunkwise forward (ragged length), its final state handed to the multi-token decode step:
+    # together they must equal the recurrence over the whole sequence
+    from paper_2606_08804_b200 import binding as qd
+    S, Tp = 6, 150
+    cfg = replace(gen.CONFIGS["cfg1"], B=2, H=3, T=Tp + 2 * S, regime="trained_like", seed=89)
+    d = gen.make_chunk_inputs(cfg)
+    t = gu.dev_inputs(d, cfg.dtype)
+    c = lambda x, a, b: x[:, a:b].contiguous()
+    names = ("q", "k", "v", "beta", "alpha", "lam")
+    pre = [c(t[n], 0, Tp) for n in names]
+    o_pre, state, _ = qd.chunk_fwd(*pre, t["h0"])
+    outs = [o_pre]
+    for j in range(2):
+        seg = [c(t[n], Tp + j * S, Tp + (j + 1) * S) for n in names]
+        outs.append(qd.recurrent_steps(*seg, state))
+    torch.cuda.synchronize()
+    ro, rh = gu.oracle_fwd(d)
+    assert gu.rel_err(torch.cat(outs, dim=1), ro) <= 2e-2
+    assert gu.rel_err(state, rh) <= 2e-2
+
+
+def test_multi_token_step_null_coefficients_and_argument_errors():
+    from paper_2606_08804_b200 import binding as qd
+    cfg = replace(gen.CONFIGS["cfg1"], B=2, H=2, T=3, seed=97)
+    d = dict(gen.make_chunk_inputs(cfg), alpha=None, lam=None)
+    t = gu.dev_inputs(d, cfg.dtype)
+    state = t["h0"].clone()
+    o = qd.recurrent_steps(t["q"], t["k"], t["v"], t["beta"], None, None, state)
+    torch.cuda.synchronize()
+    ro, rh = gu.oracle_fwd(d)
+    assert gu.rel_err(o, ro) <= 2e-2 and gu.rel_err(state, rh) <= 2e-2
+    lib = qd.load()
+    fake = 0x1000
+    assert lib.qdelta_recurrent_steps(1, 0, 1, 64, 64, 0, fake, fake, fake, fake, None, None, fake, fake, None) == 1
+    assert lib.qdelta_recurrent_steps(1, 2, 1, 96, 64, 0, fake, fake, fake, fake, None, None, fake, fake, None) == 2
