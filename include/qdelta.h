@@ -64,8 +64,12 @@ typedef enum { QD_F32 = 0, QD_BF16 = 1 } qd_dtype;
 /* flags of qdelta_chunk_fwd / qdelta_chunk_bwd */
 enum {
     QD_FWD_SAVE_FOR_BWD = 1,  /* fwd: also keep the per-chunk states etc. in a backward-sized workspace */
-    QD_BWD_REUSE_FWD = 2      /* bwd: the workspace still holds what a QD_FWD_SAVE_FOR_BWD forward of the
-                                 SAME inputs left there; skip the recomputation */
+    QD_BWD_REUSE_FWD = 2,     /* bwd: the workspace still holds what a QD_FWD_SAVE_FOR_BWD forward of the
+                                 SAME inputs (and the same QD_COEF_LOGITS setting) left there; skip the recomputation */
+    QD_COEF_LOGITS = 4        /* fwd, bwd, qdelta_recurrent_steps: beta, alpha and lambda hold the pre-activation
+                                 logits z of sigmoid gates (Appendix B: lambda = sigmoid(W h + b)); the kernels use
+                                 sigmoid(z), computed in fp32, and the backward writes dbeta, dalpha, dlambda as
+                                 derivatives with respect to the logits.  NULL alpha / lambda still mean 1 / 0. */
 };
 
 typedef struct {
@@ -135,13 +139,13 @@ int qdelta_recurrent_step(int B, int H, int dk, int dv, int dtype,
  * those of the chunkwise calls:
  *     q,k [B,S,H,dk]   v,o [B,S,H,dv]   beta/alpha/lambda [B,S,H]   (alpha, lambda may be NULL)
  *     state [B,H,dk,dv] fp32, UPDATED IN PLACE to the state after the S-th token;  o_s is read out after token s.
- * The result is bit-identical to S calls of qdelta_recurrent_step.  S >= 1; for long runs of tokens (a prompt) use
+ * The result is bit-identical to S calls of qdelta_recurrent_step.  flags: 0 or QD_COEF_LOGITS.  S >= 1; for long runs of tokens (a prompt) use
  * qdelta_chunk_fwd with h0 / hT, which runs on the tensor cores.  Needs no workspace.
  */
 int qdelta_recurrent_steps(int B, int S, int H, int dk, int dv, int dtype,
                            const void *q, const void *k, const void *v,
                            const void *beta, const void *alpha, const void *lambda,
-                           float *state, void *o, qd_stream stream);
+                           float *state, void *o, unsigned flags, qd_stream stream);
 
 /* Copies the device status word of `workspace` to *status_out (a qd_status) with a blocking
  * 4-byte device-to-host copy on `stream`.  Returns QD_OK or QD_ERR_CUDA / QD_ERR_INVALID_ARG. */

@@ -99,3 +99,34 @@ def decode(state, q, k, v, beta, alpha=None, lam=None):
     tr = lambda a: None if a is None else np.moveaxis(np.asarray(a, np.float64), 0, 1)
     o, hT = forward(tr(q), tr(k), tr(v), tr(beta), tr(alpha), tr(lam), state)
     return np.moveaxis(o, 1, 0), hT
+
+
+def _sigmoid(z):
+    """sigma(z) in fp64 without overflow for large |z|."""
+    z = np.asarray(z, np.float64)
+    e = np.exp(-np.abs(z))
+    return np.where(z >= 0, 1.0 / (1.0 + e), e / (1.0 + e))
+
+
+def gates_from_logits(zbeta, zalpha=None, zlam=None):
+    """The coefficients as sigmoid gates of pre-activation logits (Appendix B writes lambda this way; beta and alpha
+    are gates in (0,1) as well).  An absent alpha / lambda stays absent (alpha == 1, lambda == 0)."""
+    g = lambda z: None if z is None else _sigmoid(z)
+    return _sigmoid(zbeta), g(zalpha), g(zlam)
+
+
+def forward_logits(q, k, v, zbeta, zalpha=None, zlam=None, h0=None):
+    """forward() with beta, alpha, lambda given as logits."""
+    beta, alpha, lam = gates_from_logits(zbeta, zalpha, zlam)
+    return forward(q, k, v, beta, alpha, lam, h0)
+
+
+def backward_logits(q, k, v, zbeta, zalpha, zlam, h0, dO, dhT=None, ckpt=64):
+    """backward() with beta, alpha, lambda given as logits: dbeta, dalpha, dlam are the derivatives with respect to the
+    logits, by the chain rule d sigma(z)/dz = sigma(z)(1 - sigma(z)).  Gradients of absent logits are returned as None."""
+    beta, alpha, lam = gates_from_logits(zbeta, zalpha, zlam)
+    g = backward(q, k, v, beta, alpha, lam, h0, dO, dhT, ckpt)
+    g["dbeta"] = g["dbeta"] * beta * (1.0 - beta)
+    g["dalpha"] = None if alpha is None else g["dalpha"] * alpha * (1.0 - alpha)
+    g["dlam"] = None if lam is None else g["dlam"] * lam * (1.0 - lam)
+    return g

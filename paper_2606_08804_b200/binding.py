@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libqdelta.so")
 
 QD_F32, QD_BF16 = 0, 1
-QD_FWD_SAVE_FOR_BWD, QD_BWD_REUSE_FWD = 1, 2
+QD_FWD_SAVE_FOR_BWD, QD_BWD_REUSE_FWD, QD_COEF_LOGITS = 1, 2, 4
 
 EXPORTS = ("qdelta_chunk_workspace_bytes", "qdelta_chunk_fwd", "qdelta_chunk_bwd",
            "qdelta_recurrent_step", "qdelta_workspace_status", "qdelta_status_string",
@@ -57,7 +57,7 @@ def load():
     lib.qdelta_recurrent_step.restype = i
     lib.qdelta_recurrent_step.argtypes = [i] * 5 + [vp] * 8 + [vp]
     lib.qdelta_recurrent_steps.restype = i
-    lib.qdelta_recurrent_steps.argtypes = [i] * 6 + [vp] * 8 + [vp]
+    lib.qdelta_recurrent_steps.argtypes = [i] * 6 + [vp] * 8 + [u, vp]
     lib.qdelta_workspace_status.restype = i
     lib.qdelta_workspace_status.argtypes = [vp, ctypes.POINTER(i), vp]
     lib.qdelta_status_string.restype = ctypes.c_char_p
@@ -155,8 +155,9 @@ def workspace_status(workspace: torch.Tensor) -> int:
 
 
 def chunk_fwd(q, k, v, beta, alpha=None, lam=None, h0=None, chunk=64, save_for_bwd=False,
-              workspace=None, o=None, hT=None, want_hT=True):
-    """Chunkwise forward.  Returns (o, hT, workspace).  All tensors live on the GPU."""
+              workspace=None, o=None, hT=None, want_hT=True, logits=False):
+    """Chunkwise forward.  Returns (o, hT, workspace).  All tensors live on the GPU.
+    logits=True: beta, alpha, lam hold the logits of sigmoid gates (the kernels apply the sigmoid)."""
     lib = load()
     s = make_shape(q, v, chunk)
     B, T, H, dk, dv, dt = s.B, s.T, s.H, s.dk, s.dv, q.dtype
@@ -172,7 +173,8 @@ def chunk_fwd(q, k, v, beta, alpha=None, lam=None, h0=None, chunk=64, save_for_b
         _ptr(alpha, dt, (B, T, H), "alpha"), _ptr(lam, dt, (B, T, H), "lam"),
         _ptr(h0, torch.float32, (B, H, dk, dv), "h0"), _ptr(o, dt, (B, T, H, dv), "o"),
         _ptr(hT, torch.float32, (B, H, dk, dv), "hT"),
-        workspace.data_ptr(), workspace.numel(), QD_FWD_SAVE_FOR_BWD if save_for_bwd else 0, _stream())
+        workspace.data_ptr(), workspace.numel(),
+        (QD_FWD_SAVE_FOR_BWD if save_for_bwd else 0) | (QD_COEF_LOGITS if logits else 0), _stream())
     _check(rc, "qdelta_chunk_fwd")
     return o, hT, workspace
 
@@ -204,8 +206,9 @@ def chunk_fwd_static(q, k, v, beta, alpha, lam, h0, o, hT=None, status=None, chu
 
 
 def chunk_bwd(q, k, v, beta, alpha, lam, h0, dO, dhT=None, chunk=64, workspace=None,
-              reuse_fwd=False, out=None, want_dh0=True):
-    """Chunkwise backward.  Returns dict(dq, dk, dv, dbeta, dalpha, dlam, dh0) of GPU tensors."""
+              reuse_fwd=False, out=None, want_dh0=True, logits=False):
+    """Chunkwise backward.  Returns dict(dq, dk, dv, dbeta, dalpha, dlam, dh0) of GPU tensors.
+    logits=True: beta, alpha, lam are logits and dbeta, dalpha, dlam are gradients with respect to them."""
     lib = load()
     s = make_shape(q, v, chunk)
     B, T, H, dk, dv, dt = s.B, s.T, s.H, s.dk, s.dv, q.dtype
@@ -233,7 +236,8 @@ def chunk_bwd(q, k, v, beta, alpha, lam, h0, dO, dhT=None, chunk=64, workspace=N
         _ptr(g["dv"], dt, (B, T, H, dv), "dv"), _ptr(g["dbeta"], f32, (B, T, H), "dbeta"),
         _ptr(g["dalpha"], f32, (B, T, H), "dalpha"), _ptr(g["dlam"], f32, (B, T, H), "dlam"),
         _ptr(g["dh0"], f32, (B, H, dk, dv), "dh0"),
-        workspace.data_ptr(), workspace.numel(), QD_BWD_REUSE_FWD if reuse_fwd else 0, _stream())
+        workspace.data_ptr(), workspace.numel(),
+        (QD_BWD_REUSE_FWD if reuse_fwd else 0) | (QD_COEF_LOGITS if logits else 0), _stream())
     _check(rc, "qdelta_chunk_bwd")
     return g
 
@@ -255,7 +259,7 @@ def recurrent_step(q, k, v, beta, alpha, lam, state, o=None):
     return o
 
 
-def recurrent_steps(q, k, v, beta, alpha, lam, state, o=None):
+def recurrent_steps(q, k, v, beta, alpha, lam, state, o=None, logits=False):
     """S decode tokens per call: q,k [B,S,H,dk], v [B,S,H,dv], coefficients [B,S,H]; `state` [B,H,dk,dv] fp32 is
     updated in place to the state after the last token.  Returns o [B,S,H,dv]."""
     lib = load()
@@ -268,6 +272,6 @@ def recurrent_steps(q, k, v, beta, alpha, lam, state, o=None):
         B, S, H, dk, dv, _dtype_code(q), _ptr(q, dt, (B, S, H, dk), "q"), _ptr(k, dt, (B, S, H, dk), "k"),
         _ptr(v, dt, (B, S, H, dv), "v"), _ptr(beta, dt, (B, S, H), "beta"), _ptr(alpha, dt, (B, S, H), "alpha"),
         _ptr(lam, dt, (B, S, H), "lam"), _ptr(state, torch.float32, (B, H, dk, dv), "state"),
-        _ptr(o, dt, (B, S, H, dv), "o"), _stream())
+        _ptr(o, dt, (B, S, H, dv), "o"), QD_COEF_LOGITS if logits else 0, _stream())
     _check(rc, "qdelta_recurrent_steps")
     return o

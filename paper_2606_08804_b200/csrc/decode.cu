@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(NT) k_decode(int dv, const IO* __restrict__ q,
 // arithmetic of one token is exactly that of k_decode, in the same order, so S tokens here give bit-identical results to
 // S single-token calls.
 template <typename IO, int DK, int DVS, int NT>
-__global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, const IO* __restrict__ q, const IO* __restrict__ k,
+__global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, int logits, const IO* __restrict__ q, const IO* __restrict__ k,
                                                      const IO* __restrict__ v, const IO* __restrict__ beta,
                                                      const IO* __restrict__ alpha, const IO* __restrict__ lam,
                                                      float* __restrict__ state, IO* __restrict__ o) {
@@ -108,9 +108,9 @@ __global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, const
 
     for (int s = 0; s < S; ++s) {
         const size_t row = ((size_t)b * S + s) * H + hh;        // token row of this head in the [B, S, H] view
-        const float be = ld(beta, row);
-        const float al = alpha ? ld(alpha, row) : 1.f;
-        const float la = lam ? ld(lam, row) : 0.f;
+        const float be = gate(ld(beta, row), logits);
+        const float al = alpha ? gate(ld(alpha, row), logits) : 1.f;
+        const float la = lam ? gate(ld(lam, row), logits) : 0.f;
         float kq = 0.f;
         for (int i = tid; i < DK; i += NT) {
             const float qi = ld(q, row * DK + i), ki = ld(k, row * DK + i);
@@ -160,10 +160,10 @@ __global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, const
 
 template <typename IO, int DK>
 cudaError_t launch_multi(int B, int S, int H, int dv, const void* q, const void* k, const void* v, const void* beta,
-                         const void* alpha, const void* lam, float* state, void* o, cudaStream_t stream) {
+                         const void* alpha, const void* lam, float* state, void* o, bool logits, cudaStream_t stream) {
     constexpr int DVS = 64, NT = 128;
     dim3 grid((unsigned)(dv / DVS) * (unsigned)(B * H));
-    k_decode_multi<IO, DK, DVS, NT><<<grid, NT, 0, stream>>>(S, H, dv, (const IO*)q, (const IO*)k, (const IO*)v,
+    k_decode_multi<IO, DK, DVS, NT><<<grid, NT, 0, stream>>>(S, H, dv, logits ? 1 : 0, (const IO*)q, (const IO*)k, (const IO*)v,
                                                              (const IO*)beta, (const IO*)alpha, (const IO*)lam,
                                                              state, (IO*)o);
     return cudaGetLastError();
@@ -195,13 +195,13 @@ cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const 
 
 cudaError_t decode_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
                          const void* beta, const void* alpha, const void* lam, float* state, void* o,
-                         cudaStream_t stream) {
+                         bool logits, cudaStream_t stream) {
     if (dtype == QD_BF16) {
-        if (dk == 128) return launch_multi<__nv_bfloat16, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, stream);
-        return launch_multi<__nv_bfloat16, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, stream);
+        if (dk == 128) return launch_multi<__nv_bfloat16, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, stream);
+        return launch_multi<__nv_bfloat16, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, stream);
     }
-    if (dk == 128) return launch_multi<float, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, stream);
-    return launch_multi<float, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, stream);
+    if (dk == 128) return launch_multi<float, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, stream);
+    return launch_multi<float, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, stream);
 }
 
 }  // namespace qd

@@ -95,6 +95,7 @@ struct ChunkArgs {
     WsLayout L;
     TcLayout TL;
     bool save;       // forward: keep hs and D
+    bool logits;     // beta, alpha, lambda hold pre-activation logits: the kernels apply the sigmoid (QD_COEF_LOGITS)
     bool own_predecessor;   // backward: the kernel enqueued before the reverse chain is this library's forward chain
     cudaStream_t stream;
 };
@@ -117,7 +118,16 @@ cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const 
 
 cudaError_t decode_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
                          const void* beta, const void* alpha, const void* lam, float* state, void* o,
-                         cudaStream_t stream);
+                         bool logits, cudaStream_t stream);
+
+// ---- gates given as logits (QD_COEF_LOGITS) ---------------------------------------------------------
+// The coefficients of the rule are sigmoid gates (Appendix B gives lambda = sigmoid(W h + b); beta and alpha
+// likewise lie in (0,1)).  With the flag the kernels take the pre-activation z and form the gate themselves, in fp32.
+__device__ __forceinline__ float gate(float z, bool logits) { return logits ? 1.f / (1.f + expf(-z)) : z; }
+// log of the forget gate: log(alpha), or log sigmoid(z) = min(z,0) - log1p(exp(-|z|)) without forming 1 - tiny
+__device__ __forceinline__ float log_gate(float z, bool logits) {
+    return logits ? fminf(z, 0.f) - log1pf(expf(-fabsf(z))) : logf(z);
+}
 
 // ---- storage-dtype helpers -------------------------------------------------------------------
 template <typename T> __device__ __forceinline__ float ld(const T* p, size_t i);

@@ -32,6 +32,7 @@ struct Ptrs {
     void *P, *W, *U, *D, *dD;
     float *hs, *dhs, *kdhd, *dhh, *scratch;
     int nslices, save;
+    int logits;                      // beta, alpha, lambda are logits of sigmoid gates
 };
 
 // Register-tiled product: every thread owns TM x TN outputs of an M x N result with inner
@@ -77,14 +78,14 @@ __device__ __forceinline__ void load_coeffs(const Ptrs& p, size_t row0, int live
     const int t = threadIdx.x;
     if (t < C) {
         const size_t r = row0 + (size_t)t * p.H;
-        sbeta[t] = t < live ? ld((const IO*)p.beta, r) : 0.f;
-        slam[t] = (t < live && p.lam) ? ld((const IO*)p.lam, r) : 0.f;
-        salpha[t] = (t < live && p.alpha) ? ld((const IO*)p.alpha, r) : 1.f;
+        sbeta[t] = t < live ? gate(ld((const IO*)p.beta, r), p.logits) : 0.f;
+        slam[t] = (t < live && p.lam) ? gate(ld((const IO*)p.lam, r), p.logits) : 0.f;
+        salpha[t] = (t < live && p.alpha) ? log_gate(ld((const IO*)p.alpha, r), p.logits) : 0.f;     // log alpha
     }
     __syncthreads();
     if (t == 0) {
         float acc = 0.f;
-        for (int r = 0; r < C; ++r) { acc += logf(salpha[r]); sg[r] = acc; }
+        for (int r = 0; r < C; ++r) { acc += salpha[r]; sg[r] = acc; }
     }
     __syncthreads();
 }
@@ -330,9 +331,9 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
         // S0 coefficients
         if (tid < C) {
             const size_t r = row0 + (size_t)tid * H;
-            sbeta[tid] = tid < live ? ld((const IO*)p.beta, r) : 0.f;
-            slam[tid] = (tid < live && p.lam) ? ld((const IO*)p.lam, r) : 0.f;
-            salpha[tid] = (tid < live && p.alpha) ? ld((const IO*)p.alpha, r) : 1.f;
+            sbeta[tid] = tid < live ? gate(ld((const IO*)p.beta, r), p.logits) : 0.f;
+            slam[tid] = (tid < live && p.lam) ? gate(ld((const IO*)p.lam, r), p.logits) : 0.f;
+            salpha[tid] = (tid < live && p.alpha) ? gate(ld((const IO*)p.alpha, r), p.logits) : 1.f;
             sg[tid] = p.g[wrow0 + tid];
         }
         __syncthreads();
@@ -456,9 +457,11 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
         __syncthreads();
         if (tid < live) {
             const size_t r = row0 + (size_t)tid * H;
-            p.dbeta[r] = sdbeta[tid];
-            if (p.dlam) p.dlam[r] = sdlam[tid];
-            if (p.dalpha) p.dalpha[r] = sdg[tid] / salpha[tid];
+            // with logit inputs the gradients are taken w.r.t. the logits: sigmoid' = s (1 - s), (log sigmoid)' = 1 - s
+            const float be = sbeta[tid], la = slam[tid], al = salpha[tid];
+            p.dbeta[r] = p.logits ? sdbeta[tid] * be * (1.f - be) : sdbeta[tid];
+            if (p.dlam) p.dlam[r] = p.logits ? sdlam[tid] * la * (1.f - la) : sdlam[tid];
+            if (p.dalpha) p.dalpha[r] = p.logits ? sdg[tid] * (1.f - al) : sdg[tid] / al;
         }
         __syncthreads();
     }
@@ -476,7 +479,7 @@ Ptrs make_ptrs(const ChunkArgs& a) {
     p.hs = (float*)(a.ws + a.L.hs); p.dhs = (float*)(a.ws + a.L.dhs);
     p.kdhd = (float*)(a.ws + a.L.kdhd); p.dhh = (float*)(a.ws + a.L.dhh);
     p.scratch = (float*)(a.ws + a.L.scratch);
-    p.nslices = a.L.nslices; p.save = a.save ? 1 : 0;
+    p.nslices = a.L.nslices; p.save = a.save ? 1 : 0; p.logits = a.logits ? 1 : 0;
     return p;
 }
 

@@ -294,6 +294,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
 
 // =================================================================================================
 struct ChunkBwdParams {
+    int logits;                // beta, alpha, lambda are logits of sigmoid gates; their gradients are taken w.r.t. the logits
     int T, Tp, H, N, BH, total;   // T tokens per sequence, Tp = 64 N rows per sequence in the workspace; total = BH*N chunks
     const bf16 *beta, *alpha, *lam;
     const float* g;
@@ -452,9 +453,9 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             const int b_ = bh_ / p.H, hh_ = bh_ % p.H;
             const bool live = n_ * C + tid < p.T;             // tokens past the end of the sequence: beta = 0, alpha = 1
             const size_t cr = ((size_t)b_ * p.T + (size_t)n_ * C + tid) * p.H + hh_;
-            cf_beta = live ? __bfloat162float(p.beta[cr]) : 0.f;
-            cf_lam = (live && p.lam) ? __bfloat162float(p.lam[cr]) : 0.f;
-            cf_alpha = (live && p.alpha) ? __bfloat162float(p.alpha[cr]) : 1.f;
+            cf_beta = live ? gate(__bfloat162float(p.beta[cr]), p.logits) : 0.f;
+            cf_lam = (live && p.lam) ? gate(__bfloat162float(p.lam[cr]), p.logits) : 0.f;
+            cf_alpha = (live && p.alpha) ? gate(__bfloat162float(p.alpha[cr]), p.logits) : 1.f;
             cf_g = p.g[(size_t)bh_ * p.Tp + (size_t)n_ * C + tid];
         }
     };
@@ -840,7 +841,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             rPP += srow[0][w4][r]; dbt += srow[1][w4][r] + srow[4][w4][r]; t2 += srow[2][w4][r]; rAA += srow[3][w4][r] + srow[5][w4][r];
         }
         dg_pre = rPP - cPP + t2 + rAA - cAA;
-        if (r < live) p.dbeta[(row0 + r) * p.H + hh] = dbt;
+        // with logit inputs: d/dz of sigmoid(z) is sigmoid(z) (1 - sigmoid(z))
+        if (r < live) p.dbeta[(row0 + r) * p.H + hh] = p.logits ? dbt * sbeta[r] * (1.f - sbeta[r]) : dbt;
     }
     if (next_id < p.total) fetch_coef(next_id);
     wait(&bm_5, ph);
@@ -904,7 +906,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         for (int w4 = 0; w4 < 4; ++w4) { kd += sred[0][w4][r]; dl += sred[1][w4][r]; t1 += sred[2][w4][r]; }
         sdg[r] = t1 + dg_pre - kd;
         skd[r] = kd;                            // summed below into dg of the last token
-        if (want_dl && r < live) p.dlam[(row0 + r) * p.H + hh] = dl;
+        if (want_dl && r < live) p.dlam[(row0 + r) * p.H + hh] = p.logits ? dl * slam[r] * (1.f - slam[r]) : dl;
     }
     csync();
     if (tid < 32 && want_da) {
@@ -926,8 +928,10 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             if (lane + o < 32) sfx += t;
         }
         if (p.dalpha) {
-            if (2 * lane < live) p.dalpha[(row0 + 2 * lane) * p.H + hh] = sfx / salpha[2 * lane];
-            if (2 * lane + 1 < live) p.dalpha[(row0 + 2 * lane + 1) * p.H + hh] = (sfx - a) / salpha[2 * lane + 1];
+            // d log alpha -> d alpha = d log alpha / alpha;  with logit inputs d/dz log sigmoid(z) = 1 - sigmoid(z)
+            const float a0 = salpha[2 * lane], a1 = salpha[2 * lane + 1];
+            if (2 * lane < live) p.dalpha[(row0 + 2 * lane) * p.H + hh] = p.logits ? sfx * (1.f - a0) : sfx / a0;
+            if (2 * lane + 1 < live) p.dalpha[(row0 + 2 * lane + 1) * p.H + hh] = p.logits ? (sfx - a) * (1.f - a1) : (sfx - a) / a1;
         }
     }
     __syncthreads();                     // every read of this chunk's tiles and scratch is done
@@ -993,6 +997,7 @@ cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
     p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
     p.g = (const float*)(a.ws + a.TL.g);
     p.dbeta = a.dbeta; p.dalpha = a.dalpha; p.dlam = a.dlam;
+    p.logits = a.logits ? 1 : 0;
     p.status = (unsigned*)(a.ws + a.TL.status);
     // the instance without lambda / without the forget gate needs the input AND its gradient to be absent
     const bool lam = a.lam || a.dlam, alpha = a.alpha || a.dalpha;

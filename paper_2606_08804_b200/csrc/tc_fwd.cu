@@ -38,6 +38,7 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 
 // =================================================================================================
 struct PrepParams {
+    int logits;                // beta, alpha, lambda are logits of sigmoid gates
     int T, Tp, H, N, BH;       // T tokens per sequence; the workspace holds Tp = 64 N >= T rows per sequence (N even)
     const bf16 *beta, *alpha, *lam;
     float* g;
@@ -109,10 +110,9 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         // a token past the end of the sequence is an exact no-op of the recurrence: beta = 0, alpha = 1 (and q = k = v = 0)
         const bool live = t0 + tid < p.T;
         const size_t crow = ((size_t)b * p.T + t0 + tid) * p.H + hh;
-        sbeta[tid] = live ? __bfloat162float(p.beta[crow]) : 0.f;
-        slam[tid] = (live && p.lam) ? __bfloat162float(p.lam[crow]) : 0.f;
-        const float alpha = (live && p.alpha) ? __bfloat162float(p.alpha[crow]) : 1.f;
-        float g = logf(alpha);
+        sbeta[tid] = live ? gate(__bfloat162float(p.beta[crow]), p.logits) : 0.f;
+        slam[tid] = (live && p.lam) ? gate(__bfloat162float(p.lam[crow]), p.logits) : 0.f;
+        float g = (live && p.alpha) ? log_gate(__bfloat162float(p.alpha[crow]), p.logits) : 0.f;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const float t = __shfl_up_sync(0xffffffffu, g, o);
@@ -679,6 +679,7 @@ cudaError_t tc_prep(const ChunkArgs& a) {
         return cudaErrorInvalidValue;
     PrepParams p{};
     p.T = s.T; p.Tp = Tp; p.H = s.H; p.N = Tp / kChunk; p.BH = s.B * s.H;
+    p.logits = a.logits ? 1 : 0;
     p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
     p.g = (float*)(a.ws + a.TL.g);
     p.Qg = (bf16*)(a.ws + a.TL.Qg); p.P = (bf16*)(a.ws + a.TL.P);

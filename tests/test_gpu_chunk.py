@@ -330,3 +330,42 @@ def test_gradients_of_absent_coefficients_on_request(dtype):
         torch.cuda.synchronize()
         for n in ("dq", "dk", "dv", "dbeta", "dalpha", "dlam", "dh0"):
             gu.check(_label(cfg, " absent coefficients, gradients requested"), n, g[n], ref[n], cfg.dtype, state=(n == "dh0"))
+
+
+@pytest.mark.parametrize("dtype,T", [("bf16", 300), ("f32", 192)])
+def test_gates_from_logits(dtype, T):
+    # QD_COEF_LOGITS: beta, alpha, lambda are pre-activation logits (lambda's centred on the -0.8 bias of Appendix B);
+    # the kernels apply the sigmoid and return gradients with respect to the logits.  Forward, backward (both modes),
+    # and the multi-token decode step.
+    from oracle import recurrence as orc
+    from paper_2606_08804_b200 import binding as qd
+    base = gen.CONFIGS["cfg2"] if dtype == "bf16" else replace(gen.CONFIGS["cfg0"], h0=True, backward=True)
+    cfg = replace(base, B=2, H=3, T=T, seed=101)
+    d = gen.make_chunk_inputs(cfg)
+    r = np.random.default_rng(7)
+    rnd = (lambda x: gen.round_bf16(x.astype(np.float32))) if dtype == "bf16" else (lambda x: x.astype(np.float32))
+    shp = (cfg.B, cfg.T, cfg.H)
+    z = dict(beta=rnd(r.normal(0.0, 1.5, shp)), alpha=rnd(r.normal(3.0, 1.5, shp)), lam=rnd(r.normal(-0.8, 1.0, shp)))
+    d = dict(d, **z)
+    t = gu.dev_inputs(d, cfg.dtype)
+    ro, rh = orc.forward_logits(d["q"], d["k"], d["v"], z["beta"], z["alpha"], z["lam"], d["h0"])
+    ref = orc.backward_logits(d["q"], d["k"], d["v"], z["beta"], z["alpha"], z["lam"], d["h0"], d["dO"], d["dhT"])
+    lab = _label(cfg, " logits")
+    for reuse in (False, True):
+        o, hT, ws = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], save_for_bwd=reuse, logits=True)
+        g = qd.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], t["dO"], t["dhT"],
+                         workspace=ws if reuse else None, reuse_fwd=reuse, logits=True)
+        torch.cuda.synchronize()
+        gu.check(lab, "o", o, ro, cfg.dtype)
+        gu.check(lab, "hT", hT, rh, cfg.dtype, state=True)
+        for n in ("dq", "dk", "dv", "dbeta", "dalpha", "dlam", "dh0"):
+            gu.check(lab, n, g[n], ref[n], cfg.dtype, state=(n == "dh0"))
+    # decode: the first 5 tokens through the multi-token step with logits
+    S = 5
+    c = lambda x: x[:, :S].contiguous()
+    state = t["h0"].clone()
+    od = qd.recurrent_steps(c(t["q"]), c(t["k"]), c(t["v"]), c(t["beta"]), c(t["alpha"]), c(t["lam"]), state, logits=True)
+    torch.cuda.synchronize()
+    ro5, rh5 = orc.forward_logits(d["q"][:, :S], d["k"][:, :S], d["v"][:, :S], z["beta"][:, :S], z["alpha"][:, :S],
+                                  z["lam"][:, :S], d["h0"])
+    assert gu.rel_err(od, ro5) <= gu.TOL[dtype] and gu.rel_err(state, rh5) <= gu.TOL[dtype]

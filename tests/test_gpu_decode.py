@@ -160,5 +160,6 @@ def test_multi_token_step_null_coefficients_and_argument_errors():
     assert gu.rel_err(o, ro) <= 2e-2 and gu.rel_err(state, rh) <= 2e-2
     lib = qd.load()
     fake = 0x1000
-    assert lib.qdelta_recurrent_steps(1, 0, 1, 64, 64, 0, fake, fake, fake, fake, None, None, fake, fake, None) == 1
-    assert lib.qdelta_recurrent_steps(1, 2, 1, 96, 64, 0, fake, fake, fake, fake, None, None, fake, fake, None) == 2
+    assert lib.qdelta_recurrent_steps(1, 0, 1, 64, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 0, None) == 1
+    assert lib.qdelta_recurrent_steps(1, 2, 1, 96, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 0, None) == 2
+    assert lib.qdelta_recurrent_steps(1, 2, 1, 64, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 8, None) == 1

@@ -115,3 +115,38 @@ def test_lambda_zero_gradients_match_gated_delta_rule_fd():
             arr[i] = old - eps; lm = _gdr_loss(q, k, v, beta, alpha, S0, dO, dST)
             arr[i] = old
             assert abs((lp - lm) / (2 * eps) - ga[i]) <= 2e-7 * max(1.0, abs(ga[i])), (gname, i)
+
+
+def test_logit_gates_forward_is_sigmoid_composition_and_gradients_match_finite_differences():
+    # forward_logits / backward_logits: the gates are sigmoid(z); pinned by the values of the sigmoid at known points
+    # and by central finite differences of the whole composite with respect to every logit
+    assert np.allclose(orc.gates_from_logits(np.array([0.0, np.log(3.0), -np.log(3.0), 800.0, -800.0]))[0],
+                       [0.5, 0.75, 0.25, 1.0, 0.0], rtol=0, atol=1e-15)
+    d, up = _rand(21)
+    r = np.random.default_rng(22)
+    z = dict(beta=r.normal(0, 1.5, d["beta"].shape), alpha=r.normal(1.0, 1.0, d["alpha"].shape), lam=r.normal(-0.8, 1.0, d["lam"].shape))
+    sig = lambda x: 1.0 / (1.0 + np.exp(-x))
+    o1, h1 = orc.forward_logits(d["q"], d["k"], d["v"], z["beta"], z["alpha"], z["lam"], d["h0"])
+    o2, h2 = orc.forward(d["q"], d["k"], d["v"], sig(z["beta"]), sig(z["alpha"]), sig(z["lam"]), d["h0"])
+    assert np.allclose(o1, o2, rtol=1e-13, atol=1e-13) and np.allclose(h1, h2, rtol=1e-13, atol=1e-13)
+
+    def loss():
+        o, hT = orc.forward_logits(d["q"], d["k"], d["v"], z["beta"], z["alpha"], z["lam"], d["h0"])
+        return float(np.sum(o * up["dO"]) + np.sum(hT * up["dhT"]))
+    g = orc.backward_logits(d["q"], d["k"], d["v"], z["beta"], z["alpha"], z["lam"], d["h0"], up["dO"], up["dhT"], ckpt=4)
+    eps = 1e-6
+    for name, gname in (("beta", "dbeta"), ("alpha", "dalpha"), ("lam", "dlam")):
+        flat, gflat = z[name].reshape(-1), g[gname].reshape(-1)
+        for i in range(flat.size):
+            old = flat[i]
+            flat[i] = old + eps; lp = loss()
+            flat[i] = old - eps; lm = loss()
+            flat[i] = old
+            fd = (lp - lm) / (2 * eps)
+            assert abs(fd - gflat[i]) <= 1e-6 * max(1.0, abs(fd)), (name, i, fd, gflat[i])
+    # the other gradients are those of the plain call at the same gate values; absent logits stay absent
+    g0 = orc.backward(d["q"], d["k"], d["v"], sig(z["beta"]), sig(z["alpha"]), sig(z["lam"]), d["h0"], up["dO"], up["dhT"], ckpt=4)
+    for n in ("dq", "dk", "dv", "dh0"):
+        assert np.allclose(g[n], g0[n], rtol=1e-12, atol=1e-12)
+    gn = orc.backward_logits(d["q"], d["k"], d["v"], z["beta"], None, None, d["h0"], up["dO"], up["dhT"], ckpt=4)
+    assert gn["dalpha"] is None and gn["dlam"] is None
