@@ -185,7 +185,7 @@ def workload_name(cfg, backward=True):
 class Workload:
     """Device-resident inputs, outputs and workspace of one chunkwise configuration, and its step."""
 
-    def __init__(self, torch, qd, gen, cfg, seed, backward=True, drop=()):
+    def __init__(self, torch, qd, gen, cfg, seed, backward=True, drop=(), fused=False):
         d = gen.make_chunk_inputs(cfg, seed=seed)
         bf = torch.bfloat16
         self.host, self.dev = {}, {}
@@ -202,6 +202,9 @@ class Workload:
         for n in drop:                                  # variant runs: the optional input is absent (NULL)
             self.dev[n] = None
         self.cfg, self.qd, self.backward = cfg, qd, backward
+        # fused=True: the same tensors read as un-normalised q, k and as gate logits (in-kernel L2 normalisation and
+        # sigmoid); the values differ from the plain run, the work per token does not
+        self.kw = dict(logits=True, norm_qk=True) if fused else {}
         B, T, H, dk, dv = cfg.B, cfg.T, cfg.H, cfg.dk, cfg.dv
         self.shape = qd.make_shape(self.dev["q"], self.dev["v"], cfg.chunk)
         self.ws = qd.alloc_workspace(self.shape, backward, "cuda")
@@ -212,10 +215,10 @@ class Workload:
     def step(self):
         d, qd, cfg = self.dev, self.qd, self.cfg
         qd.chunk_fwd(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"], chunk=cfg.chunk,
-                     save_for_bwd=self.backward, workspace=self.ws, o=self.o, hT=self.hT)
+                     save_for_bwd=self.backward, workspace=self.ws, o=self.o, hT=self.hT, **self.kw)
         if self.backward:
             qd.chunk_bwd(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"], d["dO"], d["dhT"],
-                         chunk=cfg.chunk, workspace=self.ws, reuse_fwd=True, out=self.grads)
+                         chunk=cfg.chunk, workspace=self.ws, reuse_fwd=True, out=self.grads, **self.kw)
 
 
 def time_regions(torch, step, steps, regions, barrier):
@@ -231,9 +234,9 @@ def time_regions(torch, step, steps, regions, barrier):
     return [e0.elapsed_time(e1) for e0, e1 in evs]
 
 
-def extra_workload(torch, qd, gen, cfg, pk, pk_kind, backward, steps, regions, drop=()):
+def extra_workload(torch, qd, gen, cfg, pk, pk_kind, backward, steps, regions, drop=(), fused=False):
     """A further configuration timed like the headline one (rank 0, one GPU): ms per step, tokens/s, roofline fraction."""
-    w = Workload(torch, qd, gen, cfg, cfg.seed, backward=backward, drop=drop)
+    w = Workload(torch, qd, gen, cfg, cfg.seed, backward=backward, drop=drop, fused=fused)
     for _ in range(3):
         w.step()
     torch.cuda.synchronize()
@@ -427,6 +430,10 @@ def run_ours(args, cfg):
             r = extra_workload(torch, qd, gen, cfg, pk, pk_kind, True, 20, 3, drop=drop)
             var[name] = {"ms_per_step": r["ms_per_step"], "speedup_vs_full_rule": base / r["ms_per_step"]}
         extras["variants"] = var
+        # pre-processing fused into the kernels: L2 normalisation of q, k and sigmoid gates (with their backward)
+        r = extra_workload(torch, qd, gen, cfg, pk, pk_kind, True, 20, 3, fused=True)
+        extras["fused_preprocessing"] = {"flags": "QD_NORM_QK | QD_COEF_LOGITS", "ms_per_step": r["ms_per_step"],
+                                         "overhead_ms_vs_plain": r["ms_per_step"] - base}
 
     # ---- decode step (separate configuration), in place over a long run of steps ------------------
     decode = bench_decode(args, qd, gen, torch, pk, pk_kind) if (rank == 0 and not args.no_extras) else None
@@ -508,8 +515,34 @@ def bench_decode(args, qd, gen, torch, pk, pk_kind):
         bytesS = nstates * (2 * cfg.dk * cfg.dv * 4 + S * (2 * (2 * cfg.dk + cfg.dv) + 6 + 2 * cfg.dv))
         multi["S=%d" % S] = {"us_per_call": msS * 1e3, "tokens_per_s": cfg.B * S / (msS * 1e-3),
                              "achieved_gbs": bytesS / (msS * 1e-3) / 1e9, "frac": bytesS / (msS * 1e-3) / 1e9 / pk["hbm_gbs"]}
+    # the same loop replayed from one CUDA graph of `pool` steps (no per-step launch cost on the host)
+    graph_us = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(pool):
+                one(i)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(pool):
+                one(i)
+        reps = max(1, nsteps // pool)
+        g.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            g.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        graph_us = e0.elapsed_time(e1) / (reps * pool) * 1e3
+    except Exception as exc:                         # graph capture is a convenience of the harness, not of the library
+        graph_us = "unavailable: %s" % type(exc).__name__
     return {"workload": "cfg4: batch=%d H=%d dk=%d dv=%d fp32 state in place, bf16 tokens" % (cfg.B, cfg.H, cfg.dk, cfg.dv),
             "steps": nsteps, "us_per_step": ms * 1e3, "tokens_per_s": cfg.B / (ms * 1e-3), "multi_token": multi,
+            "us_per_step_cuda_graph": graph_us,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / pk["hbm_gbs"], "peak_kind": "of " + pk_kind,
                          "algorithmic_bytes_per_launch": bytes_step, "state_larger_than_l2": True}}

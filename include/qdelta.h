@@ -66,10 +66,15 @@ enum {
     QD_FWD_SAVE_FOR_BWD = 1,  /* fwd: also keep the per-chunk states etc. in a backward-sized workspace */
     QD_BWD_REUSE_FWD = 2,     /* bwd: the workspace still holds what a QD_FWD_SAVE_FOR_BWD forward of the
                                  SAME inputs (and the same QD_COEF_LOGITS setting) left there; skip the recomputation */
-    QD_COEF_LOGITS = 4        /* fwd, bwd, qdelta_recurrent_steps: beta, alpha and lambda hold the pre-activation
+    QD_COEF_LOGITS = 4,       /* fwd, bwd, qdelta_recurrent_steps: beta, alpha and lambda hold the pre-activation
                                  logits z of sigmoid gates (Appendix B: lambda = sigmoid(W h + b)); the kernels use
                                  sigmoid(z), computed in fp32, and the backward writes dbeta, dalpha, dlambda as
                                  derivatives with respect to the logits.  NULL alpha / lambda still mean 1 / 0. */
+    QD_NORM_QK = 8            /* fwd, bwd, qdelta_recurrent_steps: q and k are given un-normalised; the kernels use
+                                 q / sqrt(|q|^2 + 1e-6) and k / sqrt(|k|^2 + 1e-6), per token and head (the L2
+                                 normalisation that otherwise precedes the call), and the backward writes dq, dk as
+                                 derivatives with respect to the un-normalised q, k.  A QD_BWD_REUSE_FWD backward must
+                                 carry the same setting as its forward. */
 };
 
 typedef struct {
@@ -139,7 +144,7 @@ int qdelta_recurrent_step(int B, int H, int dk, int dv, int dtype,
  * those of the chunkwise calls:
  *     q,k [B,S,H,dk]   v,o [B,S,H,dv]   beta/alpha/lambda [B,S,H]   (alpha, lambda may be NULL)
  *     state [B,H,dk,dv] fp32, UPDATED IN PLACE to the state after the S-th token;  o_s is read out after token s.
- * The result is bit-identical to S calls of qdelta_recurrent_step.  flags: 0 or QD_COEF_LOGITS.  S >= 1; for long runs of tokens (a prompt) use
+ * The result is bit-identical to S calls of qdelta_recurrent_step.  flags: 0, QD_COEF_LOGITS, QD_NORM_QK.  S >= 1; for long runs of tokens (a prompt) use
  * qdelta_chunk_fwd with h0 / hT, which runs on the tensor cores.  Needs no workspace.
  */
 int qdelta_recurrent_steps(int B, int S, int H, int dk, int dv, int dtype,

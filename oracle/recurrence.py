@@ -130,3 +130,43 @@ def backward_logits(q, k, v, zbeta, zalpha, zlam, h0, dO, dhT=None, ckpt=64):
     g["dalpha"] = None if alpha is None else g["dalpha"] * alpha * (1.0 - alpha)
     g["dlam"] = None if lam is None else g["dlam"] * lam * (1.0 - lam)
     return g
+
+
+NORM_EPS = 1e-6
+
+
+def l2_normalize(x):
+    """x / sqrt(|x|^2 + NORM_EPS) along the last axis (per token and head), fp64.  The text gives no formula for the
+    normalisation of q and k; this is the usual L2 normalisation with a small constant under the root."""
+    x = np.asarray(x, np.float64)
+    return x / np.sqrt(np.sum(x * x, axis=-1, keepdims=True) + NORM_EPS)
+
+
+def l2_normalize_backward(x, dxhat):
+    """Gradient through l2_normalize: with r = 1/sqrt(|x|^2 + eps) and x^ = r x,  dx = r (dx^ - x^ <x^, dx^>)."""
+    x = np.asarray(x, np.float64)
+    r = 1.0 / np.sqrt(np.sum(x * x, axis=-1, keepdims=True) + NORM_EPS)
+    xh = r * x
+    return r * (dxhat - xh * np.sum(xh * dxhat, axis=-1, keepdims=True))
+
+
+def forward_fused(q, k, v, beta, alpha=None, lam=None, h0=None, logits=False, norm_qk=False):
+    """forward() behind the optional pre-processing stages: L2 normalisation of q and k, gates from logits."""
+    if norm_qk:
+        q, k = l2_normalize(q), l2_normalize(k)
+    if logits:
+        beta, alpha, lam = gates_from_logits(beta, alpha, lam)
+    return forward(q, k, v, beta, alpha, lam, h0)
+
+
+def backward_fused(q, k, v, beta, alpha, lam, h0, dO, dhT=None, ckpt=64, logits=False, norm_qk=False):
+    """backward() behind the same stages: gradients with respect to what the caller passed in."""
+    qn, kn = (l2_normalize(q), l2_normalize(k)) if norm_qk else (q, k)
+    if logits:
+        g = backward_logits(qn, kn, v, beta, alpha, lam, h0, dO, dhT, ckpt)
+    else:
+        g = backward(qn, kn, v, beta, alpha, lam, h0, dO, dhT, ckpt)
+    if norm_qk:
+        g["dq"] = l2_normalize_backward(q, g["dq"])
+        g["dk"] = l2_normalize_backward(k, g["dk"])
+    return g

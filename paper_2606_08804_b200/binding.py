@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libqdelta.so")
 
 QD_F32, QD_BF16 = 0, 1
-QD_FWD_SAVE_FOR_BWD, QD_BWD_REUSE_FWD, QD_COEF_LOGITS = 1, 2, 4
+QD_FWD_SAVE_FOR_BWD, QD_BWD_REUSE_FWD, QD_COEF_LOGITS, QD_NORM_QK = 1, 2, 4, 8
 
 EXPORTS = ("qdelta_chunk_workspace_bytes", "qdelta_chunk_fwd", "qdelta_chunk_bwd",
            "qdelta_recurrent_step", "qdelta_workspace_status", "qdelta_status_string",
@@ -155,9 +155,10 @@ def workspace_status(workspace: torch.Tensor) -> int:
 
 
 def chunk_fwd(q, k, v, beta, alpha=None, lam=None, h0=None, chunk=64, save_for_bwd=False,
-              workspace=None, o=None, hT=None, want_hT=True, logits=False):
+              workspace=None, o=None, hT=None, want_hT=True, logits=False, norm_qk=False):
     """Chunkwise forward.  Returns (o, hT, workspace).  All tensors live on the GPU.
-    logits=True: beta, alpha, lam hold the logits of sigmoid gates (the kernels apply the sigmoid)."""
+    logits=True: beta, alpha, lam hold the logits of sigmoid gates (the kernels apply the sigmoid).
+    norm_qk=True: q and k are un-normalised, the kernels L2-normalise them per token and head."""
     lib = load()
     s = make_shape(q, v, chunk)
     B, T, H, dk, dv, dt = s.B, s.T, s.H, s.dk, s.dv, q.dtype
@@ -174,7 +175,8 @@ def chunk_fwd(q, k, v, beta, alpha=None, lam=None, h0=None, chunk=64, save_for_b
         _ptr(h0, torch.float32, (B, H, dk, dv), "h0"), _ptr(o, dt, (B, T, H, dv), "o"),
         _ptr(hT, torch.float32, (B, H, dk, dv), "hT"),
         workspace.data_ptr(), workspace.numel(),
-        (QD_FWD_SAVE_FOR_BWD if save_for_bwd else 0) | (QD_COEF_LOGITS if logits else 0), _stream())
+        (QD_FWD_SAVE_FOR_BWD if save_for_bwd else 0) | (QD_COEF_LOGITS if logits else 0) | (QD_NORM_QK if norm_qk else 0),
+        _stream())
     _check(rc, "qdelta_chunk_fwd")
     return o, hT, workspace
 
@@ -206,9 +208,10 @@ def chunk_fwd_static(q, k, v, beta, alpha, lam, h0, o, hT=None, status=None, chu
 
 
 def chunk_bwd(q, k, v, beta, alpha, lam, h0, dO, dhT=None, chunk=64, workspace=None,
-              reuse_fwd=False, out=None, want_dh0=True, logits=False):
+              reuse_fwd=False, out=None, want_dh0=True, logits=False, norm_qk=False):
     """Chunkwise backward.  Returns dict(dq, dk, dv, dbeta, dalpha, dlam, dh0) of GPU tensors.
-    logits=True: beta, alpha, lam are logits and dbeta, dalpha, dlam are gradients with respect to them."""
+    logits=True: beta, alpha, lam are logits and dbeta, dalpha, dlam are gradients with respect to them.
+    norm_qk=True: q, k are un-normalised and dq, dk are gradients with respect to them."""
     lib = load()
     s = make_shape(q, v, chunk)
     B, T, H, dk, dv, dt = s.B, s.T, s.H, s.dk, s.dv, q.dtype
@@ -237,7 +240,8 @@ def chunk_bwd(q, k, v, beta, alpha, lam, h0, dO, dhT=None, chunk=64, workspace=N
         _ptr(g["dalpha"], f32, (B, T, H), "dalpha"), _ptr(g["dlam"], f32, (B, T, H), "dlam"),
         _ptr(g["dh0"], f32, (B, H, dk, dv), "dh0"),
         workspace.data_ptr(), workspace.numel(),
-        (QD_BWD_REUSE_FWD if reuse_fwd else 0) | (QD_COEF_LOGITS if logits else 0), _stream())
+        (QD_BWD_REUSE_FWD if reuse_fwd else 0) | (QD_COEF_LOGITS if logits else 0) | (QD_NORM_QK if norm_qk else 0),
+        _stream())
     _check(rc, "qdelta_chunk_bwd")
     return g
 
@@ -259,7 +263,7 @@ def recurrent_step(q, k, v, beta, alpha, lam, state, o=None):
     return o
 
 
-def recurrent_steps(q, k, v, beta, alpha, lam, state, o=None, logits=False):
+def recurrent_steps(q, k, v, beta, alpha, lam, state, o=None, logits=False, norm_qk=False):
     """S decode tokens per call: q,k [B,S,H,dk], v [B,S,H,dv], coefficients [B,S,H]; `state` [B,H,dk,dv] fp32 is
     updated in place to the state after the last token.  Returns o [B,S,H,dv]."""
     lib = load()
@@ -272,6 +276,6 @@ def recurrent_steps(q, k, v, beta, alpha, lam, state, o=None, logits=False):
         B, S, H, dk, dv, _dtype_code(q), _ptr(q, dt, (B, S, H, dk), "q"), _ptr(k, dt, (B, S, H, dk), "k"),
         _ptr(v, dt, (B, S, H, dv), "v"), _ptr(beta, dt, (B, S, H), "beta"), _ptr(alpha, dt, (B, S, H), "alpha"),
         _ptr(lam, dt, (B, S, H), "lam"), _ptr(state, torch.float32, (B, H, dk, dv), "state"),
-        _ptr(o, dt, (B, S, H, dv), "o"), QD_COEF_LOGITS if logits else 0, _stream())
+        _ptr(o, dt, (B, S, H, dv), "o"), (QD_COEF_LOGITS if logits else 0) | (QD_NORM_QK if norm_qk else 0), _stream())
     _check(rc, "qdelta_recurrent_steps")
     return o

@@ -18,6 +18,7 @@ WsLayout ws_layout(const qd_shape& s) {
     L.P = take(BH * T * kChunk * io);
     L.W = take(BH * T * s.dk * io);
     L.U = take(BH * T * s.dv * io);
+    L.rqk = take(2 * BH * T * 4);
     L.fwd_end = off;
     L.nslices = s.dv / kSliceSimt;
     L.bwd_ctas = 296;
@@ -27,7 +28,7 @@ WsLayout ws_layout(const qd_shape& s) {
     L.dD = take(BH * T * s.dv * io);
     L.kdhd = take((size_t)L.nslices * BH * T * 4);
     L.dhh = take((size_t)L.nslices * BH * N * 4);
-    L.scratch = take((size_t)L.bwd_ctas * 4 * kChunk * s.dk * 4);
+    L.scratch = take((size_t)L.bwd_ctas * 6 * kChunk * s.dk * 4);
     L.bwd_end = off;
     return L;
 }
@@ -116,12 +117,13 @@ int qdelta_chunk_fwd(const qd_shape* shape, const void* q, const void* k, const 
     const void* coef[] = {beta, alpha, lambda};
     for (const void* p : coef)
         if (p && ((uintptr_t)p & (shape->dtype == QD_BF16 ? 1 : 3))) return QD_ERR_INVALID_ARG;
-    if (flags & ~(unsigned)(QD_FWD_SAVE_FOR_BWD | QD_COEF_LOGITS)) return QD_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(QD_FWD_SAVE_FOR_BWD | QD_COEF_LOGITS | QD_NORM_QK)) return QD_ERR_INVALID_ARG;
     ChunkArgs a{};
     a.s = *shape;
     a.L = ws_layout(*shape);
     a.save = (flags & QD_FWD_SAVE_FOR_BWD) != 0;
     a.logits = (flags & QD_COEF_LOGITS) != 0;
+    a.norm = (flags & QD_NORM_QK) != 0;
     if (!workspace || workspace_bytes < qdelta_chunk_workspace_bytes(shape, a.save ? 1 : 0)) return QD_ERR_WORKSPACE;
     a.q = q; a.k = k; a.v = v; a.beta = beta; a.alpha = alpha; a.lam = lambda; a.h0 = h0; a.o = o; a.hT = hT;
     a.ws = (char*)workspace;
@@ -155,12 +157,13 @@ int qdelta_chunk_bwd(const qd_shape* shape, const void* q, const void* k, const 
     const void* gcoef[] = {dbeta, dalpha, dlambda};
     for (const void* p : gcoef)
         if (p && ((uintptr_t)p & 3)) return QD_ERR_INVALID_ARG;
-    if (flags & ~(unsigned)(QD_BWD_REUSE_FWD | QD_COEF_LOGITS)) return QD_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(QD_BWD_REUSE_FWD | QD_COEF_LOGITS | QD_NORM_QK)) return QD_ERR_INVALID_ARG;
     ChunkArgs a{};
     a.s = *shape;
     a.L = ws_layout(*shape);
     a.save = true;
     a.logits = (flags & QD_COEF_LOGITS) != 0;
+    a.norm = (flags & QD_NORM_QK) != 0;
     if (!workspace || workspace_bytes < qdelta_chunk_workspace_bytes(shape, 1)) return QD_ERR_WORKSPACE;
     a.q = q; a.k = k; a.v = v; a.beta = beta; a.alpha = alpha; a.lam = lambda; a.h0 = h0;
     a.dO = dO; a.dhT = dhT; a.dq = dq; a.dk = dk; a.dv = dv;
@@ -222,7 +225,7 @@ int qdelta_recurrent_steps(int B, int S, int H, int dk, int dv, int dtype, const
                            const void* beta, const void* alpha, const void* lambda, float* state, void* o,
                            unsigned flags, qd_stream stream) {
     if (B <= 0 || H <= 0 || S <= 0) return QD_ERR_INVALID_ARG;
-    if (flags & ~(unsigned)QD_COEF_LOGITS) return QD_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(QD_COEF_LOGITS | QD_NORM_QK)) return QD_ERR_INVALID_ARG;
     if (dtype != QD_F32 && dtype != QD_BF16) return QD_ERR_UNSUPPORTED;
     if ((dk != 64 && dk != 128) || (dv != 64 && dv != 128)) return QD_ERR_UNSUPPORTED;
     if (!q || !k || !v || !beta || !state || !o) return QD_ERR_INVALID_ARG;
@@ -235,7 +238,7 @@ int qdelta_recurrent_steps(int B, int S, int H, int dk, int dv, int dtype, const
         if (p && ((uintptr_t)p & (dtype == QD_BF16 ? 1 : 3))) return QD_ERR_INVALID_ARG;
     if (timed(ST_DECODE, (cudaStream_t)stream, [&] {
             return decode_steps(B, S, H, dk, dv, dtype, q, k, v, beta, alpha, lambda, state, o,
-                                (flags & QD_COEF_LOGITS) != 0, (cudaStream_t)stream);
+                                (flags & QD_COEF_LOGITS) != 0, (flags & QD_NORM_QK) != 0, (cudaStream_t)stream);
         }) != cudaSuccess)
         return QD_ERR_CUDA;
     return QD_OK;

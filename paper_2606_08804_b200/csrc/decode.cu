@@ -86,7 +86,7 @@ __global__ void __launch_bounds__(NT) k_decode(int dv, const IO* __restrict__ q,
 // arithmetic of one token is exactly that of k_decode, in the same order, so S tokens here give bit-identical results to
 // S single-token calls.
 template <typename IO, int DK, int DVS, int NT>
-__global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, int logits, const IO* __restrict__ q, const IO* __restrict__ k,
+__global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, int logits, int norm, const IO* __restrict__ q, const IO* __restrict__ k,
                                                      const IO* __restrict__ v, const IO* __restrict__ beta,
                                                      const IO* __restrict__ alpha, const IO* __restrict__ lam,
                                                      float* __restrict__ state, IO* __restrict__ o) {
@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, int l
     __shared__ float sx[DK], sq[DK], sk[DK];
     __shared__ float redx[RP][DVS], redq[RP][DVS];
     __shared__ float sdelta[DVS];
-    __shared__ float skq[NT / 32];
+    __shared__ float skq[NT / 32], snq[NT / 32], snk[NT / 32];
     const int nsl = dv / DVS, bh = blockIdx.x / nsl, j0 = (blockIdx.x % nsl) * DVS, tid = threadIdx.x;
     const int b = bh / H, hh = bh % H;
     const int c4 = tid % C4, rg = tid / C4;
@@ -112,14 +112,42 @@ __global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, int l
         const float al = alpha ? gate(ld(alpha, row), logits) : 1.f;
         const float la = lam ? gate(ld(lam, row), logits) : 0.f;
         float kq = 0.f;
-        for (int i = tid; i < DK; i += NT) {
-            const float qi = ld(q, row * DK + i), ki = ld(k, row * DK + i);
-            sq[i] = qi; sk[i] = ki; sx[i] = fmaf(la, qi, ki);
-            kq = fmaf(ki, qi, kq);
-        }
+        if (norm) {
+            // q^ = q / sqrt(|q|^2 + eps), k^ likewise: three block-wide sums, then the token's arrays are rescaled
+            float ssq = 0.f, ssk = 0.f;
+            for (int i = tid; i < DK; i += NT) {
+                const float qi = ld(q, row * DK + i), ki = ld(k, row * DK + i);
+                sq[i] = qi; sk[i] = ki;
+                ssq = fmaf(qi, qi, ssq); ssk = fmaf(ki, ki, ssk); kq = fmaf(ki, qi, kq);
+            }
 #pragma unroll
-        for (int w = 16; w > 0; w >>= 1) kq += __shfl_xor_sync(0xffffffffu, kq, w);
-        if ((tid & 31) == 0) skq[tid >> 5] = kq;
+            for (int w = 16; w > 0; w >>= 1) {
+                kq += __shfl_xor_sync(0xffffffffu, kq, w);
+                ssq += __shfl_xor_sync(0xffffffffu, ssq, w);
+                ssk += __shfl_xor_sync(0xffffffffu, ssk, w);
+            }
+            if ((tid & 31) == 0) { skq[tid >> 5] = kq; snq[tid >> 5] = ssq; snk[tid >> 5] = ssk; }
+            __syncthreads();
+            float tq = 0.f, tk = 0.f, tkq = 0.f;
+#pragma unroll
+            for (int w = 0; w < NT / 32; ++w) { tq += snq[w]; tk += snk[w]; tkq += skq[w]; }
+            const float rq = 1.f / sqrtf(tq + kNormEps), rk = 1.f / sqrtf(tk + kNormEps);
+            __syncthreads();
+            for (int i = tid; i < DK; i += NT) {
+                const float qi = sq[i] * rq, ki = sk[i] * rk;
+                sq[i] = qi; sk[i] = ki; sx[i] = fmaf(la, qi, ki);
+            }
+            if (tid == 0) { skq[0] = tkq * rq * rk; for (int w = 1; w < NT / 32; ++w) skq[w] = 0.f; }
+        } else {
+            for (int i = tid; i < DK; i += NT) {
+                const float qi = ld(q, row * DK + i), ki = ld(k, row * DK + i);
+                sq[i] = qi; sk[i] = ki; sx[i] = fmaf(la, qi, ki);
+                kq = fmaf(ki, qi, kq);
+            }
+#pragma unroll
+            for (int w = 16; w > 0; w >>= 1) kq += __shfl_xor_sync(0xffffffffu, kq, w);
+            if ((tid & 31) == 0) skq[tid >> 5] = kq;
+        }
         __syncthreads();
 
         float4 ax = make_float4(0.f, 0.f, 0.f, 0.f), aq = ax;
@@ -160,10 +188,11 @@ __global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, int l
 
 template <typename IO, int DK>
 cudaError_t launch_multi(int B, int S, int H, int dv, const void* q, const void* k, const void* v, const void* beta,
-                         const void* alpha, const void* lam, float* state, void* o, bool logits, cudaStream_t stream) {
+                         const void* alpha, const void* lam, float* state, void* o, bool logits, bool norm,
+                         cudaStream_t stream) {
     constexpr int DVS = 64, NT = 128;
     dim3 grid((unsigned)(dv / DVS) * (unsigned)(B * H));
-    k_decode_multi<IO, DK, DVS, NT><<<grid, NT, 0, stream>>>(S, H, dv, logits ? 1 : 0, (const IO*)q, (const IO*)k, (const IO*)v,
+    k_decode_multi<IO, DK, DVS, NT><<<grid, NT, 0, stream>>>(S, H, dv, logits ? 1 : 0, norm ? 1 : 0, (const IO*)q, (const IO*)k, (const IO*)v,
                                                              (const IO*)beta, (const IO*)alpha, (const IO*)lam,
                                                              state, (IO*)o);
     return cudaGetLastError();
@@ -195,13 +224,13 @@ cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const 
 
 cudaError_t decode_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
                          const void* beta, const void* alpha, const void* lam, float* state, void* o,
-                         bool logits, cudaStream_t stream) {
+                         bool logits, bool norm, cudaStream_t stream) {
     if (dtype == QD_BF16) {
-        if (dk == 128) return launch_multi<__nv_bfloat16, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, stream);
-        return launch_multi<__nv_bfloat16, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, stream);
+        if (dk == 128) return launch_multi<__nv_bfloat16, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, stream);
+        return launch_multi<__nv_bfloat16, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, stream);
     }
-    if (dk == 128) return launch_multi<float, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, stream);
-    return launch_multi<float, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, stream);
+    if (dk == 128) return launch_multi<float, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, stream);
+    return launch_multi<float, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, stream);
 }
 
 }  // namespace qd

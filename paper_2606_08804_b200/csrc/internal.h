@@ -29,6 +29,7 @@ struct WsLayout {
     size_t kdhd;     // fp32 [S][BH*T]     per d_v-slice partial of <(K-> dh)_r, Delta_r>
     size_t dhh;      // fp32 [S][BH*N]     per d_v-slice partial of <dh, h>_F
     size_t scratch;  // fp32 per-CTA scratch of the SIMT chunk backward
+    size_t rqk;      // fp32 [2][BH*T]     QD_NORM_QK: 1/|q_t|, then 1/|k_t|
     size_t bwd_end;
     int nslices;
     int bwd_ctas;
@@ -46,6 +47,7 @@ struct TcLayout {
     size_t P;        // bf16 [BH*T][C]         Gamma o (Q K^T), causal incl. diagonal
     size_t Wt;       // bf16 [BH*N][dk][C]     (T diag(gamma) X)^T per chunk
     size_t Ut;       // bf16 [BH*N][dv][C]     (T V)^T per chunk
+    size_t rqk;      // fp32 [2][BH*T]         QD_NORM_QK: 1/|q_t|, then 1/|k_t|
     size_t fwd_end;
     // kept for / produced by the backward
     size_t Mt;       // bf16 [BH*N][C][C]      ((I+A)^-1)^T per chunk: [column][row]
@@ -96,6 +98,7 @@ struct ChunkArgs {
     TcLayout TL;
     bool save;       // forward: keep hs and D
     bool logits;     // beta, alpha, lambda hold pre-activation logits: the kernels apply the sigmoid (QD_COEF_LOGITS)
+    bool norm;       // q and k are L2-normalised per token and head inside the kernels (QD_NORM_QK)
     bool own_predecessor;   // backward: the kernel enqueued before the reverse chain is this library's forward chain
     cudaStream_t stream;
 };
@@ -118,7 +121,11 @@ cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const 
 
 cudaError_t decode_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
                          const void* beta, const void* alpha, const void* lam, float* state, void* o,
-                         bool logits, cudaStream_t stream);
+                         bool logits, bool norm, cudaStream_t stream);
+
+// ---- in-kernel L2 normalisation of q and k (QD_NORM_QK) ------------------------------------------------
+// x^ = x / sqrt(sum x^2 + kNormEps), per token and head.  Its backward: dx = r (dx^ - x^ <x^, dx^>), r = 1/sqrt(sum x^2 + eps).
+constexpr float kNormEps = 1e-6f;
 
 // ---- gates given as logits (QD_COEF_LOGITS) ---------------------------------------------------------
 // The coefficients of the rule are sigmoid gates (Appendix B gives lambda = sigmoid(W h + b); beta and alpha

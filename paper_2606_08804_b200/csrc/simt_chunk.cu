@@ -33,6 +33,7 @@ struct Ptrs {
     float *hs, *dhs, *kdhd, *dhh, *scratch;
     int nslices, save;
     int logits;                      // beta, alpha, lambda are logits of sigmoid gates
+    float* rqk;                      // non-null (QD_NORM_QK): q and k are L2-normalised in here; [0, BH*Tp) 1/|q_t|, then 1/|k_t|
 };
 
 // Register-tiled product: every thread owns TM x TN outputs of an M x N result with inner
@@ -69,6 +70,38 @@ __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
     return x;
+}
+
+// 1/|q_r| and 1/|k_r| of one chunk into shared memory: computed from the rows (and kept in the workspace) by the
+// preparation kernel, read back from the workspace by the others.  Without normalisation both are 1.
+template <typename IO, bool COMPUTE>
+__device__ __forceinline__ void load_norms(const Ptrs& p, size_t row0, size_t wrow0, int live, float* srq, float* srk) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (!p.rqk) {
+        if (threadIdx.x < C) { srq[threadIdx.x] = 1.f; srk[threadIdx.x] = 1.f; }
+    } else if (COMPUTE) {
+        const size_t nrows = (size_t)p.B * p.H * p.Tp;
+        for (int r = warp; r < C; r += NT / 32) {
+            float sq = 0.f, sk = 0.f;
+            if (r < live)
+                for (int d = lane; d < p.dk; d += 32) {
+                    const float qv = ld((const IO*)p.q, (row0 + (size_t)r * p.H) * p.dk + d);
+                    const float kv = ld((const IO*)p.k, (row0 + (size_t)r * p.H) * p.dk + d);
+                    sq = fmaf(qv, qv, sq); sk = fmaf(kv, kv, sk);
+                }
+            sq = warp_sum(sq); sk = warp_sum(sk);
+            if (lane == 0) {
+                const float rq = 1.f / sqrtf(sq + kNormEps), rk = 1.f / sqrtf(sk + kNormEps);
+                srq[r] = rq; srk[r] = rk;
+                p.rqk[wrow0 + r] = rq; p.rqk[nrows + wrow0 + r] = rk;
+            }
+        }
+    } else if (threadIdx.x < C) {
+        const size_t nrows = (size_t)p.B * p.H * p.Tp;
+        srq[threadIdx.x] = p.rqk[wrow0 + threadIdx.x];
+        srk[threadIdx.x] = p.rqk[nrows + wrow0 + threadIdx.x];
+    }
+    __syncthreads();
 }
 
 // Coefficients of one chunk into shared memory: beta, lambda, alpha, g (cumulative log alpha).
@@ -110,7 +143,7 @@ __device__ __forceinline__ void invert_unit_lower(const float* sA, float* sM) {
 template <typename IO>
 __global__ void __launch_bounds__(NT) k_prep(Ptrs p) {
     __shared__ float sA[C * LD], sM[C * LD];
-    __shared__ float sbeta[C], slam[C], salpha[C], sg[C];
+    __shared__ float sbeta[C], slam[C], salpha[C], sg[C], srq[C], srk[C];
     const int ch = blockIdx.x, n = ch % p.N, bh = ch / p.N, b = bh / p.H, hh = bh % p.H;
     const int dk = p.dk, dv = p.dv, H = p.H;
     const size_t row0 = ((size_t)b * p.T + (size_t)n * C) * H + hh;   // token row of local r: row0 + r*H
@@ -119,9 +152,10 @@ __global__ void __launch_bounds__(NT) k_prep(Ptrs p) {
     const IO *q = (const IO*)p.q, *k = (const IO*)p.k, *v = (const IO*)p.v;
     load_coeffs<IO>(p, row0, live, sbeta, slam, salpha, sg);
     if (threadIdx.x < C) p.g[wrow0 + threadIdx.x] = sg[threadIdx.x];
+    load_norms<IO, true>(p, row0, wrow0, live, srq, srk);
 
-    auto Qf = [&](int r, int d) { return r < live ? ld(q, (row0 + (size_t)r * H) * dk + d) : 0.f; };
-    auto Kf = [&](int r, int d) { return r < live ? ld(k, (row0 + (size_t)r * H) * dk + d) : 0.f; };
+    auto Qf = [&](int r, int d) { return r < live ? srq[r] * ld(q, (row0 + (size_t)r * H) * dk + d) : 0.f; };
+    auto Kf = [&](int r, int d) { return r < live ? srk[r] * ld(k, (row0 + (size_t)r * H) * dk + d) : 0.f; };
     auto Xf = [&](int r, int d) { return fmaf(slam[r], Qf(r, d), Kf(r, d)); };
     // A = strictLower(beta_r Gamma_ri (x_r . k_i))
     mm<4, 4>(C, C, dk, Xf, [&](int d, int i) { return Kf(i, d); },
@@ -154,6 +188,7 @@ __global__ void __launch_bounds__(NT) k_chain_fwd(Ptrs p) {
     float* sD = sh + dk * DS;       // [C][DS]   Delta slice
     float* sO = sD + C * DS;        // [C][DS]
     float* sg = sO + C * DS;        // [C]
+    float *srq = sg + C, *srk = srq + C;
     const int nsl = dv / DS, j0 = (blockIdx.x % nsl) * DS, bh = blockIdx.x / nsl, b = bh / H, hh = bh % H;
     const IO *q = (const IO*)p.q, *k = (const IO*)p.k;
     for (int e = threadIdx.x; e < dk * DS; e += NT) {
@@ -165,7 +200,7 @@ __global__ void __launch_bounds__(NT) k_chain_fwd(Ptrs p) {
         const size_t wrow0 = (size_t)bh * p.Tp + (size_t)n * C;
         const int live = min(C, p.T - n * C);
         if (threadIdx.x < C) sg[threadIdx.x] = p.g[wrow0 + threadIdx.x];
-        __syncthreads();
+        load_norms<IO, false>(p, row0, wrow0, live, srq, srk);
         if (p.save) {
             float* dst = p.hs + ((size_t)bh * p.N + n) * dk * dv;
             for (int e = threadIdx.x; e < dk * DS; e += NT) dst[(size_t)(e / DS) * dv + j0 + e % DS] = sh[e];
@@ -179,7 +214,7 @@ __global__ void __launch_bounds__(NT) k_chain_fwd(Ptrs p) {
                      if (p.save) st((IO*)p.D, (wrow0 + r) * dv + j0 + j, d);
                  });
         // inter-chunk part of the output: diag(gamma) Q h
-        mm<2, 4>(C, DS, dk, [&](int r, int i) { return r < live ? ld(q, (row0 + (size_t)r * H) * dk + i) : 0.f; }, hf,
+        mm<2, 4>(C, DS, dk, [&](int r, int i) { return r < live ? srq[r] * ld(q, (row0 + (size_t)r * H) * dk + i) : 0.f; }, hf,
                  [&](int r, int j, float acc) { sO[r * DS + j] = expf(sg[r]) * acc; });
         __syncthreads();
         // intra-chunk part: P Delta
@@ -191,7 +226,7 @@ __global__ void __launch_bounds__(NT) k_chain_fwd(Ptrs p) {
         // h <- gamma_C h + K->^T Delta
         const float gC = sg[C - 1];
         mm<4, 4>(dk, DS, C,
-                 [&](int i, int r) { return r < live ? ld(k, (row0 + (size_t)r * H) * dk + i) * expf(gC - sg[r]) : 0.f; },
+                 [&](int i, int r) { return r < live ? srk[r] * ld(k, (row0 + (size_t)r * H) * dk + i) * expf(gC - sg[r]) : 0.f; },
                  [&](int r, int j) { return sD[r * DS + j]; },
                  [&](int i, int j, float acc) { sh[i * DS + j] = fmaf(expf(gC), sh[i * DS + j], acc); });
         __syncthreads();
@@ -214,6 +249,7 @@ __global__ void __launch_bounds__(NT) k_chain_bwd(Ptrs p) {
     float* sdD = sdh + dk * DS;      // [C][DS]
     float* sKD = sdD + C * DS;       // [C][DS]  (K-> dh) o Delta
     float* sg = sKD + C * DS;        // [C]
+    float *srq = sg + C, *srk = srq + C;
     const int nsl = dv / DS, sl = blockIdx.x % nsl, j0 = sl * DS, bh = blockIdx.x / nsl, b = bh / H, hh = bh % H;
     const IO *q = (const IO*)p.q, *k = (const IO*)p.k, *dO = (const IO*)p.dO;
     const size_t BHT = (size_t)p.B * H * p.Tp, BHN = (size_t)p.B * H * p.N;
@@ -224,7 +260,7 @@ __global__ void __launch_bounds__(NT) k_chain_bwd(Ptrs p) {
         const size_t wrow0 = (size_t)bh * p.Tp + (size_t)n * C;
         const int live = min(C, p.T - n * C);
         if (threadIdx.x < C) sg[threadIdx.x] = p.g[wrow0 + threadIdx.x];
-        __syncthreads();
+        load_norms<IO, false>(p, row0, wrow0, live, srq, srk);
         // keep dh of this chunk's exit state; partial <dh, h_entry>_F over this slice
         {
             float* dst = p.dhs + ((size_t)bh * p.N + n) * dk * dv;
@@ -247,7 +283,7 @@ __global__ void __launch_bounds__(NT) k_chain_bwd(Ptrs p) {
         const float gC = sg[C - 1];
         // K-> dh
         mm<2, 4>(C, DS, dk,
-                 [&](int s, int i) { return s < live ? ld(k, (row0 + (size_t)s * H) * dk + i) * expf(gC - sg[s]) : 0.f; },
+                 [&](int s, int i) { return s < live ? srk[s] * ld(k, (row0 + (size_t)s * H) * dk + i) * expf(gC - sg[s]) : 0.f; },
                  [&](int i, int j) { return sdh[i * DS + j]; },
                  [&](int s, int j, float acc) {
                      sdD[s * DS + j] = acc;
@@ -271,7 +307,7 @@ __global__ void __launch_bounds__(NT) k_chain_bwd(Ptrs p) {
         // dh_in = gamma_C dh + (diag(gamma) Q)^T dO - W<-^T dDelta    (one product over 2C terms)
         mm<4, 4>(dk, DS, 2 * C,
                  [&](int i, int kk) {
-                     return kk < C ? (kk < live ? ld(q, (row0 + (size_t)kk * H) * dk + i) * expf(sg[kk]) : 0.f)
+                     return kk < C ? (kk < live ? srq[kk] * ld(q, (row0 + (size_t)kk * H) * dk + i) * expf(sg[kk]) : 0.f)
                                    : -ld((const IO*)p.W, (wrow0 + kk - C) * dk + i);
                  },
                  [&](int kk, int j) {
@@ -306,10 +342,12 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
     float* st2 = st1 + C;            // rowsum(dXg o gamma X)
     float* sdlam = st2 + C;
     float* sdg = sdlam + C;
+    float *srq = sdg + C, *srk = srq + C;
     const int dk = p.dk, dv = p.dv, H = p.H;
     const IO *q = (const IO*)p.q, *k = (const IO*)p.k, *v = (const IO*)p.v, *dO = (const IO*)p.dO;
-    float* sc = p.scratch + (size_t)blockIdx.x * 4 * C * dk;
+    float* sc = p.scratch + (size_t)blockIdx.x * 6 * C * dk;
     float *dW = sc, *dXg = sc + C * dk, *dX = sc + 2 * C * dk, *dQ1 = sc + 3 * C * dk;
+    float *dKh = sc + 4 * C * dk, *dQh = sc + 5 * C * dk;      // QD_NORM_QK: gradients w.r.t. the normalised rows
     const size_t BHT = (size_t)p.B * H * p.Tp, BHN = (size_t)p.B * H * p.N;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -320,8 +358,8 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
         const int live = min(C, p.T - n * C);
         const float* hs = p.hs + ((size_t)bh * p.N + n) * dk * dv;
         const float* dhs = p.dhs + ((size_t)bh * p.N + n) * dk * dv;
-        auto Qf = [&](int r, int d) { return r < live ? ld(q, (row0 + (size_t)r * H) * dk + d) : 0.f; };
-        auto Kf = [&](int r, int d) { return r < live ? ld(k, (row0 + (size_t)r * H) * dk + d) : 0.f; };
+        auto Qf = [&](int r, int d) { return r < live ? srq[r] * ld(q, (row0 + (size_t)r * H) * dk + d) : 0.f; };
+        auto Kf = [&](int r, int d) { return r < live ? srk[r] * ld(k, (row0 + (size_t)r * H) * dk + d) : 0.f; };
         auto Vf = [&](int r, int j) { return r < live ? ld(v, (row0 + (size_t)r * H) * dv + j) : 0.f; };
         auto dOf = [&](int r, int j) { return r < live ? ld(dO, (row0 + (size_t)r * H) * dv + j) : 0.f; };
         auto Xf = [&](int r, int d) { return fmaf(slam[r], Qf(r, d), Kf(r, d)); };
@@ -336,7 +374,7 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
             salpha[tid] = (tid < live && p.alpha) ? gate(ld((const IO*)p.alpha, r), p.logits) : 1.f;
             sg[tid] = p.g[wrow0 + tid];
         }
-        __syncthreads();
+        load_norms<IO, false>(p, row0, wrow0, live, srq, srk);
         if (tid < C) { sgam[tid] = expf(sg[tid]); segc[tid] = expf(sg[C - 1] - sg[tid]); }
         // S1 Gram X K^T, and A
         mm<4, 4>(C, C, dk, Xf, [&](int d, int i) { return Kf(i, d); },
@@ -419,12 +457,14 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
                      return kk < C ? Xf(kk, d) : (kk < 2 * C ? Qf(kk - C, d) : dhs[(size_t)d * dv + kk - 2 * C]);
                  },
                  [&](int i, int d, float acc) {
-                     if (i < live) st((IO*)p.dk_, (row0 + (size_t)i * H) * dk + d, acc + dX[i * dk + d]);
+                     if (p.rqk) dKh[i * dk + d] = acc + dX[i * dk + d];
+                     else if (i < live) st((IO*)p.dk_, (row0 + (size_t)i * H) * dk + d, acc + dX[i * dk + d]);
                  });
         mm<4, 4>(C, dk, C, [&](int r, int s) { return m3[r * LD + s]; }, Kf,
                  [&](int r, int d, float acc) {
-                     if (r < live)
-                         st((IO*)p.dq, (row0 + (size_t)r * H) * dk + d, acc + dQ1[r * dk + d] + slam[r] * dX[r * dk + d]);
+                     const float val = acc + dQ1[r * dk + d] + slam[r] * dX[r * dk + d];
+                     if (p.rqk) dQh[r * dk + d] = val;
+                     else if (r < live) st((IO*)p.dq, (row0 + (size_t)r * H) * dk + d, val);
                  });
         for (int r = warp; r < C; r += NT / 32) {
             float a1 = 0.f, a2 = 0.f, a3 = 0.f;
@@ -438,6 +478,21 @@ __global__ void __launch_bounds__(NT) k_chunk_bwd(Ptrs p, int nchunks) {
             if (lane == 0) { st1[r] = a1; st2[r] = a2; sdlam[r] = a3; }
         }
         __syncthreads();
+        if (p.rqk) {
+            // through the normalisation: dx = r (dx^ - x^ <x^, dx^>), one warp per row
+            for (int r = warp; r < live; r += NT / 32) {
+                float cq = 0.f, ck = 0.f;
+                for (int d = lane; d < dk; d += 32) {
+                    cq = fmaf(dQh[r * dk + d], Qf(r, d), cq);
+                    ck = fmaf(dKh[r * dk + d], Kf(r, d), ck);
+                }
+                cq = warp_sum(cq); ck = warp_sum(ck);
+                for (int d = lane; d < dk; d += 32) {
+                    st((IO*)p.dq, (row0 + (size_t)r * H) * dk + d, srq[r] * (dQh[r * dk + d] - Qf(r, d) * cq));
+                    st((IO*)p.dk_, (row0 + (size_t)r * H) * dk + d, srk[r] * (dKh[r * dk + d] - Kf(r, d) * ck));
+                }
+            }
+        }
         // S11 decay gradient: dg, reverse in-chunk cumulative sum, d alpha = d log alpha / alpha
         if (tid < C) {
             float kd = 0.f;
@@ -480,6 +535,7 @@ Ptrs make_ptrs(const ChunkArgs& a) {
     p.kdhd = (float*)(a.ws + a.L.kdhd); p.dhh = (float*)(a.ws + a.L.dhh);
     p.scratch = (float*)(a.ws + a.L.scratch);
     p.nslices = a.L.nslices; p.save = a.save ? 1 : 0; p.logits = a.logits ? 1 : 0;
+    p.rqk = a.norm ? (float*)(a.ws + a.L.rqk) : nullptr;
     return p;
 }
 
@@ -498,7 +554,7 @@ cudaError_t simt_prep(const ChunkArgs& a) {
 
 cudaError_t simt_chain_fwd(const ChunkArgs& a) {
     Ptrs p = make_ptrs(a);
-    const size_t smem = sizeof(float) * ((size_t)a.s.dk * DS + 2 * C * DS + C);
+    const size_t smem = sizeof(float) * ((size_t)a.s.dk * DS + 2 * C * DS + 3 * C);
     dim3 grid((unsigned)(a.s.dv / DS) * (unsigned)(a.s.B * a.s.H));
     cudaError_t e;
     if (a.s.dtype == QD_BF16) {
@@ -513,7 +569,7 @@ cudaError_t simt_chain_fwd(const ChunkArgs& a) {
 
 cudaError_t simt_chain_bwd(const ChunkArgs& a) {
     Ptrs p = make_ptrs(a);
-    const size_t smem = sizeof(float) * ((size_t)a.s.dk * DS + 2 * C * DS + C);
+    const size_t smem = sizeof(float) * ((size_t)a.s.dk * DS + 2 * C * DS + 3 * C);
     dim3 grid((unsigned)(a.s.dv / DS) * (unsigned)(a.s.B * a.s.H));
     cudaError_t e;
     if (a.s.dtype == QD_BF16) {
@@ -530,7 +586,7 @@ cudaError_t simt_chunk_bwd(const ChunkArgs& a) {
     Ptrs p = make_ptrs(a);
     const int nchunks = a.s.B * a.s.H * p.N;
     const int grid = nchunks < a.L.bwd_ctas ? nchunks : a.L.bwd_ctas;
-    const size_t smem = sizeof(float) * (5 * C * LD + 11 * C);
+    const size_t smem = sizeof(float) * (5 * C * LD + 13 * C);
     cudaError_t e;
     if (a.s.dtype == QD_BF16) {
         if ((e = set_smem(k_chunk_bwd<__nv_bfloat16>, smem)) != cudaSuccess) return e;

@@ -14,6 +14,8 @@
 #include "internal.h"
 #include "sm100.cuh"
 
+#include <type_traits>
+
 namespace qd {
 namespace {
 using namespace sm100;
@@ -51,6 +53,7 @@ __device__ __forceinline__ void fold(float* v, int lane, int off) {
 struct ChainBwdParams {
     int Tp, H, N;              // Tp = 64 N rows per sequence in the workspace
     int dhT_early;             // the kernel before this one in the stream is the library's own: dhT is older than it
+    const float* rk;           // non-null (QD_NORM_QK): 1/|k_t| per workspace row, folded into the per-token scale
     const float* g;
     const float* dhT;
     float* dh0;
@@ -249,15 +252,18 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
         const int ln = tid & 31;
         const float* gl = gseq + (size_t)(p.N - 1) * C;               // cumulative log-decays of the last chunk
         float g0 = gl[ln], g1 = gl[32 + ln], gc = gl[C - 1];
+        const float* rkseq = p.rk ? p.rk + (size_t)bh * p.Tp : nullptr;
+        float r0 = rkseq ? rkseq[(size_t)(p.N - 1) * C + ln] : 1.f, r1 = rkseq ? rkseq[(size_t)(p.N - 1) * C + 32 + ln] : 1.f;
         for (int it = 0; it < p.N; ++it) {
             const int n = p.N - 1 - it;
-            sG[it & 1][ln] = __expf(gc - g0);
-            sG[it & 1][32 + ln] = __expf(gc - g1);
+            sG[it & 1][ln] = __expf(gc - g0) * r0;
+            sG[it & 1][32 + ln] = __expf(gc - g1) * r1;
             if (ln == 0) sG[it & 1][64] = __expf(gc);
             __syncwarp();
             if (n > 0) {                                      // in flight while this chunk is processed
                 const float* gn = gseq + (size_t)(n - 1) * C;
                 g0 = gn[ln]; g1 = gn[32 + ln]; gc = gn[C - 1];
+                if (rkseq) { r0 = rkseq[(size_t)(n - 1) * C + ln]; r1 = rkseq[(size_t)(n - 1) * C + 32 + ln]; }
             }
             if (lead) {
                 tma_store_wait_read_n<0>();               // dDelta^T tile of the previous chunk has been read
@@ -295,6 +301,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
 // =================================================================================================
 struct ChunkBwdParams {
     int logits;                // beta, alpha, lambda are logits of sigmoid gates; their gradients are taken w.r.t. the logits
+    const float* rqk;          // QD_NORM_QK: 1/|q_t| per workspace row, then (BH*Tp further) 1/|k_t|
     int T, Tp, H, N, BH, total;   // T tokens per sequence, Tp = 64 N rows per sequence in the workspace; total = BH*N chunks
     const bf16 *beta, *alpha, *lam;
     const float* g;
@@ -337,8 +344,12 @@ __device__ __forceinline__ void ld8(uint32_t taddr, float* v) { tmem_ld8(taddr, 
 // HAS_LAM = false: lambda is absent and d lambda is not asked for (the gated delta rule, Eq. 3): X = K, nothing is built,
 // no column sum for d lambda.  HAS_ALPHA = false: alpha is absent and d alpha is not asked for (no forget gate; with
 // HAS_LAM = false too this is DeltaNet, Eq. 2): every decay factor is 1 and none of the sums that only feed d alpha is
-// taken.  The <true, true> instance serves every other case (an absent input then reads as lambda = 0, alpha = 1).
-template <bool HAS_LAM, bool HAS_ALPHA>
+// taken.  The <true, true> instances serve every other case (an absent input then reads as lambda = 0, alpha = 1).
+// NORM (QD_NORM_QK): the Q and K tiles arrive un-normalised and are normalised in place with the factors the forward
+// left in the workspace; dq and dk are taken through the normalisation, dx = r (dx^ - x^ <x^, dx^>), which needs the
+// row sums <x^, dx^> before anything can be stored: the last epilogue then runs twice, once for the sums and once
+// for the stores.
+template <bool HAS_LAM, bool HAS_ALPHA, bool NORM>
 __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_constant__ CUtensorMap mapQ,
                                                               const __grid_constant__ CUtensorMap mapK,
                                                               const __grid_constant__ CUtensorMap mapV,
@@ -361,7 +372,8 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C];
     __shared__ float4 scf[C];         // per token: {gamma beta, gamma_C / gamma, gamma, lambda}, one load in the last epilogue
     __shared__ float sred[3][4][C];   // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
-    __shared__ float srow[6][kNWG][C];   // per-row partial sums over each warpgroup's columns: rPP, d beta, t2, rAA; [4], [5]: d beta and
+    __shared__ float srq[C], srk[C];   // NORM: 1/|q_t|, 1/|k_t|
+    __shared__ __align__(16) float srow[6][kNWG][C];   // per-row partial sums over each warpgroup's columns: rPP, d beta, t2, rAA; [4], [5]: d beta and
                                          // rAA of the column groups that the upper lanes take
     __shared__ float sdg[C], skd[C], swp[kBwdCompute / 32], scol[2][kBwdCompute / 64][C];
 
@@ -446,7 +458,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         tma_prefetch_2d(&mapdDt, 0, yc);
     };
     // coefficients of token tid (< C) of a chunk, fetched one chunk ahead into registers
-    float cf_beta = 0.f, cf_lam = 0.f, cf_alpha = 1.f, cf_g = 0.f;
+    float cf_beta = 0.f, cf_lam = 0.f, cf_alpha = 1.f, cf_g = 0.f, cf_rq = 1.f, cf_rk = 1.f;
     auto fetch_coef = [&](int ch) {
         if (tid < C) {
             int n_, bh_; item(ch, n_, bh_);
@@ -457,6 +469,10 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             cf_lam = (live && p.lam) ? gate(__bfloat162float(p.lam[cr]), p.logits) : 0.f;
             cf_alpha = (live && p.alpha) ? gate(__bfloat162float(p.alpha[cr]), p.logits) : 1.f;
             cf_g = p.g[(size_t)bh_ * p.Tp + (size_t)n_ * C + tid];
+            if (NORM) {
+                cf_rq = p.rqk[(size_t)bh_ * p.Tp + (size_t)n_ * C + tid];
+                cf_rk = p.rqk[(size_t)p.BH * p.Tp + (size_t)bh_ * p.Tp + (size_t)n_ * C + tid];
+            }
         }
     };
     // bounded wait; once any wait has expired every later wait returns at once and the kernel drains: all
@@ -605,6 +621,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         salpha[tid] = cf_alpha;
         sg[tid] = cf_g;
         sgam[tid] = __expf(cf_g);
+        if (NORM) { srq[tid] = cf_rq; srk[tid] = cf_rk; }
     }
     csync();
     if (tid < C) {
@@ -614,10 +631,11 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     wait(&bar_load, ph);
     wait(&bar_late, ph);
     // ---- X = K + lambda Q (the products that do not read X are already running); partial <dh,h>_F -------
-    if (has_lam) {
+    if (has_lam || NORM) {
         constexpr int kPer = 16 / (kBwdCompute / 64);     // 16-byte chunks of a row per thread
         const int r = tid & 63, part = tid >> 6;
         const float lm = slam[r];
+        const float rq = NORM ? srq[r] : 1.f, rk = NORM ? srk[r] : 1.f;
 #pragma unroll
         for (int cc = 0; cc < kPer; ++cc) {
             const int ci = part * kPer + cc;              // chunk 0..15 of the row: block ci>>3, chunk ci&7
@@ -625,9 +643,17 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             float qv[8], kv[8];
             load8(sm + oQ + off, qv);
             load8(sm + oK + off, kv);
+            if (NORM) {                                   // q^ and k^ in place: no product has read Q or K yet
 #pragma unroll
-            for (int e = 0; e < 8; ++e) kv[e] = fmaf(lm, qv[e], kv[e]);
-            sts128(sm + oX + off, pack8(kv));
+                for (int e = 0; e < 8; ++e) { qv[e] *= rq; kv[e] *= rk; }
+                sts128(sm + oQ + off, pack8(qv));
+                sts128(sm + oK + off, pack8(kv));
+            }
+            if (has_lam) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) kv[e] = fmaf(lm, qv[e], kv[e]);
+                sts128(sm + oX + off, pack8(kv));
+            }
         }
     }
     fence_proxy_async();
@@ -847,8 +873,15 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     if (next_id < p.total) fetch_coef(next_id);
     wait(&bm_5, ph);
     tc_fence_after();
-    {
-        const int i = l;                                            // d_k index; my 32 tokens c0..c0+31 in groups of 8
+    // The last epilogue: thread = d_k index i, its 16 tokens in groups of 8.  RED: take the column sums (over i, i.e.
+    // across the lanes); STO: write dk and dq, transposed, into their staging tiles.
+    // NORM: two more column sums, <k^, dk^> and <q^, dq^>, and per token {1/|k|, <k^,dk^>/|k|, 1/|q|, <q^,dq^>/|q|}; they
+    // live in the row-sum scratch, which is dead by now (the barrier below makes sure its last readers are done)
+    float (*sredN)[4][C] = reinterpret_cast<float (*)[4][C]>(&srow[0][0][0]);
+    float4* snf = reinterpret_cast<float4*>(&srow[2][0][0]);
+    auto last_pass = [&](auto red_tag, auto sto_tag) {
+        constexpr bool RED = decltype(red_tag)::value, STO = decltype(sto_tag)::value;
+        const int i = l;
         unsigned char* stk = sm + oStDk + (i >> 6) * 8192;
         unsigned char* stq = sm + oStDq + (i >> 6) * 8192;
         const unsigned char* qcol = sm + oQ + (i >> 6) * 8192;
@@ -870,29 +903,68 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 const float4 cf = scf[t];
                 const float dxe = fmaf(cf.x, dx[e], v[e]);                                  // dX^T[i][t]
                 const float kh = cf.y * u[e];                                               // (K-> ^T applied to dh Delta^T)[i][t]
-                sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(w[e] + kh + dxe));
-                // <(K-> dh)_t, Delta_t> = gamma_C/gamma_t sum_i K[t][i] (dh Delta^T)[i][t], all of it in fp32
-                u[e] = kh * __bfloat162float(*reinterpret_cast<const bf16*>(kcol + sw128_off(t, i & 63)));
                 const float q1 = cf.z * z[e];
-                sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(q1 + y[e] + cf.w * dxe));
+                float dkh = w[e] + kh + dxe;                                                // d k^ (d k without NORM)
+                float dqh = q1 + y[e] + cf.w * dxe;                                         // d q^
+                const float kv = __bfloat162float(*reinterpret_cast<const bf16*>(kcol + sw128_off(t, i & 63)));
                 const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(t, i & 63)));
-                z[e] = q1 * qv;
-                dx[e] = dxe * qv;
+                if (STO) {
+                    if (NORM) {
+                        const float4 nf = snf[t];
+                        dkh = fmaf(nf.x, dkh, -kv * nf.y);
+                        dqh = fmaf(nf.z, dqh, -qv * nf.w);
+                    }
+                    sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(dkh));
+                    sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(dqh));
+                }
+                if (RED) {
+                    // <(K-> dh)_t, Delta_t> = gamma_C/gamma_t sum_i K[t][i] (dh Delta^T)[i][t], all of it in fp32
+                    u[e] = kh * kv;
+                    z[e] = q1 * qv;
+                    dx[e] = dxe * qv;
+                    if (NORM) { w[e] = dkh * kv; y[e] = dqh * qv; }
+                }
             }
-            // column sums over the d_k index (across the lanes): d lambda, and the two that only the decay gradient needs
-            if (want_dl) {
-                const float dls = col_reduce8(dx, lane);
-                if ((lane & 3) == 0) sred[1][wq][cb + col8_of_lane(lane)] = dls;
-            }
-            if (want_da) {
-                const float t1s = col_reduce8(z, lane), kds = col_reduce8(u, lane);
-                if ((lane & 3) == 0) {
-                    const int col = cb + col8_of_lane(lane);
-                    sred[0][wq][col] = kds;
-                    sred[2][wq][col] = t1s;
+            if (RED) {
+                // column sums over the d_k index (across the lanes): d lambda, the two that only the decay gradient
+                // needs, and with NORM the two of the normalisation's backward
+                if (want_dl) {
+                    const float dls = col_reduce8(dx, lane);
+                    if ((lane & 3) == 0) sred[1][wq][cb + col8_of_lane(lane)] = dls;
+                }
+                if (want_da) {
+                    const float t1s = col_reduce8(z, lane), kds = col_reduce8(u, lane);
+                    if ((lane & 3) == 0) {
+                        const int col = cb + col8_of_lane(lane);
+                        sred[0][wq][col] = kds;
+                        sred[2][wq][col] = t1s;
+                    }
+                }
+                if (NORM) {
+                    const float cks = col_reduce8(w, lane), cqs = col_reduce8(y, lane);
+                    if ((lane & 3) == 0) {
+                        const int col = cb + col8_of_lane(lane);
+                        sredN[0][wq][col] = cks;
+                        sredN[1][wq][col] = cqs;
+                    }
                 }
             }
         }
+    };
+    if (NORM) {
+        csync();
+        last_pass(std::true_type{}, std::false_type{});
+        csync();
+        if (tid < C) {
+            float ck = 0.f, cq = 0.f;
+#pragma unroll
+            for (int w4 = 0; w4 < 4; ++w4) { ck += sredN[0][w4][tid]; cq += sredN[1][w4][tid]; }
+            snf[tid] = make_float4(srk[tid], srk[tid] * ck, srq[tid], srq[tid] * cq);
+        }
+        csync();
+        last_pass(std::false_type{}, std::true_type{});
+    } else {
+        last_pass(std::true_type{}, std::true_type{});
     }
     fence_proxy_async();
     tc_fence_before();
@@ -964,6 +1036,7 @@ cudaError_t tc_chain_bwd(const ChunkArgs& a) {
     ChainBwdParams p{};
     p.Tp = Tp; p.H = s.H; p.N = (int)N;
     p.dhT_early = a.own_predecessor ? 1 : 0;
+    p.rk = a.norm ? (const float*)(a.ws + a.TL.rqk) + BH * Tp : nullptr;
     p.g = (const float*)(a.ws + a.TL.g);
     p.dhT = a.dhT; p.dh0 = a.dh0;
     p.status = (unsigned*)(a.ws + a.TL.status);
@@ -998,11 +1071,15 @@ cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
     p.g = (const float*)(a.ws + a.TL.g);
     p.dbeta = a.dbeta; p.dalpha = a.dalpha; p.dlam = a.dlam;
     p.logits = a.logits ? 1 : 0;
+    p.rqk = a.norm ? (const float*)(a.ws + a.TL.rqk) : nullptr;
     p.status = (unsigned*)(a.ws + a.TL.status);
     // the instance without lambda / without the forget gate needs the input AND its gradient to be absent
     const bool lam = a.lam || a.dlam, alpha = a.alpha || a.dalpha;
-    auto kern = lam ? (alpha ? k_tc_chunk_bwd<true, true> : k_tc_chunk_bwd<true, false>)
-                    : (alpha ? k_tc_chunk_bwd<false, true> : k_tc_chunk_bwd<false, false>);
+    auto kern = lam ? (alpha ? k_tc_chunk_bwd<true, true, false> : k_tc_chunk_bwd<true, false, false>)
+                    : (alpha ? k_tc_chunk_bwd<false, true, false> : k_tc_chunk_bwd<false, false, false>);
+    if (a.norm)
+        kern = lam ? (alpha ? k_tc_chunk_bwd<true, true, true> : k_tc_chunk_bwd<true, false, true>)
+                   : (alpha ? k_tc_chunk_bwd<false, true, true> : k_tc_chunk_bwd<false, false, true>);
     cudaError_t e = set_smem(kern, kBwdSmem);
     if (e != cudaSuccess) return e;
     // persistent: one CTA per SM walks the work items with stride gridDim.x

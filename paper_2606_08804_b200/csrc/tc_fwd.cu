@@ -39,6 +39,7 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 // =================================================================================================
 struct PrepParams {
     int logits;                // beta, alpha, lambda are logits of sigmoid gates
+    float* rqk;                // non-null: L2-normalise q and k here; [0, BH*Tp) <- 1/|q_t|, [BH*Tp, 2 BH*Tp) <- 1/|k_t|
     int T, Tp, H, N, BH;       // T tokens per sequence; the workspace holds Tp = 64 N >= T rows per sequence (N even)
     const bf16 *beta, *alpha, *lam;
     float* g;
@@ -133,6 +134,37 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         if (warp == 0) tmem_dealloc(tbase, 256);
         return;
     }
+    // row-wise work: 16 lanes cover one 256-byte row (chunk `ch` of 16 bytes each), 16 rows per pass
+    const int ch = tid & 15, rsub = tid >> 4;
+    const uint32_t coff = (ch >> 3) * 16384;
+    if (p.rqk) {
+        // q^ = q / sqrt(|q|^2 + eps), k^ likewise, in place: everything below (and every later kernel, through
+        // diag(gamma) Q^ and the 1/|k| written here) works on the normalised rows
+        const size_t nrows = (size_t)p.BH * p.Tp;
+#pragma unroll 2
+        for (int it = 0; it < 8; ++it) {
+            const int row = it * 16 + rsub;
+            const uint32_t off = coff + sw128_chunk(row, ch & 7);
+            float qv[8], kv[8], sq = 0.f, sk = 0.f;
+            load8(sQ + off, qv);
+            load8(sK + off, kv);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { sq = fmaf(qv[e], qv[e], sq); sk = fmaf(kv[e], kv[e], sk); }
+#pragma unroll
+            for (int o = 1; o < 16; o <<= 1) {
+                sq += __shfl_xor_sync(0xffffffffu, sq, o);
+                sk += __shfl_xor_sync(0xffffffffu, sk, o);
+            }
+            const float rq = rsqrtf(sq + kNormEps), rk = rsqrtf(sk + kNormEps);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { qv[e] *= rq; kv[e] *= rk; }
+            sts128(sQ + off, pack8(qv));
+            sts128(sK + off, pack8(kv));
+            if (ch == 0) { p.rqk[wtok0 + row] = rq; p.rqk[nrows + wtok0 + row] = rk; }
+        }
+        fence_proxy_async();
+        __syncthreads();
+    }
     if (tid == 0) {
         tc_fence_after();
         // G2 = Q K^T -> columns [128,256);  without lambda also G1 = K K^T -> columns [0,128)
@@ -140,9 +172,6 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         if (!has_lam) umma_product<false, false>(tbase, smem_u32(sK), 16384, smem_u32(sK), 16384, 128, 128, false);
         umma_commit(&bar_mma);
     }
-    // row-wise work: 16 lanes cover one 256-byte row (chunk `ch` of 16 bytes each), 16 rows per pass
-    const int ch = tid & 15, rsub = tid >> 4;
-    const uint32_t coff = (ch >> 3) * 16384;
     // meanwhile: Qg = gamma Q to the workspace, a warp writes two full rows per store
     {
         bf16* qg = p.Qg + wtok0 * D + ch * 8;
@@ -345,7 +374,9 @@ struct ChainParams {
     const float* h0;
     float* hT;
     int save;                  // also store, per chunk, the bf16 entry state (mapHs) and Delta^T (mapDt)
-    int has_alpha;             // 0: no forget gate (alpha absent), every decay factor is 1
+    int scaled;                // 0: no forget gate and no key normalisation: every per-token factor on Delta is 1
+    const float* rk;           // non-null (QD_NORM_QK): 1/|k_t| per workspace row; the keys are read un-normalised and
+                               // the factor is folded into the per-token scale of Delta
     unsigned* status;
 };
 
@@ -488,7 +519,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
                         d1[e] = u[e] * sc[cc * 8 + e];
                     }
                     sts128(sD + off, pack8(u));
-                    if (p.has_alpha) sts128(sDs + off, pack8(d1));      // without a forget gate the scaled copy is Delta itself
+                    if (p.scaled) sts128(sDs + off, pack8(d1));         // all factors 1: the scaled copy is Delta itself
                 }
             }
             tc_fence_before();
@@ -525,7 +556,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         const bool lead = (tid & 31) == 0;
         grid_dep_wait();
         grid_dep_launch();
-        const uint32_t aH = smem_u32(sH), aD = smem_u32(sD), aDs = p.has_alpha ? smem_u32(sDs) : smem_u32(sD);
+        const uint32_t aH = smem_u32(sH), aD = smem_u32(sD), aDs = p.scaled ? smem_u32(sDs) : smem_u32(sD);
         for (int n = 0; n < p.N; ++n) {
             const uint32_t st = smem_u32(smem + (n & 1) * kStage);
             const uint32_t tO = tO0 + 64 * (n & 1);
@@ -575,14 +606,17 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_fwd(const __grid_con
         if (lead) { issue_load(0); if (p.N > 1) issue_load(1); }
         const int ln = tid & 31;
         float g0 = gseq[ln], g1 = gseq[32 + ln], gc = gseq[C - 1];     // cumulative log-decays of chunk 0
+        const float* rkseq = p.rk ? p.rk + (size_t)bh * p.Tp : nullptr;
+        float r0 = rkseq ? rkseq[ln] : 1.f, r1 = rkseq ? rkseq[32 + ln] : 1.f;
         for (int n = 0; n < p.N; ++n) {
-            sG[n & 1][ln] = __expf(gc - g0);
-            sG[n & 1][32 + ln] = __expf(gc - g1);
+            sG[n & 1][ln] = __expf(gc - g0) * r0;
+            sG[n & 1][32 + ln] = __expf(gc - g1) * r1;
             if (ln == 0) sG[n & 1][64] = __expf(gc);
             __syncwarp();
             if (n + 1 < p.N) {                                  // in flight while this chunk is processed
                 const float* gn = gseq + (size_t)(n + 1) * C;
                 g0 = gn[ln]; g1 = gn[32 + ln]; gc = gn[C - 1];
+                if (rkseq) { r0 = rkseq[(size_t)(n + 1) * C + ln]; r1 = rkseq[(size_t)(n + 1) * C + 32 + ln]; }
             }
             if (lead) {
                 // every store issued so far (Delta^T of chunk n-1, output of chunk n-2) has read its tile:
@@ -656,6 +690,7 @@ TcLayout tc_layout(const qd_shape& s) {
     L.P = take(BH * T * kChunk * 2);
     L.Wt = take(BH * T * s.dk * 2);
     L.Ut = take(BH * T * s.dv * 2);
+    L.rqk = take(2 * BH * T * 4);
     L.fwd_end = off;
     const size_t N = T / kChunk;
     L.Mt = take(BH * T * kChunk * 2);
@@ -680,6 +715,7 @@ cudaError_t tc_prep(const ChunkArgs& a) {
     PrepParams p{};
     p.T = s.T; p.Tp = Tp; p.H = s.H; p.N = Tp / kChunk; p.BH = s.B * s.H;
     p.logits = a.logits ? 1 : 0;
+    p.rqk = a.norm ? (float*)(a.ws + a.TL.rqk) : nullptr;
     p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
     p.g = (float*)(a.ws + a.TL.g);
     p.Qg = (bf16*)(a.ws + a.TL.Qg); p.P = (bf16*)(a.ws + a.TL.P);
@@ -711,7 +747,8 @@ cudaError_t tc_chain_fwd(const ChunkArgs& a) {
     p.g = (const float*)(a.ws + a.TL.g);
     p.h0 = a.h0; p.hT = a.hT;
     p.save = a.save ? 1 : 0;
-    p.has_alpha = a.alpha ? 1 : 0;
+    p.scaled = (a.alpha || a.norm) ? 1 : 0;
+    p.rk = a.norm ? (const float*)(a.ws + a.TL.rqk) + BH * Tp : nullptr;
     p.status = (unsigned*)(a.ws + a.TL.status);
     cudaError_t e = set_smem(k_tc_chain_fwd, kChainSmem);
     if (e != cudaSuccess) return e;

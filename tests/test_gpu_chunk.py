@@ -369,3 +369,52 @@ def test_gates_from_logits(dtype, T):
     ro5, rh5 = orc.forward_logits(d["q"][:, :S], d["k"][:, :S], d["v"][:, :S], z["beta"][:, :S], z["alpha"][:, :S],
                                   z["lam"][:, :S], d["h0"])
     assert gu.rel_err(od, ro5) <= gu.TOL[dtype] and gu.rel_err(state, rh5) <= gu.TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype,T,logits,drop", [("bf16", 300, False, ()), ("bf16", 256, True, ()), ("bf16", 192, False, ("lam", "alpha")),
+                                                 ("f32", 150, False, ()), ("f32", 128, True, ("lam",))])
+def test_in_kernel_l2_normalisation(dtype, T, logits, drop):
+    # QD_NORM_QK: q and k arrive un-normalised (rows of very different lengths); the kernels normalise them and the
+    # backward returns gradients with respect to the un-normalised rows.  Alone, with logit gates, with absent inputs.
+    from oracle import recurrence as orc
+    from paper_2606_08804_b200 import binding as qd
+    base = gen.CONFIGS["cfg2"] if dtype == "bf16" else replace(gen.CONFIGS["cfg0"], h0=True, backward=True)
+    cfg = replace(base, B=2, H=3, T=T, regime="alpha_slow", seed=103 + T)
+    d = gen.make_chunk_inputs(cfg)
+    r = np.random.default_rng(11)
+    rnd = (lambda x: gen.round_bf16(x.astype(np.float32))) if dtype == "bf16" else (lambda x: x.astype(np.float32))
+    scale = lambda shape: np.exp(r.normal(0.0, 1.0, shape[:-1] + (1,)))          # row lengths over two orders of magnitude
+    d["q"] = rnd(d["q"] * scale(d["q"].shape))
+    d["k"] = rnd(d["k"] * scale(d["k"].shape))
+    if logits:
+        shp = (cfg.B, cfg.T, cfg.H)
+        d["beta"], d["alpha"], d["lam"] = rnd(r.normal(0.0, 1.5, shp)), rnd(r.normal(3.0, 1.5, shp)), rnd(r.normal(-0.8, 1.0, shp))
+    for n in drop:
+        d[n] = None
+    t = gu.dev_inputs(d, cfg.dtype)
+    ro, rh = orc.forward_fused(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"], logits=logits, norm_qk=True)
+    ref = orc.backward_fused(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"], d["dO"], d["dhT"],
+                             logits=logits, norm_qk=True)
+    lab = _label(cfg, " norm_qk%s%s" % (" logits" if logits else "", " without " + "+".join(drop) if drop else ""))
+    for reuse in (False, True):
+        o, hT, ws = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], save_for_bwd=reuse,
+                                 logits=logits, norm_qk=True)
+        g = qd.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], t["dO"], t["dhT"],
+                         workspace=ws if reuse else None, reuse_fwd=reuse, logits=logits, norm_qk=True)
+        torch.cuda.synchronize()
+        assert qd.workspace_status(ws) == 0 if reuse else True
+        gu.check(lab, "o", o, ro, cfg.dtype)
+        gu.check(lab, "hT", hT, rh, cfg.dtype, state=True)
+        for n in ("dq", "dk", "dv", "dbeta", "dalpha", "dlam", "dh0"):
+            if g.get(n) is not None:
+                gu.check(lab, n, g[n], ref[n], cfg.dtype, state=(n == "dh0"))
+    S = 4
+    c = lambda x: None if x is None else x[:, :S].contiguous()
+    state = t["h0"].clone()
+    od = qd.recurrent_steps(c(t["q"]), c(t["k"]), c(t["v"]), c(t["beta"]), c(t["alpha"]), c(t["lam"]), state,
+                            logits=logits, norm_qk=True)
+    torch.cuda.synchronize()
+    cut = lambda a: None if a is None else a[:, :S]
+    roS, rhS = orc.forward_fused(cut(d["q"]), cut(d["k"]), cut(d["v"]), cut(d["beta"]), cut(d["alpha"]), cut(d["lam"]), d["h0"],
+                                 logits=logits, norm_qk=True)
+    assert gu.rel_err(od, roS) <= gu.TOL[dtype] and gu.rel_err(state, rhS) <= gu.TOL[dtype]

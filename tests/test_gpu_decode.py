@@ -163,3 +163,43 @@ def test_multi_token_step_null_coefficients_and_argument_errors():
     assert lib.qdelta_recurrent_steps(1, 0, 1, 64, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 0, None) == 1
     assert lib.qdelta_recurrent_steps(1, 2, 1, 96, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 0, None) == 2
     assert lib.qdelta_recurrent_steps(1, 2, 1, 64, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 8, None) == 1
+
+
+def test_decode_steps_replayed_from_a_cuda_graph():
+    # a fixed run of decode steps captured once in a CUDA graph and replayed: the library enqueues only kernels on the
+    # caller's stream (no allocation, no synchronisation), so capture works and a replay equals the eager run
+    from paper_2606_08804_b200 import binding as qd
+    cfg = replace(gen.CONFIGS["cfg4"], B=4, H=3)
+    n = 6
+    tok = gen.make_decode_tokens(cfg, 0, n)
+    dev = {k_: gu.to_dev(a, torch.bfloat16) for k_, a in tok.items()}
+    s0 = gu.to_dev(gen.make_decode_state(cfg), torch.float32)
+    outs = [torch.empty((cfg.B, cfg.H, cfg.dv), dtype=torch.bfloat16, device="cuda") for _ in range(n)]
+
+    def run(state):
+        for i in range(n):
+            qd.recurrent_step(dev["q"][i], dev["k"][i], dev["v"][i], dev["beta"][i], dev["alpha"][i], dev["lam"][i],
+                              state, outs[i])
+    eager_state = s0.clone()
+    run(eager_state)
+    torch.cuda.synchronize()
+    eager_outs = [o.clone() for o in outs]
+    state = s0.clone()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        run(state)                                   # warm-up on the capture stream
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        run(state)
+    for rep in range(2):
+        state.copy_(s0)
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(state, eager_state)
+        for a, b in zip(outs, eager_outs):
+            assert torch.equal(a, b)

@@ -150,3 +150,37 @@ def test_logit_gates_forward_is_sigmoid_composition_and_gradients_match_finite_d
         assert np.allclose(g[n], g0[n], rtol=1e-12, atol=1e-12)
     gn = orc.backward_logits(d["q"], d["k"], d["v"], z["beta"], None, None, d["h0"], up["dO"], up["dhT"], ckpt=4)
     assert gn["dalpha"] is None and gn["dlam"] is None
+
+
+def test_l2_normalisation_stage_pinned():
+    # unit rows up to the constant under the root, closed form on a 3-4-0 row, gradient orthogonal to the row
+    # direction (for eps -> 0), and central finite differences through the whole composite for q and k
+    x = np.array([[3.0, 4.0, 0.0]])
+    assert np.allclose(orc.l2_normalize(x), x / np.sqrt(25.0 + orc.NORM_EPS), rtol=0, atol=1e-15)
+    d, up = _rand(31)
+    r = np.random.default_rng(32)
+    d["q"] = 2.0 * r.standard_normal(d["q"].shape)          # un-normalised rows
+    d["k"] = 0.5 * r.standard_normal(d["k"].shape)
+    assert np.allclose(np.linalg.norm(orc.l2_normalize(d["q"]), axis=-1), 1.0, atol=1e-6)
+    gx = orc.l2_normalize_backward(d["q"], r.standard_normal(d["q"].shape))
+    assert np.max(np.abs(np.sum(gx * d["q"], axis=-1))) < 1e-5
+
+    def loss():
+        o, hT = orc.forward_fused(**d, norm_qk=True)
+        return float(np.sum(o * up["dO"]) + np.sum(hT * up["dhT"]))
+    g = orc.backward_fused(**d, **up, ckpt=4, norm_qk=True)
+    eps = 1e-6
+    for name, gname in (("q", "dq"), ("k", "dk"), ("v", "dv"), ("beta", "dbeta")):
+        flat, gflat = d[name].reshape(-1), g[gname].reshape(-1)
+        for i in range(0, flat.size, 3):
+            old = flat[i]
+            flat[i] = old + eps; lp = loss()
+            flat[i] = old - eps; lm = loss()
+            flat[i] = old
+            fd = (lp - lm) / (2 * eps)
+            assert abs(fd - gflat[i]) <= 2e-6 * max(1.0, abs(fd)), (name, i, fd, gflat[i])
+    # rows that are already unit vectors: the stage changes nothing but the 1e-6 under the root
+    d2, up2 = _rand(33)
+    o1, h1 = orc.forward_fused(**d2, norm_qk=True)
+    o2, h2 = orc.forward(**d2)
+    assert np.allclose(o1, o2, rtol=0, atol=1e-5) and np.allclose(h1, h2, rtol=0, atol=1e-5)
