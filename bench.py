@@ -243,16 +243,59 @@ def extra_workload(torch, qd, gen, cfg, pk, pk_kind, backward, steps, regions, d
     assert qd.workspace_status(w.ws) == 0, "device-side status word is set"
     times = time_regions(torch, w.step, steps, regions, torch.cuda.synchronize)
     st = region_stats(times, steps, None)
+    qd.profile_read(reset=True)
+    qd.profile_enable(True)                 # per-kernel durations, in a pass of their own (they serialise the launches)
+    for _ in range(min(steps, 5)):
+        w.step()
+    torch.cuda.synchronize()
+    qd.profile_enable(False)
+    stage_ms = {n: v[0] / v[1] for n, v in qd.profile_read(reset=True).items() if v[1] > 0}
     rl = path_roofline(cfg, pk, fwd=True, bwd=backward)
     ms = st["ms_per_step_median"]
     out = {"workload": workload_name(cfg, backward), "ms_per_step": ms, "tokens_per_s": cfg.B * cfg.T / (ms * 1e-3),
            "roofline_ms": rl["roofline_ms"], "frac": rl["roofline_ms"] / ms, "frac_nominal": rl["roofline_ms_nominal"] / ms,
-           "peak_kind": "of " + pk_kind, "regions": st}
+           "peak_kind": "of " + pk_kind, "regions": st, "stage_ms_per_launch": stage_ms}
     if drop:
         out["absent_inputs"] = list(drop)
     del w
     torch.cuda.empty_cache()
     return out
+
+
+def torch_preprocessing_ms(torch, gen, cfg, steps=10):
+    """What the stages QD_NORM_QK | QD_COEF_LOGITS fuse cost when a caller runs them as separate PyTorch operations around
+    the plain call: forward (normalise q and k, three sigmoids) and backward (through the normalisation and the
+    sigmoids), bf16 tensors of the same shape.  Context for `fused_preprocessing`, not part of the library."""
+    bf = torch.bfloat16
+    B, T, H, dk = cfg.B, cfg.T, cfg.H, cfg.dk
+    g = torch.Generator(device="cuda").manual_seed(0)
+    q, k, dqh, dkh = (torch.randn((B, T, H, dk), device="cuda", generator=g).to(bf) for _ in range(4))
+    zb, za, zl, db, da, dl = (torch.randn((B, T, H), device="cuda", generator=g).to(bf) for _ in range(6))
+
+    def step():
+        outs = []
+        for x, dxh in ((q, dqh), (k, dkh)):
+            xf = x.float()
+            r = torch.rsqrt((xf * xf).sum(-1, keepdim=True) + 1e-6)
+            xh = xf * r
+            outs.append(xh.to(bf))                                   # forward: the normalised rows the kernel is given
+            d = dxh.float()
+            outs.append((r * (d - xh * (xh * d).sum(-1, keepdim=True))).to(bf))   # backward through the normalisation
+        for z, dgate in ((zb, db), (za, da), (zl, dl)):
+            s_ = torch.sigmoid(z.float())
+            outs.append(s_.to(bf))
+            outs.append(dgate.float() * s_ * (1 - s_))
+        return outs
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
 
 
 def run_ours(args, cfg):
@@ -428,12 +471,15 @@ def run_ours(args, cfg):
         var = {}
         for name, drop in (("lambda_absent", ("lam",)), ("alpha_absent", ("alpha",)), ("both_absent", ("lam", "alpha"))):
             r = extra_workload(torch, qd, gen, cfg, pk, pk_kind, True, 20, 3, drop=drop)
-            var[name] = {"ms_per_step": r["ms_per_step"], "speedup_vs_full_rule": base / r["ms_per_step"]}
+            var[name] = {"ms_per_step": r["ms_per_step"], "speedup_vs_full_rule": base / r["ms_per_step"],
+                         "stage_ms_per_launch": r["stage_ms_per_launch"]}
         extras["variants"] = var
         # pre-processing fused into the kernels: L2 normalisation of q, k and sigmoid gates (with their backward)
         r = extra_workload(torch, qd, gen, cfg, pk, pk_kind, True, 20, 3, fused=True)
         extras["fused_preprocessing"] = {"flags": "QD_NORM_QK | QD_COEF_LOGITS", "ms_per_step": r["ms_per_step"],
-                                         "overhead_ms_vs_plain": r["ms_per_step"] - base}
+                                         "overhead_ms_vs_plain": r["ms_per_step"] - base,
+                                         "stage_ms_per_launch": r["stage_ms_per_launch"],
+                                         "same_stages_as_torch_ops_ms": torch_preprocessing_ms(torch, gen, cfg)}
 
     # ---- decode step (separate configuration), in place over a long run of steps ------------------
     decode = bench_decode(args, qd, gen, torch, pk, pk_kind) if (rank == 0 and not args.no_extras) else None

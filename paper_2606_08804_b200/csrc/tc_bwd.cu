@@ -14,7 +14,6 @@
 #include "internal.h"
 #include "sm100.cuh"
 
-#include <type_traits>
 
 namespace qd {
 namespace {
@@ -372,7 +371,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     __shared__ float sbeta[C], slam[C], salpha[C], sg[C], sgam[C];
     __shared__ float4 scf[C];         // per token: {gamma beta, gamma_C / gamma, gamma, lambda}, one load in the last epilogue
     __shared__ float sred[3][4][C];   // per-warp column sums: [0] <(K-> dh)_r, Delta_r>, [1] d lambda, [2] rowsum(dQ1 o Q)
-    __shared__ float srq[C], srk[C];   // NORM: 1/|q_t|, 1/|k_t|
+    __shared__ float2 srn[C];          // NORM: {1/|k_t|, 1/|q_t|}
     __shared__ __align__(16) float srow[6][kNWG][C];   // per-row partial sums over each warpgroup's columns: rPP, d beta, t2, rAA; [4], [5]: d beta and
                                          // rAA of the column groups that the upper lanes take
     __shared__ float sdg[C], skd[C], swp[kBwdCompute / 32], scol[2][kBwdCompute / 64][C];
@@ -621,7 +620,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         salpha[tid] = cf_alpha;
         sg[tid] = cf_g;
         sgam[tid] = __expf(cf_g);
-        if (NORM) { srq[tid] = cf_rq; srk[tid] = cf_rk; }
+        if (NORM) srn[tid] = make_float2(cf_rk, cf_rq);
     }
     csync();
     if (tid < C) {
@@ -635,7 +634,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
         constexpr int kPer = 16 / (kBwdCompute / 64);     // 16-byte chunks of a row per thread
         const int r = tid & 63, part = tid >> 6;
         const float lm = slam[r];
-        const float rq = NORM ? srq[r] : 1.f, rk = NORM ? srk[r] : 1.f;
+        const float rq = NORM ? srn[r].y : 1.f, rk = NORM ? srn[r].x : 1.f;
 #pragma unroll
         for (int cc = 0; cc < kPer; ++cc) {
             const int ci = part * kPer + cc;              // chunk 0..15 of the row: block ci>>3, chunk ci&7
@@ -873,14 +872,16 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     if (next_id < p.total) fetch_coef(next_id);
     wait(&bm_5, ph);
     tc_fence_after();
-    // The last epilogue: thread = d_k index i, its 16 tokens in groups of 8.  RED: take the column sums (over i, i.e.
-    // across the lanes); STO: write dk and dq, transposed, into their staging tiles.
-    // NORM: two more column sums, <k^, dk^> and <q^, dq^>, and per token {1/|k|, <k^,dk^>/|k|, 1/|q|, <q^,dq^>/|q|}; they
-    // live in the row-sum scratch, which is dead by now (the barrier below makes sure its last readers are done)
+    // The last epilogue: thread = d_k index i, its 16 tokens in groups of 8: dk and dq, transposed, into their staging
+    // tiles, and the column sums (over i, i.e. across the lanes) that d lambda, the decay gradient and, with NORM, the
+    // backward of the normalisation need.
+    // NORM: dx = r (dx^ - x^ <x^, dx^>).  r dx^ is staged here; the sums <k^, dk^> and <q^, dq^> go to scratch over the
+    // row sums, which are dead by now (the barrier makes sure their last readers are done); the second term is
+    // subtracted from the staged rows afterwards, once the sums are complete.
     float (*sredN)[4][C] = reinterpret_cast<float (*)[4][C]>(&srow[0][0][0]);
-    float4* snf = reinterpret_cast<float4*>(&srow[2][0][0]);
-    auto last_pass = [&](auto red_tag, auto sto_tag) {
-        constexpr bool RED = decltype(red_tag)::value, STO = decltype(sto_tag)::value;
+    float2* snf = reinterpret_cast<float2*>(&srow[2][0][0]);        // per token {<k^,dk^>/|k|, <q^,dq^>/|q|}
+    if (NORM) csync();
+    {
         const int i = l;
         unsigned char* stk = sm + oStDk + (i >> 6) * 8192;
         unsigned char* stq = sm + oStDq + (i >> 6) * 8192;
@@ -904,67 +905,71 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 const float dxe = fmaf(cf.x, dx[e], v[e]);                                  // dX^T[i][t]
                 const float kh = cf.y * u[e];                                               // (K-> ^T applied to dh Delta^T)[i][t]
                 const float q1 = cf.z * z[e];
-                float dkh = w[e] + kh + dxe;                                                // d k^ (d k without NORM)
-                float dqh = q1 + y[e] + cf.w * dxe;                                         // d q^
+                const float dkh = w[e] + kh + dxe;                                          // d k^ (d k without NORM)
+                const float dqh = q1 + y[e] + cf.w * dxe;                                   // d q^
                 const float kv = __bfloat162float(*reinterpret_cast<const bf16*>(kcol + sw128_off(t, i & 63)));
                 const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(t, i & 63)));
-                if (STO) {
-                    if (NORM) {
-                        const float4 nf = snf[t];
-                        dkh = fmaf(nf.x, dkh, -kv * nf.y);
-                        dqh = fmaf(nf.z, dqh, -qv * nf.w);
-                    }
-                    sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(dkh));
-                    sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(dqh));
-                }
-                if (RED) {
-                    // <(K-> dh)_t, Delta_t> = gamma_C/gamma_t sum_i K[t][i] (dh Delta^T)[i][t], all of it in fp32
-                    u[e] = kh * kv;
-                    z[e] = q1 * qv;
-                    dx[e] = dxe * qv;
-                    if (NORM) { w[e] = dkh * kv; y[e] = dqh * qv; }
+                float2 rn = make_float2(1.f, 1.f);
+                if (NORM) rn = srn[t];
+                sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(rn.x * dkh));
+                sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(rn.y * dqh));
+                // <(K-> dh)_t, Delta_t> = gamma_C/gamma_t sum_i K[t][i] (dh Delta^T)[i][t], all of it in fp32
+                u[e] = kh * kv;
+                z[e] = q1 * qv;
+                dx[e] = dxe * qv;
+                if (NORM) { w[e] = dkh * kv; y[e] = dqh * qv; }
+            }
+            if (want_dl) {
+                const float dls = col_reduce8(dx, lane);
+                if ((lane & 3) == 0) sred[1][wq][cb + col8_of_lane(lane)] = dls;
+            }
+            if (want_da) {
+                const float t1s = col_reduce8(z, lane), kds = col_reduce8(u, lane);
+                if ((lane & 3) == 0) {
+                    const int col = cb + col8_of_lane(lane);
+                    sred[0][wq][col] = kds;
+                    sred[2][wq][col] = t1s;
                 }
             }
-            if (RED) {
-                // column sums over the d_k index (across the lanes): d lambda, the two that only the decay gradient
-                // needs, and with NORM the two of the normalisation's backward
-                if (want_dl) {
-                    const float dls = col_reduce8(dx, lane);
-                    if ((lane & 3) == 0) sred[1][wq][cb + col8_of_lane(lane)] = dls;
-                }
-                if (want_da) {
-                    const float t1s = col_reduce8(z, lane), kds = col_reduce8(u, lane);
-                    if ((lane & 3) == 0) {
-                        const int col = cb + col8_of_lane(lane);
-                        sred[0][wq][col] = kds;
-                        sred[2][wq][col] = t1s;
-                    }
-                }
-                if (NORM) {
-                    const float cks = col_reduce8(w, lane), cqs = col_reduce8(y, lane);
-                    if ((lane & 3) == 0) {
-                        const int col = cb + col8_of_lane(lane);
-                        sredN[0][wq][col] = cks;
-                        sredN[1][wq][col] = cqs;
-                    }
+            if (NORM) {
+                const float cks = col_reduce8(w, lane), cqs = col_reduce8(y, lane);
+                if ((lane & 3) == 0) {
+                    const int col = cb + col8_of_lane(lane);
+                    sredN[0][wq][col] = cks;
+                    sredN[1][wq][col] = cqs;
                 }
             }
         }
-    };
+    }
     if (NORM) {
-        csync();
-        last_pass(std::true_type{}, std::false_type{});
         csync();
         if (tid < C) {
             float ck = 0.f, cq = 0.f;
 #pragma unroll
             for (int w4 = 0; w4 < 4; ++w4) { ck += sredN[0][w4][tid]; cq += sredN[1][w4][tid]; }
-            snf[tid] = make_float4(srk[tid], srk[tid] * ck, srq[tid], srq[tid] * cq);
+            snf[tid] = make_float2(srn[tid].x * ck, srn[tid].y * cq);
         }
         csync();
-        last_pass(std::false_type{}, std::true_type{});
-    } else {
-        last_pass(std::true_type{}, std::true_type{});
+        // staged rows (token-major, 16 bytes at a time): dk_t -= (<k^,dk^>/|k|) k^_t, dq_t likewise
+        constexpr int kPer = 16 / (kBwdCompute / 64);
+        const int r = tid & 63, part = tid >> 6;
+        const float2 nf = snf[r];
+#pragma unroll
+        for (int cc = 0; cc < kPer; ++cc) {
+            const int ci = part * kPer + cc;
+            const uint32_t off = (ci >> 3) * 8192 + sw128_chunk(r, ci & 7);
+            float a8[8], x8[8];
+            load8(sm + oStDk + off, a8);
+            load8(sm + oK + off, x8);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a8[e] = fmaf(-nf.x, x8[e], a8[e]);
+            sts128(sm + oStDk + off, pack8(a8));
+            load8(sm + oStDq + off, a8);
+            load8(sm + oQ + off, x8);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a8[e] = fmaf(-nf.y, x8[e], a8[e]);
+            sts128(sm + oStDq + off, pack8(a8));
+        }
     }
     fence_proxy_async();
     tc_fence_before();

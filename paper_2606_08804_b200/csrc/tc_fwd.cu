@@ -38,7 +38,6 @@ __device__ __forceinline__ uint4 pack8(const float* f) {
 
 // =================================================================================================
 struct PrepParams {
-    int logits;                // beta, alpha, lambda are logits of sigmoid gates
     float* rqk;                // non-null: L2-normalise q and k here; [0, BH*Tp) <- 1/|q_t|, [BH*Tp, 2 BH*Tp) <- 1/|k_t|
     int T, Tp, H, N, BH;       // T tokens per sequence; the workspace holds Tp = 64 N >= T rows per sequence (N even)
     const bf16 *beta, *alpha, *lam;
@@ -59,6 +58,10 @@ constexpr int kPrepThreads = 256;
 //   Gram epilogue         thread (row = t & 127, half = t >> 7) owns 32 columns of its TMEM lane
 //   triangular inverse    lane quad (t >> 2, t < 128) owns columns j0 + 16 k (j0 < 16) of one chunk, quad lane t & 3 the 8-row blocks t & 3 and (t & 3) + 4
 //   final epilogue        thread (d = t & 127, which = t >> 7) owns one row of U~^T resp. W~^T
+// NORM (QD_NORM_QK): L2-normalise the rows of Q and K first.  LOGITS (QD_COEF_LOGITS): the coefficients are logits of
+// sigmoid gates.  Compile-time, because even the untaken sigmoid / log-sigmoid code on the path of the scan, which
+// every later phase of the CTA waits for, cost the kernel 8 %.
+template <bool NORM, bool LOGITS>
 __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_constant__ CUtensorMap mapQ,
                                                              const __grid_constant__ CUtensorMap mapK,
                                                              const __grid_constant__ CUtensorMap mapV,
@@ -111,9 +114,9 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
         // a token past the end of the sequence is an exact no-op of the recurrence: beta = 0, alpha = 1 (and q = k = v = 0)
         const bool live = t0 + tid < p.T;
         const size_t crow = ((size_t)b * p.T + t0 + tid) * p.H + hh;
-        sbeta[tid] = live ? gate(__bfloat162float(p.beta[crow]), p.logits) : 0.f;
-        slam[tid] = (live && p.lam) ? gate(__bfloat162float(p.lam[crow]), p.logits) : 0.f;
-        float g = (live && p.alpha) ? log_gate(__bfloat162float(p.alpha[crow]), p.logits) : 0.f;
+        sbeta[tid] = live ? gate(__bfloat162float(p.beta[crow]), LOGITS) : 0.f;
+        slam[tid] = (live && p.lam) ? gate(__bfloat162float(p.lam[crow]), LOGITS) : 0.f;
+        float g = (live && p.alpha) ? log_gate(__bfloat162float(p.alpha[crow]), LOGITS) : 0.f;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const float t = __shfl_up_sync(0xffffffffu, g, o);
@@ -137,7 +140,7 @@ __global__ void __launch_bounds__(kPrepThreads, 2) k_tc_prep(const __grid_consta
     // row-wise work: 16 lanes cover one 256-byte row (chunk `ch` of 16 bytes each), 16 rows per pass
     const int ch = tid & 15, rsub = tid >> 4;
     const uint32_t coff = (ch >> 3) * 16384;
-    if (p.rqk) {
+    if (NORM) {
         // q^ = q / sqrt(|q|^2 + eps), k^ likewise, in place: everything below (and every later kernel, through
         // diag(gamma) Q^ and the 1/|k| written here) works on the normalised rows
         const size_t nrows = (size_t)p.BH * p.Tp;
@@ -714,17 +717,18 @@ cudaError_t tc_prep(const ChunkArgs& a) {
         return cudaErrorInvalidValue;
     PrepParams p{};
     p.T = s.T; p.Tp = Tp; p.H = s.H; p.N = Tp / kChunk; p.BH = s.B * s.H;
-    p.logits = a.logits ? 1 : 0;
     p.rqk = a.norm ? (float*)(a.ws + a.TL.rqk) : nullptr;
     p.beta = (const bf16*)a.beta; p.alpha = (const bf16*)a.alpha; p.lam = (const bf16*)a.lam;
     p.g = (float*)(a.ws + a.TL.g);
     p.Qg = (bf16*)(a.ws + a.TL.Qg); p.P = (bf16*)(a.ws + a.TL.P);
     p.Mt = a.save ? (bf16*)(a.ws + a.TL.Mt) : nullptr;
     p.status = (unsigned*)(a.ws + a.TL.status);
-    cudaError_t e = set_smem(k_tc_prep, kPrepSmem);
+    auto kern = a.norm ? (a.logits ? k_tc_prep<true, true> : k_tc_prep<true, false>)
+                       : (a.logits ? k_tc_prep<false, true> : k_tc_prep<false, false>);
+    cudaError_t e = set_smem(kern, kPrepSmem);
     if (e != cudaSuccess) return e;
     const int grid = s.B * s.H * (p.N / 2);
-    k_tc_prep<<<grid, kPrepThreads, kPrepSmem, a.stream>>>(mQ, mK, mV, mUt, mWt, p);
+    kern<<<grid, kPrepThreads, kPrepSmem, a.stream>>>(mQ, mK, mV, mUt, mWt, p);
     return cudaGetLastError();
 }
 

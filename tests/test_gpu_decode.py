@@ -162,7 +162,7 @@ def test_multi_token_step_null_coefficients_and_argument_errors():
     fake = 0x1000
     assert lib.qdelta_recurrent_steps(1, 0, 1, 64, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 0, None) == 1
     assert lib.qdelta_recurrent_steps(1, 2, 1, 96, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 0, None) == 2
-    assert lib.qdelta_recurrent_steps(1, 2, 1, 64, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 8, None) == 1
+    assert lib.qdelta_recurrent_steps(1, 2, 1, 64, 64, 0, fake, fake, fake, fake, None, None, fake, fake, 64, None) == 1
 
 
 def test_decode_steps_replayed_from_a_cuda_graph():
