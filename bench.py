@@ -74,10 +74,10 @@ def stage_bytes_per_token_head(dk, dv, C):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch: NOT measured by this run (a profiler cannot run inside the
-# timed program); constants from the ncu capture summarised in profiles/tc_kernels_dram_traffic_cfg2.md (full-size
+# timed program); constants from the ncu capture summarised in profiles/tc_kernels_fullsize_counters_cfg2.md (full-size
 # cfg2).  Other workloads: not captured.
-NCU_TRAFFIC_BYTES = {"cfg2": {"prep": 421.9e6, "chain_fwd": 532.8e6, "chain_bwd": 469.2e6, "chunk_bwd": 926.2e6}}
-NCU_TRAFFIC_SOURCE = "constant from profiles/tc_kernels_dram_traffic_cfg2.md (ncu, one launch each); not measured by this run"
+NCU_TRAFFIC_BYTES = {"cfg2": {"prep": 420.9e6, "chain_fwd": 533.6e6, "chain_bwd": 470.1e6, "chunk_bwd": 922.0e6}}
+NCU_TRAFFIC_SOURCE = "constant from profiles/tc_kernels_fullsize_counters_cfg2.md (ncu, one launch each); not measured by this run"
 # which pass of the path a kernel belongs to (its share of the algorithmic bytes of SURVEY section 8(d))
 STAGE_PASS = {"prep": "fwd", "chain_fwd": "fwd", "chain_bwd": "bwd", "chunk_bwd": "bwd"}
 
@@ -349,7 +349,7 @@ def run_ours(args, cfg):
     # nvidia-smi answers in ~0.1 s: keep the same step loop running (untimed) a little longer so that enough clock
     # samples are taken under this load
     t_probe = time.perf_counter()
-    while time.perf_counter() - t_probe < 1.0:
+    while not args.no_clock_probe and time.perf_counter() - t_probe < 1.0:
         for _ in range(20):
             step()
         torch.cuda.synchronize()
@@ -608,6 +608,8 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg3", "small"],
                     help="cfg2: headline (default); cfg3: long context; small: B=2 of cfg2 for profiler captures")
     ap.add_argument("--no-extras", action="store_true", help="skip the end-to-end, decode and CPU-baseline legs")
+    ap.add_argument("--no-clock-probe", action="store_true",
+                    help="do not keep the step loop running for clock samples (short runs for profiler captures)")
     args = ap.parse_args()
     from paper_2606_08804_b200 import inputs as gen
     cfg = gen.CONFIGS["cfg3" if args.workload == "cfg3" else "cfg2"]
