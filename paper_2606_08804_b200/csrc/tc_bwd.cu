@@ -873,14 +873,7 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     wait(&bm_5, ph);
     tc_fence_after();
     // The last epilogue: thread = d_k index i, its 16 tokens in groups of 8: dk and dq, transposed, into their staging
-    // tiles, and the column sums (over i, i.e. across the lanes) that d lambda, the decay gradient and, with NORM, the
-    // backward of the normalisation need.
-    // NORM: dx = r (dx^ - x^ <x^, dx^>).  r dx^ is staged here; the sums <k^, dk^> and <q^, dq^> go to scratch over the
-    // row sums, which are dead by now (the barrier makes sure their last readers are done); the second term is
-    // subtracted from the staged rows afterwards, once the sums are complete.
-    float (*sredN)[4][C] = reinterpret_cast<float (*)[4][C]>(&srow[0][0][0]);
-    float2* snf = reinterpret_cast<float2*>(&srow[2][0][0]);        // per token {<k^,dk^>/|k|, <q^,dq^>/|q|}
-    if (NORM) csync();
+    // tiles, and the column sums (over i, i.e. across the lanes) that d lambda and the decay gradient need.
     {
         const int i = l;
         unsigned char* stk = sm + oStDk + (i >> 6) * 8192;
@@ -904,21 +897,16 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                 const float4 cf = scf[t];
                 const float dxe = fmaf(cf.x, dx[e], v[e]);                                  // dX^T[i][t]
                 const float kh = cf.y * u[e];                                               // (K-> ^T applied to dh Delta^T)[i][t]
-                const float q1 = cf.z * z[e];
-                const float dkh = w[e] + kh + dxe;                                          // d k^ (d k without NORM)
-                const float dqh = q1 + y[e] + cf.w * dxe;                                   // d q^
-                const float kv = __bfloat162float(*reinterpret_cast<const bf16*>(kcol + sw128_off(t, i & 63)));
-                const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(t, i & 63)));
-                float2 rn = make_float2(1.f, 1.f);
-                if (NORM) rn = srn[t];
-                sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(rn.x * dkh));
-                sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(rn.y * dqh));
+                sts16(stk + sw128_off(t, i & 63), __float2bfloat16_rn(w[e] + kh + dxe));    // d k  (d k^ with NORM)
                 // <(K-> dh)_t, Delta_t> = gamma_C/gamma_t sum_i K[t][i] (dh Delta^T)[i][t], all of it in fp32
-                u[e] = kh * kv;
+                u[e] = kh * __bfloat162float(*reinterpret_cast<const bf16*>(kcol + sw128_off(t, i & 63)));
+                const float q1 = cf.z * z[e];
+                sts16(stq + sw128_off(t, i & 63), __float2bfloat16_rn(q1 + y[e] + cf.w * dxe));   // d q  (d q^ with NORM)
+                const float qv = __bfloat162float(*reinterpret_cast<const bf16*>(qcol + sw128_off(t, i & 63)));
                 z[e] = q1 * qv;
                 dx[e] = dxe * qv;
-                if (NORM) { w[e] = dkh * kv; y[e] = dqh * qv; }
             }
+            // column sums over the d_k index (across the lanes): d lambda, and the two that only the decay gradient needs
             if (want_dl) {
                 const float dls = col_reduce8(dx, lane);
                 if ((lane & 3) == 0) sred[1][wq][cb + col8_of_lane(lane)] = dls;
@@ -931,29 +919,20 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
                     sred[2][wq][col] = t1s;
                 }
             }
-            if (NORM) {
-                const float cks = col_reduce8(w, lane), cqs = col_reduce8(y, lane);
-                if ((lane & 3) == 0) {
-                    const int col = cb + col8_of_lane(lane);
-                    sredN[0][wq][col] = cks;
-                    sredN[1][wq][col] = cqs;
-                }
-            }
         }
     }
     if (NORM) {
-        csync();
-        if (tid < C) {
-            float ck = 0.f, cq = 0.f;
-#pragma unroll
-            for (int w4 = 0; w4 < 4; ++w4) { ck += sredN[0][w4][tid]; cq += sredN[1][w4][tid]; }
-            snf[tid] = make_float2(srn[tid].x * ck, srn[tid].y * cq);
-        }
-        csync();
-        // staged rows (token-major, 16 bytes at a time): dk_t -= (<k^,dk^>/|k|) k^_t, dq_t likewise
+        // Through the normalisation: dx = r (dx^ - x^ <x^, dx^>).  The staged tiles hold dk^ and dq^ token-major, like the
+        // K^ and Q^ tiles, so both steps are row-wise passes with 16-byte accesses: thread (row r, part) takes two
+        // 16-byte chunks of its row; first the partial row dot products (eight parts per row, summed through scratch
+        // over the dead row sums), then the corrected rows.
+        float (*part_k)[C] = reinterpret_cast<float (*)[C]>(&srow[0][0][0]);     // [8][C]
+        float (*part_q)[C] = reinterpret_cast<float (*)[C]>(&srow[2][0][0]);     // [8][C]
         constexpr int kPer = 16 / (kBwdCompute / 64);
+        static_assert(kBwdCompute / 64 == 8 && kNWG == 4, "scratch of the row dot products: 8 parts of 64 rows, twice");
         const int r = tid & 63, part = tid >> 6;
-        const float2 nf = snf[r];
+        csync();                             // the staged tiles are complete; the row sums have been consumed
+        float ck = 0.f, cq = 0.f;
 #pragma unroll
         for (int cc = 0; cc < kPer; ++cc) {
             const int ci = part * kPer + cc;
@@ -962,12 +941,33 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
             load8(sm + oStDk + off, a8);
             load8(sm + oK + off, x8);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) a8[e] = fmaf(-nf.x, x8[e], a8[e]);
+            for (int e = 0; e < 8; ++e) ck = fmaf(a8[e], x8[e], ck);
+            load8(sm + oStDq + off, a8);
+            load8(sm + oQ + off, x8);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) cq = fmaf(a8[e], x8[e], cq);
+        }
+        part_k[part][r] = ck;
+        part_q[part][r] = cq;
+        csync();
+        ck = 0.f; cq = 0.f;
+#pragma unroll
+        for (int pp = 0; pp < 8; ++pp) { ck += part_k[pp][r]; cq += part_q[pp][r]; }
+        const float2 rn = srn[r];            // {1/|k|, 1/|q|}
+#pragma unroll
+        for (int cc = 0; cc < kPer; ++cc) {
+            const int ci = part * kPer + cc;
+            const uint32_t off = (ci >> 3) * 8192 + sw128_chunk(r, ci & 7);
+            float a8[8], x8[8];
+            load8(sm + oStDk + off, a8);
+            load8(sm + oK + off, x8);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a8[e] = rn.x * fmaf(-ck, x8[e], a8[e]);
             sts128(sm + oStDk + off, pack8(a8));
             load8(sm + oStDq + off, a8);
             load8(sm + oQ + off, x8);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) a8[e] = fmaf(-nf.y, x8[e], a8[e]);
+            for (int e = 0; e < 8; ++e) a8[e] = rn.y * fmaf(-cq, x8[e], a8[e]);
             sts128(sm + oStDq + off, pack8(a8));
         }
     }
