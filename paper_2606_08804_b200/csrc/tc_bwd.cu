@@ -301,6 +301,7 @@ __global__ void __launch_bounds__(kChainThreads) k_tc_chain_bwd(const __grid_con
 struct ChunkBwdParams {
     int logits;                // beta, alpha, lambda are logits of sigmoid gates; their gradients are taken w.r.t. the logits
     const float* rqk;          // QD_NORM_QK: 1/|q_t| per workspace row, then (BH*Tp further) 1/|k_t|
+    int group;                 // GROUPED instances: sequences per group of work items
     int T, Tp, H, N, BH, total;   // T tokens per sequence, Tp = 64 N rows per sequence in the workspace; total = BH*N chunks
     const bf16 *beta, *alpha, *lam;
     const float* g;
@@ -348,7 +349,7 @@ __device__ __forceinline__ void ld8(uint32_t taddr, float* v) { tmem_ld8(taddr, 
 // left in the workspace; dq and dk are taken through the normalisation, dx = r (dx^ - x^ <x^, dx^>), which needs the
 // row sums <x^, dx^> before anything can be stored: the last epilogue then runs twice, once for the sums and once
 // for the stores.
-template <bool HAS_LAM, bool HAS_ALPHA, bool NORM>
+template <bool HAS_LAM, bool HAS_ALPHA, bool NORM, bool GROUPED>
 __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_constant__ CUtensorMap mapQ,
                                                               const __grid_constant__ CUtensorMap mapK,
                                                               const __grid_constant__ CUtensorMap mapV,
@@ -401,9 +402,24 @@ __global__ void __launch_bounds__(kBwdThreads) k_tc_chunk_bwd(const __grid_const
     // The tiles of a chunk arrive in two groups.  "early": V, dO, M^T, P -- their regions are dead once the
     // last products of the previous chunk have finished; "late": Q, Delta^T, dDelta^T, h^T, dh^T -- regions
     // that the previous chunk uses up to its end (staging tiles of the stores, scratch of the reductions).
-    // Work item `ch` is chunk n_ of sequence bh_, sequence-major.  (Chunk-major numbering, which would take the tiles the
-    // reverse chain wrote last first, was measured 10 % slower.)
-    auto item = [&](int ch, int& n_, int& bh_) { bh_ = ch / p.N; n_ = ch - bh_ * p.N; };
+    // Work item `ch` is chunk n_ of sequence bh_.  GROUPED = false: sequence-major numbering.  GROUPED = true: items are
+    // numbered in groups of p.group sequences, chunk-major inside a group, so that at any time the CTAs of the grid work
+    // on a few chunk indices of p.group sequences instead of on ~148 consecutive chunks of one long sequence.  Measured,
+    // sequence-major against groups of 32: 0.330 / 0.316 ms on 32 sequences of 128 chunks, 0.347 / 0.320 on 16 of 256,
+    // 1.47 / 1.18 on 32 of 512, no gain on 128 sequences of 32 chunks; all sequences at a time (chunk-major) was the
+    // slowest there.  Compile-time, because the kernel's code generation is at a knife's edge: the grouped arithmetic
+    // compiled into the sequence-major path cost it 3.5 %, as a non-inlined function 14 %.
+    auto item = [&](int ch, int& n_, int& bh_) {
+        if (GROUPED) {
+            const int per = p.group * p.N, grp = ch / per, r = ch - grp * per;
+            const int g0 = grp * p.group, gs = min(p.group, p.BH - g0);       // the last group may be smaller
+            n_ = r / gs;
+            bh_ = g0 + r - n_ * gs;
+        } else {
+            bh_ = ch / p.N;
+            n_ = ch - bh_ * p.N;
+        }
+    };
     auto issue_early = [&](int ch) {
         int n_, bh_; item(ch, n_, bh_);
         const int b_ = bh_ / p.H, hh_ = bh_ % p.H;
@@ -1080,11 +1096,20 @@ cudaError_t tc_chunk_bwd(const ChunkArgs& a) {
     p.status = (unsigned*)(a.ws + a.TL.status);
     // the instance without lambda / without the forget gate needs the input AND its gradient to be absent
     const bool lam = a.lam || a.dlam, alpha = a.alpha || a.dalpha;
-    auto kern = lam ? (alpha ? k_tc_chunk_bwd<true, true, false> : k_tc_chunk_bwd<true, false, false>)
-                    : (alpha ? k_tc_chunk_bwd<false, true, false> : k_tc_chunk_bwd<false, false, false>);
-    if (a.norm)
-        kern = lam ? (alpha ? k_tc_chunk_bwd<true, true, true> : k_tc_chunk_bwd<true, false, true>)
-                   : (alpha ? k_tc_chunk_bwd<false, true, true> : k_tc_chunk_bwd<false, false, true>);
+    const bool grouped = N >= 64;         // long sequences: work items in groups of 32 sequences (see the kernel)
+    p.group = 32;
+    using Kern = decltype(&k_tc_chunk_bwd<true, true, false, false>);
+    static const Kern table[16] = {
+        k_tc_chunk_bwd<false, false, false, false>, k_tc_chunk_bwd<false, false, false, true>,
+        k_tc_chunk_bwd<false, false, true, false>,  k_tc_chunk_bwd<false, false, true, true>,
+        k_tc_chunk_bwd<false, true, false, false>,  k_tc_chunk_bwd<false, true, false, true>,
+        k_tc_chunk_bwd<false, true, true, false>,   k_tc_chunk_bwd<false, true, true, true>,
+        k_tc_chunk_bwd<true, false, false, false>,  k_tc_chunk_bwd<true, false, false, true>,
+        k_tc_chunk_bwd<true, false, true, false>,   k_tc_chunk_bwd<true, false, true, true>,
+        k_tc_chunk_bwd<true, true, false, false>,   k_tc_chunk_bwd<true, true, false, true>,
+        k_tc_chunk_bwd<true, true, true, false>,    k_tc_chunk_bwd<true, true, true, true>,
+    };
+    const Kern kern = table[(lam ? 8 : 0) + (alpha ? 4 : 0) + (a.norm ? 2 : 0) + (grouped ? 1 : 0)];
     cudaError_t e = set_smem(kern, kBwdSmem);
     if (e != cudaSuccess) return e;
     // persistent: one CTA per SM walks the work items with stride gridDim.x
