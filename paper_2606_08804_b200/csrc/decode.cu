@@ -85,8 +85,8 @@ __global__ void __launch_bounds__(NT) k_decode(int dv, const IO* __restrict__ q,
 // for S tokens instead of S of each.  Token tensors are token-major [B, S, H, d] like those of the chunkwise calls.  The
 // arithmetic of one token is exactly that of k_decode, in the same order, so S tokens here give bit-identical results to
 // S single-token calls.
-template <typename IO, int DK, int DVS, int NT>
-__global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, int logits, int norm, const IO* __restrict__ q, const IO* __restrict__ k,
+template <typename IO, int DK, int DVS, int NT, bool LOGITS, bool NORM>      // the two pre-processing flags, compile-time
+__global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, const IO* __restrict__ q, const IO* __restrict__ k,
                                                      const IO* __restrict__ v, const IO* __restrict__ beta,
                                                      const IO* __restrict__ alpha, const IO* __restrict__ lam,
                                                      float* __restrict__ state, IO* __restrict__ o) {
@@ -108,11 +108,11 @@ __global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, int l
 
     for (int s = 0; s < S; ++s) {
         const size_t row = ((size_t)b * S + s) * H + hh;        // token row of this head in the [B, S, H] view
-        const float be = gate(ld(beta, row), logits);
-        const float al = alpha ? gate(ld(alpha, row), logits) : 1.f;
-        const float la = lam ? gate(ld(lam, row), logits) : 0.f;
+        const float be = gate(ld(beta, row), LOGITS);
+        const float al = alpha ? gate(ld(alpha, row), LOGITS) : 1.f;
+        const float la = lam ? gate(ld(lam, row), LOGITS) : 0.f;
         float kq = 0.f;
-        if (norm) {
+        if (NORM) {
             // q^ = q / sqrt(|q|^2 + eps), k^ likewise: three block-wide sums, then the token's arrays are rescaled
             float ssq = 0.f, ssk = 0.f;
             for (int i = tid; i < DK; i += NT) {
@@ -192,9 +192,10 @@ cudaError_t launch_multi(int B, int S, int H, int dv, const void* q, const void*
                          cudaStream_t stream) {
     constexpr int DVS = 64, NT = 128;
     dim3 grid((unsigned)(dv / DVS) * (unsigned)(B * H));
-    k_decode_multi<IO, DK, DVS, NT><<<grid, NT, 0, stream>>>(S, H, dv, logits ? 1 : 0, norm ? 1 : 0, (const IO*)q, (const IO*)k, (const IO*)v,
-                                                             (const IO*)beta, (const IO*)alpha, (const IO*)lam,
-                                                             state, (IO*)o);
+    auto kern = logits ? (norm ? k_decode_multi<IO, DK, DVS, NT, true, true> : k_decode_multi<IO, DK, DVS, NT, true, false>)
+                       : (norm ? k_decode_multi<IO, DK, DVS, NT, false, true> : k_decode_multi<IO, DK, DVS, NT, false, false>);
+    kern<<<grid, NT, 0, stream>>>(S, H, dv, (const IO*)q, (const IO*)k, (const IO*)v, (const IO*)beta, (const IO*)alpha,
+                                  (const IO*)lam, state, (IO*)o);
     return cudaGetLastError();
 }
 
