@@ -418,3 +418,52 @@ def test_in_kernel_l2_normalisation(dtype, T, logits, drop):
     roS, rhS = orc.forward_fused(cut(d["q"]), cut(d["k"]), cut(d["v"]), cut(d["beta"]), cut(d["alpha"]), cut(d["lam"]), d["h0"],
                                  logits=logits, norm_qk=True)
     assert gu.rel_err(od, roS) <= gu.TOL[dtype] and gu.rel_err(state, rhS) <= gu.TOL[dtype]
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_random_shapes_flags_and_absent_inputs(case):
+    # seeded sweep over what the entry points accept: any T, either path, absent optional inputs, both pre-processing
+    # flags, backward with and without the forward's workspace -- each case against the oracle
+    from oracle import recurrence as orc
+    from paper_2606_08804_b200 import binding as qd
+    r = np.random.default_rng(1000 + case)
+    tc = case % 2 == 0                                   # even cases: bf16 d = 128 (tensor cores); odd: fp32 path shapes
+    if tc:
+        base, dk, dv, dtype = gen.CONFIGS["cfg2"], 128, 128, "bf16"
+    else:
+        dk, dv = [(64, 64), (128, 64), (64, 128)][case % 3]
+        dtype = "f32" if case % 4 == 1 else "bf16"
+        base = replace(gen.CONFIGS["cfg0"], h0=True, backward=True, dtype=dtype)
+    B, H = int(r.integers(1, 4)), int(r.integers(1, 5))
+    T = int(r.integers(1, 400))
+    regime = gen.REGIMES[int(r.integers(0, len(gen.REGIMES)))]
+    cfg = replace(base, B=B, H=H, T=T, dk=dk, dv=dv, regime=regime, seed=2000 + case)
+    d = gen.make_chunk_inputs(cfg)
+    logits, norm = bool(r.integers(0, 2)), bool(r.integers(0, 2))
+    rnd = (lambda x: gen.round_bf16(x.astype(np.float32))) if dtype == "bf16" else (lambda x: x.astype(np.float32))
+    if norm:
+        d["q"] = rnd(d["q"] * np.exp(r.normal(0, 0.7, d["q"].shape[:-1] + (1,))))
+        d["k"] = rnd(d["k"] * np.exp(r.normal(0, 0.7, d["k"].shape[:-1] + (1,))))
+    if logits:
+        shp = (B, T, H)
+        d["beta"], d["alpha"], d["lam"] = rnd(r.normal(0, 1.5, shp)), rnd(r.normal(3, 1.5, shp)), rnd(r.normal(-0.8, 1, shp))
+    for n in ("alpha", "lam", "h0", "dhT"):
+        if r.random() < 0.25:
+            d[n] = None
+    t = gu.dev_inputs(d, cfg.dtype)
+    assert qd.chunk_path(qd.make_shape(t["q"], t["v"], 64)) == ("tensor_core" if tc else "fp32")
+    ro, rh = orc.forward_fused(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"], logits=logits, norm_qk=norm)
+    ref = orc.backward_fused(d["q"], d["k"], d["v"], d["beta"], d["alpha"], d["lam"], d["h0"], d["dO"], d["dhT"],
+                             logits=logits, norm_qk=norm)
+    lab = _label(cfg, " sweep %d logits=%d norm=%d absent=%s" % (case, logits, norm, [n for n in ("alpha", "lam", "h0", "dhT") if d[n] is None]))
+    for reuse in (False, True):
+        o, hT, ws = qd.chunk_fwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], save_for_bwd=reuse,
+                                 logits=logits, norm_qk=norm)
+        g = qd.chunk_bwd(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"], t["dO"], t["dhT"],
+                         workspace=ws if reuse else None, reuse_fwd=reuse, logits=logits, norm_qk=norm)
+        torch.cuda.synchronize()
+        gu.check(lab, "o", o, ro, cfg.dtype)
+        gu.check(lab, "hT", hT, rh, cfg.dtype, state=True)
+        for n in ("dq", "dk", "dv", "dbeta", "dalpha", "dlam", "dh0"):
+            if g.get(n) is not None:
+                gu.check(lab, n, g[n], ref[n], cfg.dtype, state=(n == "dh0"))
