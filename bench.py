@@ -76,7 +76,7 @@ def stage_bytes_per_token_head(dk, dv, C):
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch: NOT measured by this run (a profiler cannot run inside the
 # timed program); constants from the ncu capture summarised in profiles/tc_kernels_fullsize_counters_cfg2.md (full-size
 # cfg2).  Other workloads: not captured.
-NCU_TRAFFIC_BYTES = {"cfg2": {"prep": 420.9e6, "chain_fwd": 533.6e6, "chain_bwd": 470.1e6, "chunk_bwd": 922.0e6}}
+NCU_TRAFFIC_BYTES = {"cfg2": {"prep": 421.7e6, "chain_fwd": 532.6e6, "chain_bwd": 470.2e6, "chunk_bwd": 922.1e6}}
 NCU_TRAFFIC_SOURCE = "constant from profiles/tc_kernels_fullsize_counters_cfg2.md (ncu, one launch each); not measured by this run"
 # which pass of the path a kernel belongs to (its share of the algorithmic bytes of SURVEY section 8(d))
 STAGE_PASS = {"prep": "fwd", "chain_fwd": "fwd", "chain_bwd": "bwd", "chunk_bwd": "bwd"}
