@@ -467,3 +467,28 @@ def test_random_shapes_flags_and_absent_inputs(case):
         for n in ("dq", "dk", "dv", "dbeta", "dalpha", "dlam", "dh0"):
             if g.get(n) is not None:
                 gu.check(lab, n, g[n], ref[n], cfg.dtype, state=(n == "dh0"))
+
+
+def test_autograd_front_end():
+    # torch.autograd wrapper: gradients of a scalar loss on o and hT equal the oracle's reverse pass
+    from paper_2606_08804_b200.autograd import qdelta_chunk
+    cfg = replace(gen.CONFIGS["cfg2"], B=2, H=2, T=200, regime="alpha_slow", seed=107)
+    d = gen.make_chunk_inputs(cfg)
+    t = gu.dev_inputs(d, cfg.dtype)
+    leaves = {n: t[n].clone().requires_grad_(True) for n in ("q", "k", "v", "beta", "alpha", "lam", "h0")}
+    o, hT = qdelta_chunk(**leaves)
+    loss = (o.float() * t["dO"].float()).sum() + (hT * t["dhT"]).sum()
+    loss.backward()
+    torch.cuda.synchronize()
+    ro, rh = gu.oracle_fwd(d)
+    ref = gu.oracle_bwd(d)
+    lab = _label(cfg, " autograd")
+    gu.check(lab, "o", o, ro, cfg.dtype)
+    gu.check(lab, "hT", hT, rh, cfg.dtype, state=True)
+    for n, gn in (("q", "dq"), ("k", "dk"), ("v", "dv"), ("beta", "dbeta"), ("alpha", "dalpha"), ("lam", "dlam"), ("h0", "dh0")):
+        # coefficient gradients come back in the coefficients' dtype (bf16): one more rounding than the raw fp32 ones
+        gu.check(lab, gn, leaves[n].grad, ref[gn], cfg.dtype, state=(n == "h0"))
+    # without any input requiring grad the forward does not keep a backward-sized workspace
+    with torch.no_grad():
+        o2, _ = qdelta_chunk(t["q"], t["k"], t["v"], t["beta"], t["alpha"], t["lam"], t["h0"])
+    assert torch.equal(o2, o.detach())
