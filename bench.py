@@ -561,6 +561,24 @@ def bench_decode(args, qd, gen, torch, pk, pk_kind):
         bytesS = nstates * (2 * cfg.dk * cfg.dv * 4 + S * (2 * (2 * cfg.dk + cfg.dv) + 6 + 2 * cfg.dv))
         multi["S=%d" % S] = {"us_per_call": msS * 1e3, "tokens_per_s": cfg.B * S / (msS * 1e-3),
                              "achieved_gbs": bytesS / (msS * 1e-3) / 1e9, "frac": bytesS / (msS * 1e-3) / 1e9 / pk["hbm_gbs"]}
+    # reduced-precision option: the same step with the state stored in bf16 (QD_STATE_BF16), one token per call
+    st16 = state.to(bf)
+    tk1 = {n: t[:, :1].contiguous() for n, t in tk.items()}          # one token of the last multi-token set
+    o1 = torch.empty((cfg.B, 1, cfg.H, cfg.dv), dtype=bf, device="cuda")
+    for _ in range(5):
+        qd.recurrent_steps(tk1["q"], tk1["k"], tk1["v"], tk1["beta"], tk1["alpha"], tk1["lam"], st16, o1)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(nsteps):
+        qd.recurrent_steps(tk1["q"], tk1["k"], tk1["v"], tk1["beta"], tk1["alpha"], tk1["lam"], st16, o1)
+    e1.record()
+    torch.cuda.synchronize()
+    ms16 = e0.elapsed_time(e1) / nsteps
+    bytes16 = nstates * (2 * cfg.dk * cfg.dv * 2 + 2 * (2 * cfg.dk + cfg.dv) + 6 + 2 * cfg.dv)
+    bf16_state = {"us_per_step": ms16 * 1e3, "tokens_per_s": cfg.B / (ms16 * 1e-3), "achieved_gbs": bytes16 / (ms16 * 1e-3) / 1e9,
+                  "frac": bytes16 / (ms16 * 1e-3) / 1e9 / pk["hbm_gbs"],
+                  "note": "reduced-precision OPTION (state rounded to bf16 once per call); not the configuration's fp32 state"}
+    del st16
     # the same loop replayed from one CUDA graph of `pool` steps (no per-step launch cost on the host)
     graph_us = None
     try:
@@ -588,7 +606,7 @@ def bench_decode(args, qd, gen, torch, pk, pk_kind):
         graph_us = "unavailable: %s" % type(exc).__name__
     return {"workload": "cfg4: batch=%d H=%d dk=%d dv=%d fp32 state in place, bf16 tokens" % (cfg.B, cfg.H, cfg.dk, cfg.dv),
             "steps": nsteps, "us_per_step": ms * 1e3, "tokens_per_s": cfg.B / (ms * 1e-3), "multi_token": multi,
-            "us_per_step_cuda_graph": graph_us,
+            "us_per_step_cuda_graph": graph_us, "bf16_state_option": bf16_state,
             "roofline": {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                          "frac": gbs / pk["hbm_gbs"], "peak_kind": "of " + pk_kind,
                          "algorithmic_bytes_per_launch": bytes_step, "state_larger_than_l2": True}}

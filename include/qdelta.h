@@ -70,11 +70,17 @@ enum {
                                  logits z of sigmoid gates (Appendix B: lambda = sigmoid(W h + b)); the kernels use
                                  sigmoid(z), computed in fp32, and the backward writes dbeta, dalpha, dlambda as
                                  derivatives with respect to the logits.  NULL alpha / lambda still mean 1 / 0. */
-    QD_NORM_QK = 8            /* fwd, bwd, qdelta_recurrent_steps: q and k are given un-normalised; the kernels use
+    QD_NORM_QK = 8,           /* fwd, bwd, qdelta_recurrent_steps: q and k are given un-normalised; the kernels use
                                  q / sqrt(|q|^2 + 1e-6) and k / sqrt(|k|^2 + 1e-6), per token and head (the L2
                                  normalisation that otherwise precedes the call), and the backward writes dq, dk as
                                  derivatives with respect to the un-normalised q, k.  A QD_BWD_REUSE_FWD backward must
                                  carry the same setting as its forward. */
+    QD_STATE_BF16 = 16        /* qdelta_recurrent_steps only: `state` points to bf16 [B,H,dk,dv] instead of fp32 (half the
+                                 bytes of a decode step).  The state is widened to fp32 when read, the S tokens of the
+                                 call are applied in fp32, and it is rounded to bf16 once when written back.  This is
+                                 a reduced-precision OPTION, not the method's fp32 state: every call adds a rounding of
+                                 relative size 2^-9 to the state, which the forget gate damps by alpha per token; with
+                                 alpha == 1 (no forgetting) the error grows like sqrt(calls) * 2^-9. */
 };
 
 typedef struct {
@@ -143,14 +149,16 @@ int qdelta_recurrent_step(int B, int H, int dk, int dv, int dtype,
  * state is read once and written once for all S tokens instead of once per token.  Token tensors are token-major like
  * those of the chunkwise calls:
  *     q,k [B,S,H,dk]   v,o [B,S,H,dv]   beta/alpha/lambda [B,S,H]   (alpha, lambda may be NULL)
- *     state [B,H,dk,dv] fp32, UPDATED IN PLACE to the state after the S-th token;  o_s is read out after token s.
- * The result is bit-identical to S calls of qdelta_recurrent_step.  flags: 0, QD_COEF_LOGITS, QD_NORM_QK.  S >= 1; for long runs of tokens (a prompt) use
+ *     state [B,H,dk,dv] fp32 (bf16 with QD_STATE_BF16), UPDATED IN PLACE to the state after the S-th token;
+ *     o_s is read out after token s.
+ * With an fp32 state the result is bit-identical to S calls of qdelta_recurrent_step.
+ * flags: any of QD_COEF_LOGITS, QD_NORM_QK, QD_STATE_BF16.  S >= 1; for long runs of tokens (a prompt) use
  * qdelta_chunk_fwd with h0 / hT, which runs on the tensor cores.  Needs no workspace.
  */
 int qdelta_recurrent_steps(int B, int S, int H, int dk, int dv, int dtype,
                            const void *q, const void *k, const void *v,
                            const void *beta, const void *alpha, const void *lambda,
-                           float *state, void *o, unsigned flags, qd_stream stream);
+                           void *state, void *o, unsigned flags, qd_stream stream);
 
 /* Copies the device status word of `workspace` to *status_out (a qd_status) with a blocking
  * 4-byte device-to-host copy on `stream`.  Returns QD_OK or QD_ERR_CUDA / QD_ERR_INVALID_ARG. */

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libqdelta.so")
 
 QD_F32, QD_BF16 = 0, 1
-QD_FWD_SAVE_FOR_BWD, QD_BWD_REUSE_FWD, QD_COEF_LOGITS, QD_NORM_QK = 1, 2, 4, 8
+QD_FWD_SAVE_FOR_BWD, QD_BWD_REUSE_FWD, QD_COEF_LOGITS, QD_NORM_QK, QD_STATE_BF16 = 1, 2, 4, 8, 16
 
 EXPORTS = ("qdelta_chunk_workspace_bytes", "qdelta_chunk_fwd", "qdelta_chunk_bwd",
            "qdelta_recurrent_step", "qdelta_workspace_status", "qdelta_status_string",
@@ -265,17 +265,22 @@ def recurrent_step(q, k, v, beta, alpha, lam, state, o=None):
 
 def recurrent_steps(q, k, v, beta, alpha, lam, state, o=None, logits=False, norm_qk=False):
     """S decode tokens per call: q,k [B,S,H,dk], v [B,S,H,dv], coefficients [B,S,H]; `state` [B,H,dk,dv] fp32 is
-    updated in place to the state after the last token.  Returns o [B,S,H,dv]."""
+    updated in place to the state after the last token.  Returns o [B,S,H,dv].  A bf16 `state` selects the
+    reduced-precision state option (QD_STATE_BF16)."""
     lib = load()
     B, S, H, dk = q.shape
     dv = v.shape[-1]
     dt = q.dtype
+    if state.dtype not in (torch.float32, torch.bfloat16):
+        raise QdeltaError("state must be fp32, or bf16 for the reduced-precision state option")
+    state_bf16 = state.dtype == torch.bfloat16
     if o is None:
         o = torch.empty((B, S, H, dv), dtype=dt, device=q.device)
     rc = lib.qdelta_recurrent_steps(
         B, S, H, dk, dv, _dtype_code(q), _ptr(q, dt, (B, S, H, dk), "q"), _ptr(k, dt, (B, S, H, dk), "k"),
         _ptr(v, dt, (B, S, H, dv), "v"), _ptr(beta, dt, (B, S, H), "beta"), _ptr(alpha, dt, (B, S, H), "alpha"),
-        _ptr(lam, dt, (B, S, H), "lam"), _ptr(state, torch.float32, (B, H, dk, dv), "state"),
-        _ptr(o, dt, (B, S, H, dv), "o"), (QD_COEF_LOGITS if logits else 0) | (QD_NORM_QK if norm_qk else 0), _stream())
+        _ptr(lam, dt, (B, S, H), "lam"), _ptr(state, None, (B, H, dk, dv), "state"),
+        _ptr(o, dt, (B, S, H, dv), "o"),
+        (QD_COEF_LOGITS if logits else 0) | (QD_NORM_QK if norm_qk else 0) | (QD_STATE_BF16 if state_bf16 else 0), _stream())
     _check(rc, "qdelta_recurrent_steps")
     return o

@@ -222,10 +222,10 @@ int qdelta_recurrent_step(int B, int H, int dk, int dv, int dtype, const void* q
 }
 
 int qdelta_recurrent_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
-                           const void* beta, const void* alpha, const void* lambda, float* state, void* o,
+                           const void* beta, const void* alpha, const void* lambda, void* state, void* o,
                            unsigned flags, qd_stream stream) {
     if (B <= 0 || H <= 0 || S <= 0) return QD_ERR_INVALID_ARG;
-    if (flags & ~(unsigned)(QD_COEF_LOGITS | QD_NORM_QK)) return QD_ERR_INVALID_ARG;
+    if (flags & ~(unsigned)(QD_COEF_LOGITS | QD_NORM_QK | QD_STATE_BF16)) return QD_ERR_INVALID_ARG;
     if (dtype != QD_F32 && dtype != QD_BF16) return QD_ERR_UNSUPPORTED;
     if ((dk != 64 && dk != 128) || (dv != 64 && dv != 128)) return QD_ERR_UNSUPPORTED;
     if (!q || !k || !v || !beta || !state || !o) return QD_ERR_INVALID_ARG;
@@ -238,7 +238,8 @@ int qdelta_recurrent_steps(int B, int S, int H, int dk, int dv, int dtype, const
         if (p && ((uintptr_t)p & (dtype == QD_BF16 ? 1 : 3))) return QD_ERR_INVALID_ARG;
     if (timed(ST_DECODE, (cudaStream_t)stream, [&] {
             return decode_steps(B, S, H, dk, dv, dtype, q, k, v, beta, alpha, lambda, state, o,
-                                (flags & QD_COEF_LOGITS) != 0, (flags & QD_NORM_QK) != 0, (cudaStream_t)stream);
+                                (flags & QD_COEF_LOGITS) != 0, (flags & QD_NORM_QK) != 0, (flags & QD_STATE_BF16) != 0,
+                                (cudaStream_t)stream);
         }) != cudaSuccess)
         return QD_ERR_CUDA;
     return QD_OK;

@@ -85,11 +85,13 @@ __global__ void __launch_bounds__(NT) k_decode(int dv, const IO* __restrict__ q,
 // for S tokens instead of S of each.  Token tensors are token-major [B, S, H, d] like those of the chunkwise calls.  The
 // arithmetic of one token is exactly that of k_decode, in the same order, so S tokens here give bit-identical results to
 // S single-token calls.
-template <typename IO, int DK, int DVS, int NT, bool LOGITS, bool NORM>      // the two pre-processing flags, compile-time
+// SB16 (QD_STATE_BF16): the state is STORED in bf16 (half the bytes of the step); it is widened to fp32 when read, all S
+// tokens of the call are applied in fp32, and it is rounded to bf16 once, when written back.
+template <typename IO, int DK, int DVS, int NT, bool LOGITS, bool NORM, bool SB16>      // flags, compile-time
 __global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, const IO* __restrict__ q, const IO* __restrict__ k,
                                                      const IO* __restrict__ v, const IO* __restrict__ beta,
                                                      const IO* __restrict__ alpha, const IO* __restrict__ lam,
-                                                     float* __restrict__ state, IO* __restrict__ o) {
+                                                     void* __restrict__ state_, IO* __restrict__ o) {
     constexpr int C4 = DVS / 4, RP = NT / C4, NP = DK / RP;
     static_assert(NT % C4 == 0 && DK % RP == 0, "bad decode tiling");
     __shared__ float sx[DK], sq[DK], sk[DK];
@@ -100,11 +102,22 @@ __global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, const
     const int b = bh / H, hh = bh % H;
     const int c4 = tid % C4, rg = tid / C4;
 
-    float4* base = reinterpret_cast<float4*>(state + (size_t)bh * DK * dv + j0) + c4;
+    // four consecutive d_v columns per thread and row: 16 bytes of an fp32 state, 8 bytes of a bf16 state
+    float4* base = reinterpret_cast<float4*>(static_cast<float*>(state_) + (size_t)bh * DK * dv + j0) + c4;
+    uint2* base16 = reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(state_) + (size_t)bh * DK * dv + j0) + c4;
     const int rstride = dv / 4;
     float4 h[NP];
 #pragma unroll
-    for (int pz = 0; pz < NP; ++pz) h[pz] = __ldcs(base + (size_t)(pz * RP + rg) * rstride);
+    for (int pz = 0; pz < NP; ++pz) {
+        if (SB16) {
+            const uint2 u = __ldcs(base16 + (size_t)(pz * RP + rg) * rstride);
+            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.x));
+            const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.y));
+            h[pz] = make_float4(lo.x, lo.y, hi.x, hi.y);
+        } else {
+            h[pz] = __ldcs(base + (size_t)(pz * RP + rg) * rstride);
+        }
+    }
 
     for (int s = 0; s < S; ++s) {
         const size_t row = ((size_t)b * S + s) * H + hh;        // token row of this head in the [B, S, H] view
@@ -183,17 +196,30 @@ __global__ void __launch_bounds__(NT) k_decode_multi(int S, int H, int dv, const
         __syncthreads();                 // the token's shared arrays are rewritten by the next one
     }
 #pragma unroll
-    for (int pz = 0; pz < NP; ++pz) __stcs(base + (size_t)(pz * RP + rg) * rstride, h[pz]);
+    for (int pz = 0; pz < NP; ++pz) {
+        if (SB16) {
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(h[pz].x, h[pz].y), hi = __floats2bfloat162_rn(h[pz].z, h[pz].w);
+            uint2 u;
+            u.x = *reinterpret_cast<const unsigned*>(&lo);
+            u.y = *reinterpret_cast<const unsigned*>(&hi);
+            __stcs(base16 + (size_t)(pz * RP + rg) * rstride, u);
+        } else {
+            __stcs(base + (size_t)(pz * RP + rg) * rstride, h[pz]);
+        }
+    }
 }
 
 template <typename IO, int DK>
 cudaError_t launch_multi(int B, int S, int H, int dv, const void* q, const void* k, const void* v, const void* beta,
-                         const void* alpha, const void* lam, float* state, void* o, bool logits, bool norm,
+                         const void* alpha, const void* lam, void* state, void* o, bool logits, bool norm, bool sb16,
                          cudaStream_t stream) {
     constexpr int DVS = 64, NT = 128;
     dim3 grid((unsigned)(dv / DVS) * (unsigned)(B * H));
-    auto kern = logits ? (norm ? k_decode_multi<IO, DK, DVS, NT, true, true> : k_decode_multi<IO, DK, DVS, NT, true, false>)
-                       : (norm ? k_decode_multi<IO, DK, DVS, NT, false, true> : k_decode_multi<IO, DK, DVS, NT, false, false>);
+    auto kern = logits ? (norm ? k_decode_multi<IO, DK, DVS, NT, true, true, false> : k_decode_multi<IO, DK, DVS, NT, true, false, false>)
+                       : (norm ? k_decode_multi<IO, DK, DVS, NT, false, true, false> : k_decode_multi<IO, DK, DVS, NT, false, false, false>);
+    if (sb16)
+        kern = logits ? (norm ? k_decode_multi<IO, DK, DVS, NT, true, true, true> : k_decode_multi<IO, DK, DVS, NT, true, false, true>)
+                      : (norm ? k_decode_multi<IO, DK, DVS, NT, false, true, true> : k_decode_multi<IO, DK, DVS, NT, false, false, true>);
     kern<<<grid, NT, 0, stream>>>(S, H, dv, (const IO*)q, (const IO*)k, (const IO*)v, (const IO*)beta, (const IO*)alpha,
                                   (const IO*)lam, state, (IO*)o);
     return cudaGetLastError();
@@ -224,14 +250,14 @@ cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const 
 }
 
 cudaError_t decode_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
-                         const void* beta, const void* alpha, const void* lam, float* state, void* o,
-                         bool logits, bool norm, cudaStream_t stream) {
+                         const void* beta, const void* alpha, const void* lam, void* state, void* o,
+                         bool logits, bool norm, bool sb16, cudaStream_t stream) {
     if (dtype == QD_BF16) {
-        if (dk == 128) return launch_multi<__nv_bfloat16, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, stream);
-        return launch_multi<__nv_bfloat16, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, stream);
+        if (dk == 128) return launch_multi<__nv_bfloat16, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, sb16, stream);
+        return launch_multi<__nv_bfloat16, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, sb16, stream);
     }
-    if (dk == 128) return launch_multi<float, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, stream);
-    return launch_multi<float, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, stream);
+    if (dk == 128) return launch_multi<float, 128>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, sb16, stream);
+    return launch_multi<float, 64>(B, S, H, dv, q, k, v, beta, alpha, lam, state, o, logits, norm, sb16, stream);
 }
 
 }  // namespace qd

@@ -120,8 +120,8 @@ cudaError_t decode_step(int BH, int dk, int dv, int dtype, const void* q, const 
                         cudaStream_t stream);
 
 cudaError_t decode_steps(int B, int S, int H, int dk, int dv, int dtype, const void* q, const void* k, const void* v,
-                         const void* beta, const void* alpha, const void* lam, float* state, void* o,
-                         bool logits, bool norm, cudaStream_t stream);
+                         const void* beta, const void* alpha, const void* lam, void* state, void* o,
+                         bool logits, bool norm, bool state_bf16, cudaStream_t stream);
 
 // ---- in-kernel L2 normalisation of q and k (QD_NORM_QK) ------------------------------------------------
 // x^ = x / sqrt(sum x^2 + kNormEps), per token and head.  Its backward: dx = r (dx^ - x^ <x^, dx^>), r = 1/sqrt(sum x^2 + eps).

@@ -203,3 +203,33 @@ def test_decode_steps_replayed_from_a_cuda_graph():
         assert torch.equal(state, eager_state)
         for a, b in zip(outs, eager_outs):
             assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("S", [1, 4])
+def test_decode_with_bf16_state_storage(S):
+    # QD_STATE_BF16: the state lives in bf16 between calls (fp32 inside a call).  Checked against the oracle run with
+    # exactly that rounding between calls, and -- in the forgetful regime of the decode configuration, where the gate
+    # damps the rounding -- against the plain fp64 oracle within the bf16 bar.
+    from paper_2606_08804_b200 import binding as qd
+    cfg = replace(gen.CONFIGS["cfg4"], B=3, H=4)
+    calls = 200 // S
+    s0 = gen.round_bf16(gen.make_decode_state(cfg))
+    state = gu.Guarded((cfg.B, cfg.H, cfg.dk, cfg.dv), torch.bfloat16, fill=torch.from_numpy(s0).cuda().to(torch.bfloat16))
+    ref_r = s0.astype(np.float64)            # oracle state, rounded to bf16 after every call
+    ref_x = s0.astype(np.float64)            # oracle state, never rounded
+    worst_r = worst_x = 0.0
+    for c in range(calls):
+        tok = gen.make_decode_tokens(cfg, c * S, S)
+        dev = {n: gu.to_dev(np.ascontiguousarray(np.moveaxis(a, 0, 1)), torch.bfloat16) for n, a in tok.items()}
+        o = qd.recurrent_steps(dev["q"], dev["k"], dev["v"], dev["beta"], dev["alpha"], dev["lam"], state.t)
+        o_r, ref_r = orc.decode(ref_r, tok["q"], tok["k"], tok["v"], tok["beta"], tok["alpha"], tok["lam"])
+        ref_r = gen.round_bf16(ref_r.astype(np.float32)).astype(np.float64)
+        o_x, ref_x = orc.decode(ref_x, tok["q"], tok["k"], tok["v"], tok["beta"], tok["alpha"], tok["lam"])
+        if c % 10 == 9 or c == calls - 1:
+            torch.cuda.synchronize()
+            worst_r = max(worst_r, gu.rel_err(o, np.moveaxis(o_r, 0, 1)))
+            worst_x = max(worst_x, gu.rel_err(o, np.moveaxis(o_x, 0, 1)))
+    torch.cuda.synchronize()
+    assert state.intact()
+    assert worst_r <= 2e-2 and gu.rel_err(state.t.float(), ref_r) <= 2e-2, (worst_r,)
+    assert worst_x <= 2e-2 and gu.rel_err(state.t.float(), ref_x) <= 2e-2, (worst_x,)
